@@ -1,0 +1,185 @@
+/*
+ * libcsb -- compressed-structured-block (CSB) sparse products and the fused
+ * LSTM / GRU time loop on one NVIDIA B200 (sm_100a).
+ *
+ * The operations follow "CSB-RNN" (arXiv 2005.05758):
+ *   - the CSB matrix and its storage format: Section 3.1.1;
+ *   - the CSB matrix-vector product (the CSB-Engine's job): Sections 4.2, 4.3.1;
+ *   - the recurrent cell around it (products, sigmoid, tanh, element-wise
+ *     product and sum, the c/h context link): Section 2.1.
+ *
+ * Conventions for every entry point
+ *   - Returns CSB_OK (0) or a negative csb_status; no C++ exception crosses the
+ *     boundary.  csb_last_error() gives a thread-local detail string.
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA
+ *     global memory on the device the matrix was encoded for.  All buffers are
+ *     owned by the caller and are neither retained nor freed by the library;
+ *     handles (csb_matrix_t) are owned by the library until csb_free().
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Product calls only enqueue work; the recurrent calls additionally wait
+ *     for their status word unless CSB_FLAG_ASYNC is given.
+ *   - Matrix shape R x C: rows are output neurons, columns input neurons;
+ *     blocks are block_r x block_c (1..256 each), block b = bi * nbc + bj in
+ *     row-major block order; a short last block is allowed.
+ *   - There is no CPU fallback: a call that needs the GPU fails with
+ *     CSB_ERR_CUDA / CSB_ERR_UNSUPPORTED when no sm_100 device is present.
+ */
+#ifndef CSB_H_
+#define CSB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum csb_status {
+    CSB_OK = 0,
+    CSB_ERR_INVALID_ARG = -1,  /* null pointer, negative size, bad enum            */
+    CSB_ERR_SHAPE = -2,        /* shapes of the arguments do not fit each other    */
+    CSB_ERR_DTYPE = -3,        /* unknown value type                               */
+    CSB_ERR_ALLOC = -4,        /* host or device allocation failed                 */
+    CSB_ERR_CUDA = -5,         /* a CUDA runtime call failed (see csb_last_error)  */
+    CSB_ERR_LAUNCH = -6,       /* the persistent grid cannot be co-resident        */
+    CSB_ERR_TIMEOUT = -7,      /* a bounded device-side wait expired               */
+    CSB_ERR_UNSUPPORTED = -8   /* valid request this build does not implement      */
+} csb_status;
+
+enum { CSB_F32 = 0, CSB_F16 = 1 };          /* storage type of the packed values */
+enum { CSB_FLAG_ASYNC = 1u,                 /* recurrent calls: do not wait for the status word */
+       CSB_FLAG_HOST_IO = 2u };             /* recurrent calls: sequence and state pointers are host memory */
+
+typedef struct csb_matrix csb_matrix_t;     /* opaque: canonical arrays + device layout + schedule */
+
+/* Tuning knobs of the one-shot planning step; zero means "library default". */
+typedef struct csb_plan_opts {
+    int ctas;            /* persistent grid size of the product kernels (default: SM count) */
+    int warps_per_cta;   /* warps per CTA (default 16)                                       */
+    int stage_bytes;     /* bytes per shared-memory ring stage of one warp (default 3072)    */
+    int stages;          /* ring depth per warp (default 3)                                  */
+} csb_plan_opts;
+
+/* The canonical CSB arrays of Section 3.1.1 (n{}, m{}, RowIdx{}, ColIdx{}, Val{}) plus
+ * the offsets the paper leaves out.  All pointers are host memory borrowed from the
+ * handle and stay valid until csb_free(). */
+typedef struct csb_view {
+    int64_t rows, cols;
+    int32_t block_r, block_c;
+    int64_t nbr, nbc, nblk, nnz;
+    int32_t val_dtype;           /* CSB_F32 | CSB_F16                                  */
+    const uint16_t* m;           /* [nblk] kept rows per block                         */
+    const uint16_t* n;           /* [nblk] kept columns per block                      */
+    const uint8_t* row_idx;      /* in-block indices, 0-based, ascending, concatenated */
+    const uint8_t* col_idx;
+    const uint64_t* val_off;     /* [nblk+1] exclusive prefix sum of m*n               */
+    const uint32_t* ridx_off;    /* [nblk+1] exclusive prefix sum of m                 */
+    const uint32_t* cidx_off;    /* [nblk+1] exclusive prefix sum of n                 */
+    const void* val;             /* [nnz] kernel matrices, row-major inside a block    */
+} csb_view_t;
+
+/* Figures derived at encode / plan time. */
+typedef struct csb_info {
+    int64_t nnz;                 /* stored weights, sum of m_b * n_b                        */
+    double pruning_rate;         /* rows * cols / nnz (Section 1)                           */
+    double nio;                  /* normalized index overhead, sum(m+n) / nnz (Sec. 6.2.1)  */
+    int64_t algorithmic_bytes;   /* values + index lists + 6-byte block headers             */
+    int64_t device_stream_bytes; /* bytes of the private device layout actually streamed    */
+    int32_t plan_ctas, plan_warps;
+    double balance;              /* mean / max of the per-warp scheduled cost (1 = perfect) */
+} csb_info_t;
+
+/*
+ * csb_encode -- build the CSB storage format (Section 3.1.1) from a dense weight and
+ * per-block keep masks, and plan its execution on `device`.
+ *   dense     host, float32, rows x cols, row stride ld (>= cols) elements.
+ *   row_keep  host, [nblk * block_r] bytes; byte b*block_r + i != 0 keeps in-block row i of
+ *             block b.  col_keep likewise, [nblk * block_c].  Bytes that fall beyond the
+ *             matrix edge in a short last block are ignored.
+ *   val_dtype CSB_F32 keeps the bit patterns; CSB_F16 rounds to binary16, nearest-even.
+ *   device    CUDA device ordinal, or -1 for the host-side arrays only (csb_view works,
+ *             products fail with CSB_ERR_UNSUPPORTED).
+ *   opts      may be NULL.
+ * A block with no kept row or no kept column stores no values but still lists the other
+ * side's indices.  On success *out owns copies of everything; the inputs may be released.
+ * Errors: INVALID_ARG (null, sizes <= 0, ld < cols, blocks outside 1..256), DTYPE, ALLOC, CUDA.
+ */
+int csb_encode(const float* dense, int64_t rows, int64_t cols, int64_t ld, int block_r, int block_c,
+               const uint8_t* row_keep, const uint8_t* col_keep, int val_dtype, int device,
+               const csb_plan_opts* opts, csb_matrix_t** out);
+
+/* Borrow the canonical arrays (host memory, valid until csb_free). */
+int csb_view(const csb_matrix_t* A, csb_view_t* out);
+
+/* Encoder / planner statistics. */
+int csb_info(const csb_matrix_t* A, csb_info_t* out);
+
+/* Release a handle and everything planned from it (NULL is a no-op).  Must not run while
+ * work using the handle is still in flight. */
+void csb_free(csb_matrix_t* A);
+
+/*
+ * csb_spmv -- y = A . x, the CSB matrix-vector product (Sections 4.2, 4.3.1): per block the kept
+ * inputs are read through ColIdx, multiplied by the kernel matrix and accumulated into the
+ * outputs through RowIdx; blocks of a block-row accumulate into the same outputs.
+ *   x  device, float32 [cols];  y  device, float32 [rows], overwritten (rows kept in no block
+ *   become exactly 0).  fp32 accumulation, fixed summation order (bit-reproducible).
+ * Asynchronous on `stream`.  Calls on the same handle must not overlap on the GPU: they share
+ * the handle's scratch for partial block-row sums.
+ */
+int csb_spmv(const csb_matrix_t* A, const float* x, float* y, void* stream);
+
+/*
+ * csb_spmm -- Y[b, :] = A . X[b, :] for b < batch (the same product with a batch of vectors).
+ *   X  device, float32, batch rows of `cols` values, row stride ldx >= cols;
+ *   Y  device, float32, batch rows of `rows` values, row stride ldy >= rows, overwritten.
+ * batch = 0 is a no-op.  Same ordering / overlap rules as csb_spmv.
+ */
+int csb_spmm(const csb_matrix_t* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy,
+             void* stream);
+
+/*
+ * csb_lstm_forward -- a stack of LSTM layers over a whole sequence in one persistent kernel
+ * (Section 2.1; one CSB product per layer and step, gate arithmetic fused behind it).
+ *   W[l]     CSB matrix [4*H, I_l + H], I_0 = I, I_l = H above; stacked gate rows i, f, g, o;
+ *            columns [0, I_l) multiply the layer input, the rest multiply h_{t-1}.
+ *   bias[l]  device float32 [4*H], or NULL (bias may itself be NULL = no bias anywhere).
+ *   x        float32 [T, B, I];  h0, c0  float32 [L, B, H] or NULL (zeros);
+ *   y        float32 [T, B, H] top layer's h_t, or NULL;  hT, cT  float32 [L, B, H] or NULL.
+ *   Per layer and step:  z = W.[u_t ; h_{t-1}] + b;  c_t = s(z_f)*c_{t-1} + s(z_i)*tanh(z_g);
+ *   h_t = s(z_o)*tanh(c_t), with s the logistic function and u_t the layer's input.
+ *   flags    CSB_FLAG_ASYNC: return without waiting (the status word is then not checked).
+ *            CSB_FLAG_HOST_IO: x, h0, c0, y, hT, cT are HOST pointers; the call copies them
+ *            through device staging buffers on `stream` and waits for the result.
+ * The first call for a given (W..., B) builds and caches the time-loop schedule and its
+ * device state (allocates, synchronises); later calls reuse it.  T = 0 or B = 0 is a no-op.
+ * Errors: SHAPE (rows != 4H, cols != I_l + H, layers disagree), LAUNCH (grid cannot be
+ * co-resident; nothing was launched), TIMEOUT (the bounded grid barrier gave up; outputs are
+ * undefined, the context stays usable), CUDA.
+ */
+int csb_lstm_forward(int n_layers, const csb_matrix_t* const* W, const float* const* bias,
+                     const float* x, int64_t T, int B, const float* h0, const float* c0,
+                     float* y, float* hT, float* cT, unsigned flags, void* stream);
+
+/*
+ * csb_gru_forward -- same for GRU layers.  W[l] is [3*H, I_l + H], rows r, z, n; bias[l] is
+ * device float32 [4*H] = b_r, b_z, b_in, b_hn.  The reset gate acts after the recurrent product:
+ *   r = s(zx_r + zh_r + b_r);  z = s(zx_z + zh_z + b_z);
+ *   n = tanh(zx_n + b_in + r * (zh_n + b_hn));  h_t = (1 - z) * n + z * h_{t-1},
+ * where zx / zh are the parts of the product over the input / hidden columns.
+ */
+int csb_gru_forward(int n_layers, const csb_matrix_t* const* W, const float* const* bias,
+                    const float* x, int64_t T, int B, const float* h0, float* y, float* hT,
+                    unsigned flags, void* stream);
+
+/* Short text for a status code; never NULL. */
+const char* csb_strerror(int status);
+
+/* Detail of the calling thread's most recent failure ("" if none); valid until that thread's
+ * next library call. */
+const char* csb_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CSB_H_ */

@@ -1,0 +1,188 @@
+"""ctypes binding of libcsb: argument marshalling only.
+
+Every function mirrors one entry point of include/csb.h under the same name.
+Device buffers are torch CUDA tensors (torch is used for device memory and
+streams only); host buffers are numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcsb.so")
+if not os.path.exists(_LIB_PATH):
+    raise ImportError("libcsb.so is not built: run `python -m paper_2005_05758_b200.build` "
+                      "(there is no CPU fallback)")
+lib = C.CDLL(_LIB_PATH)
+
+CSB_F32, CSB_F16 = 0, 1
+CSB_FLAG_ASYNC, CSB_FLAG_HOST_IO = 1, 2
+_DT = {"f32": CSB_F32, "f16": CSB_F16}
+
+
+class csb_plan_opts(C.Structure):
+    _fields_ = [("ctas", C.c_int), ("warps_per_cta", C.c_int), ("stage_bytes", C.c_int), ("stages", C.c_int)]
+
+
+class csb_view_t(C.Structure):
+    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("block_r", C.c_int32), ("block_c", C.c_int32),
+                ("nbr", C.c_int64), ("nbc", C.c_int64), ("nblk", C.c_int64), ("nnz", C.c_int64),
+                ("val_dtype", C.c_int32),
+                ("m", C.POINTER(C.c_uint16)), ("n", C.POINTER(C.c_uint16)),
+                ("row_idx", C.POINTER(C.c_uint8)), ("col_idx", C.POINTER(C.c_uint8)),
+                ("val_off", C.POINTER(C.c_uint64)), ("ridx_off", C.POINTER(C.c_uint32)),
+                ("cidx_off", C.POINTER(C.c_uint32)), ("val", C.c_void_p)]
+
+
+class csb_info_t(C.Structure):
+    _fields_ = [("nnz", C.c_int64), ("pruning_rate", C.c_double), ("nio", C.c_double),
+                ("algorithmic_bytes", C.c_int64), ("device_stream_bytes", C.c_int64),
+                ("plan_ctas", C.c_int32), ("plan_warps", C.c_int32), ("balance", C.c_double)]
+
+
+_P = C.c_void_p
+lib.csb_encode.argtypes = [_P, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, _P, _P, C.c_int, C.c_int,
+                           C.POINTER(csb_plan_opts), C.POINTER(_P)]
+lib.csb_view.argtypes = [_P, C.POINTER(csb_view_t)]
+lib.csb_info.argtypes = [_P, C.POINTER(csb_info_t)]
+lib.csb_free.argtypes = [_P]
+lib.csb_free.restype = None
+lib.csb_spmv.argtypes = [_P, _P, _P, _P]
+lib.csb_spmm.argtypes = [_P, _P, C.c_int64, C.c_int, _P, C.c_int64, _P]
+lib.csb_lstm_forward.argtypes = [C.c_int, C.POINTER(_P), C.POINTER(_P), _P, C.c_int64, C.c_int, _P, _P, _P, _P, _P,
+                                 C.c_uint, _P]
+lib.csb_gru_forward.argtypes = [C.c_int, C.POINTER(_P), C.POINTER(_P), _P, C.c_int64, C.c_int, _P, _P, _P,
+                                C.c_uint, _P]
+lib.csb_strerror.argtypes = [C.c_int]
+lib.csb_strerror.restype = C.c_char_p
+lib.csb_last_error.restype = C.c_char_p
+for _f in ("csb_encode", "csb_view", "csb_info", "csb_spmv", "csb_spmm", "csb_lstm_forward", "csb_gru_forward"):
+    getattr(lib, _f).restype = C.c_int
+
+
+class CsbError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        super().__init__("%s (%d): %s" % (lib.csb_strerror(status).decode(), status,
+                                         lib.csb_last_error().decode()))
+
+
+def _check(status: int) -> None:
+    if status != 0:
+        raise CsbError(status)
+
+
+def _ptr(t) -> Optional[int]:
+    """Address of a torch tensor / numpy array (None stays NULL)."""
+    if t is None:
+        return None
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return getattr(stream, "cuda_stream", stream)
+
+
+class CsbMatrix:
+    """Owner of a csb_matrix_t handle."""
+
+    def __init__(self, handle: int):
+        self.handle = handle
+
+    def view(self) -> dict:
+        v = csb_view_t()
+        _check(lib.csb_view(self.handle, C.byref(v)))
+        nblk, nnz = v.nblk, v.nnz
+
+        def arr(p, n, dt):
+            if n == 0:
+                return np.zeros(0, dt)
+            return np.ctypeslib.as_array(C.cast(p, C.POINTER(C.c_uint8)), shape=(n * np.dtype(dt).itemsize,)).view(dt).copy()
+
+        ro = arr(v.ridx_off, nblk + 1, np.uint32)
+        co = arr(v.cidx_off, nblk + 1, np.uint32)
+        vdt = np.float16 if v.val_dtype == CSB_F16 else np.float32
+        return {"rows": v.rows, "cols": v.cols, "block_r": v.block_r, "block_c": v.block_c, "nbr": v.nbr,
+                "nbc": v.nbc, "nnz": nnz, "val_dtype": "f16" if v.val_dtype == CSB_F16 else "f32",
+                "m": arr(v.m, nblk, np.uint16), "n": arr(v.n, nblk, np.uint16),
+                "row_idx": arr(v.row_idx, int(ro[-1]), np.uint8), "col_idx": arr(v.col_idx, int(co[-1]), np.uint8),
+                "val_off": arr(v.val_off, nblk + 1, np.uint64), "ridx_off": ro, "cidx_off": co,
+                "val": arr(v.val, nnz, vdt)}
+
+    def info(self) -> dict:
+        o = csb_info_t()
+        _check(lib.csb_info(self.handle, C.byref(o)))
+        return {k: getattr(o, k) for k, _ in csb_info_t._fields_}
+
+    def free(self) -> None:
+        if self.handle:
+            lib.csb_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def csb_encode(dense: np.ndarray, block_r: int, block_c: int, row_keep: np.ndarray, col_keep: np.ndarray,
+               val_dtype: str = "f16", device: int = 0, opts: Optional[dict] = None) -> CsbMatrix:
+    dense = np.ascontiguousarray(dense, dtype=np.float32)
+    rk = np.ascontiguousarray(row_keep, dtype=np.uint8)
+    ck = np.ascontiguousarray(col_keep, dtype=np.uint8)
+    rows, cols = dense.shape
+    nblk = -(-rows // block_r) * -(-cols // block_c) if block_r > 0 and block_c > 0 else 0
+    if block_r > 0 and block_c > 0 and (rk.size != nblk * block_r or ck.size != nblk * block_c):
+        raise ValueError("keep masks must hold nblk*block_r and nblk*block_c bytes")
+    o = csb_plan_opts(**opts) if opts else None
+    out = _P()
+    _check(lib.csb_encode(dense.ctypes.data, rows, cols, cols, block_r, block_c, rk.ctypes.data, ck.ctypes.data,
+                          _DT[val_dtype] if isinstance(val_dtype, str) else val_dtype, device,
+                          C.byref(o) if o else None, C.byref(out)))
+    return CsbMatrix(out.value)
+
+
+def csb_spmv(A: CsbMatrix, x, y, stream=None) -> None:
+    _check(lib.csb_spmv(A.handle, _ptr(x), _ptr(y), _stream(stream)))
+
+
+def csb_spmm(A: CsbMatrix, X, Y, stream=None) -> None:
+    batch = X.shape[0]
+    _check(lib.csb_spmm(A.handle, _ptr(X), X.stride(0) if batch else 0, batch, _ptr(Y),
+                        Y.stride(0) if batch else 0, _stream(stream)))
+
+
+def _ptr_array(items: Sequence, n: int):
+    arr = (_P * n)()
+    for i in range(n):
+        arr[i] = _ptr(items[i]) if not isinstance(items[i], CsbMatrix) else items[i].handle
+    return arr
+
+
+def csb_lstm_forward(W: Sequence[CsbMatrix], bias, x, h0, c0, y, hT, cT, flags: int = 0, stream=None) -> None:
+    L = len(W)
+    T, B = (x.shape[0], x.shape[1])
+    b = _ptr_array(bias, L) if bias is not None else None
+    _check(lib.csb_lstm_forward(L, _ptr_array(W, L), b, _ptr(x), T, B, _ptr(h0), _ptr(c0), _ptr(y), _ptr(hT),
+                                _ptr(cT), flags, _stream(stream)))
+
+
+def csb_gru_forward(W: Sequence[CsbMatrix], bias, x, h0, y, hT, flags: int = 0, stream=None) -> None:
+    L = len(W)
+    T, B = (x.shape[0], x.shape[1])
+    b = _ptr_array(bias, L) if bias is not None else None
+    _check(lib.csb_gru_forward(L, _ptr_array(W, L), b, _ptr(x), T, B, _ptr(h0), _ptr(y), _ptr(hT), flags,
+                               _stream(stream)))
+
+
+# shorter aliases
+spmv, spmm, lstm_forward, gru_forward = csb_spmv, csb_spmm, csb_lstm_forward, csb_gru_forward

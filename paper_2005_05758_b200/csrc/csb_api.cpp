@@ -1,0 +1,123 @@
+// The C ABI of libcsb: argument checks, error strings, handle lifetime.
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <new>
+
+#include "csb_internal.hpp"
+
+namespace csb {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+}
+void clear_error() { g_err[0] = 0; }
+
+static std::atomic<uint64_t> g_uid{1};
+
+}  // namespace csb
+
+using namespace csb;
+
+extern "C" {
+
+const char* csb_strerror(int status) {
+    switch (status) {
+        case CSB_OK: return "ok";
+        case CSB_ERR_INVALID_ARG: return "invalid argument";
+        case CSB_ERR_SHAPE: return "shape mismatch";
+        case CSB_ERR_DTYPE: return "unknown value type";
+        case CSB_ERR_ALLOC: return "allocation failed";
+        case CSB_ERR_CUDA: return "CUDA runtime error";
+        case CSB_ERR_LAUNCH: return "grid cannot be launched co-resident";
+        case CSB_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case CSB_ERR_UNSUPPORTED: return "unsupported";
+        default: return "unknown status";
+    }
+}
+
+const char* csb_last_error(void) { return g_err; }
+
+int csb_encode(const float* dense, int64_t rows, int64_t cols, int64_t ld, int block_r, int block_c,
+               const uint8_t* row_keep, const uint8_t* col_keep, int val_dtype, int device,
+               const csb_plan_opts* opts, csb_matrix_t** out) {
+    clear_error();
+    if (!out) { set_error("out is NULL"); return CSB_ERR_INVALID_ARG; }
+    *out = nullptr;
+    if (!dense || !row_keep || !col_keep) { set_error("dense / row_keep / col_keep is NULL"); return CSB_ERR_INVALID_ARG; }
+    if (rows <= 0 || cols <= 0 || ld < cols) { set_error("rows=%lld cols=%lld ld=%lld", (long long)rows, (long long)cols, (long long)ld); return CSB_ERR_INVALID_ARG; }
+    if (rows > 0x7fffffff || cols > 0x7fffffff) { set_error("dimensions above 2^31-1 are not supported"); return CSB_ERR_UNSUPPORTED; }
+    if (block_r < 1 || block_r > 256 || block_c < 1 || block_c > 256) { set_error("block sizes must be 1..256, got %dx%d", block_r, block_c); return CSB_ERR_INVALID_ARG; }
+    if (val_dtype != CSB_F32 && val_dtype != CSB_F16) { set_error("val_dtype %d", val_dtype); return CSB_ERR_DTYPE; }
+    if (device < -1) { set_error("device %d", device); return CSB_ERR_INVALID_ARG; }
+    csb_matrix* A = new (std::nothrow) csb_matrix();
+    if (!A) { set_error("out of host memory"); return CSB_ERR_ALLOC; }
+    A->device = device;
+    A->uid = g_uid.fetch_add(1);
+    if (opts) A->opts = *opts;
+    int rc = encode_host(dense, rows, cols, ld, block_r, block_c, row_keep, col_keep, val_dtype, A);
+    if (rc == CSB_OK) rc = validate_host(A);
+    if (rc == CSB_OK && device >= 0) {
+        try { rc = plan_product(A); }
+        catch (const std::bad_alloc&) { set_error("out of host memory while planning"); rc = CSB_ERR_ALLOC; }
+    }
+    if (rc != CSB_OK) { csb_free(A); return rc; }
+    *out = A;
+    return CSB_OK;
+}
+
+int csb_view(const csb_matrix_t* A, csb_view_t* v) {
+    clear_error();
+    if (!A || !v) { set_error("NULL argument"); return CSB_ERR_INVALID_ARG; }
+    v->rows = A->rows; v->cols = A->cols; v->block_r = A->block_r; v->block_c = A->block_c;
+    v->nbr = A->nbr; v->nbc = A->nbc; v->nblk = A->nblk; v->nnz = A->nnz; v->val_dtype = A->val_dtype;
+    v->m = A->m.data(); v->n = A->n.data(); v->row_idx = A->row_idx.data(); v->col_idx = A->col_idx.data();
+    v->val_off = A->val_off.data(); v->ridx_off = A->ridx_off.data(); v->cidx_off = A->cidx_off.data();
+    v->val = A->val.data();
+    return CSB_OK;
+}
+
+int csb_info(const csb_matrix_t* A, csb_info_t* o) {
+    clear_error();
+    if (!A || !o) { set_error("NULL argument"); return CSB_ERR_INVALID_ARG; }
+    const int64_t idx = (int64_t)A->ridx_off[A->nblk] + (int64_t)A->cidx_off[A->nblk];
+    o->nnz = A->nnz;
+    o->pruning_rate = A->nnz ? (double)A->rows * (double)A->cols / (double)A->nnz : 0.0;
+    o->nio = A->nnz ? (double)idx / (double)A->nnz : 0.0;
+    o->algorithmic_bytes = A->nnz * val_size(A->val_dtype) + idx + 6 * A->nblk;
+    o->device_stream_bytes = A->product.stream_bytes;
+    o->plan_ctas = A->product.ctas;
+    o->plan_warps = A->product.warps;
+    o->balance = A->product.balance;
+    return CSB_OK;
+}
+
+void csb_free(csb_matrix_t* A) {
+    if (!A) return;
+    drop_rnn_plans(A);
+    free_product(A);
+    delete A;
+}
+
+int csb_spmm(const csb_matrix_t* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream) {
+    clear_error();
+    if (!A) { set_error("A is NULL"); return CSB_ERR_INVALID_ARG; }
+    if (batch < 0) { set_error("batch %d", batch); return CSB_ERR_INVALID_ARG; }
+    if (batch == 0) return CSB_OK;
+    if (!X || !Y) { set_error("X or Y is NULL"); return CSB_ERR_INVALID_ARG; }
+    if (ldx < A->cols || ldy < A->rows) { set_error("ldx=%lld < cols or ldy=%lld < rows", (long long)ldx, (long long)ldy); return CSB_ERR_SHAPE; }
+    if (A->device < 0) { set_error("matrix was encoded host-only (device = -1)"); return CSB_ERR_UNSUPPORTED; }
+    return launch_product(A, X, ldx, batch, Y, ldy, stream);
+}
+
+int csb_spmv(const csb_matrix_t* A, const float* x, float* y, void* stream) {
+    if (!A) { clear_error(); set_error("A is NULL"); return CSB_ERR_INVALID_ARG; }
+    return csb_spmm(A, x, A->cols, 1, y, A->rows, stream);
+}
+
+}  // extern "C"

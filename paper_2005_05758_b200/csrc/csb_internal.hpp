@@ -1,0 +1,152 @@
+// Internal declarations shared by the host-side pieces of libcsb (encoder,
+// planner, launch glue).  Nothing here is part of the public C ABI.
+#pragma once
+
+#include <cstdint>
+#include <cstring>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "../../include/csb.h"
+
+namespace csb {
+
+// ---- error plumbing -------------------------------------------------------
+void set_error(const char* fmt, ...);   // formats into the thread-local detail string
+void clear_error();
+
+// ---- device stream format -------------------------------------------------
+// The private device layout is a byte stream per warp, cut into chunks that one
+// bulk copy moves into a shared-memory ring stage.  A chunk holds whole items;
+// an item is one block (or a slice of one) of the CSB matrix:
+//
+//   ItemHeader (16 B)
+//   col_idx[nk]  uint8   gather indices, relative to xbase
+//   row_idx[mr]  uint8   scatter indices, relative to zbase      (padded to 4 B)
+//   values       nk columns of RL "row words" each, column-major (k-major):
+//                  f16: a word is two consecutive kept rows (half2), RL = ceil(mr/2)
+//                  f32: a word is one kept row, RL = mr
+//                padding rows inside the last word are zero      (item padded to 16 B)
+//
+// Column-major kernel matrices let one lane own a pair of output rows for the
+// whole item, so products need no cross-lane reduction except across the few
+// lane groups that split the columns.
+struct ItemHeader {
+    uint16_t nk;       // kept columns in this item (<= kMaxNk)
+    uint16_t mr;       // kept rows in this item (<= 64 for f16, <= 32 for f32)
+    uint32_t xbase;    // first column of the block in the gathered vector
+    uint32_t zbase;    // first accumulator slot / matrix row of the block
+    uint32_t tail;     // bits 0..1 flush kind, bit 2 source select (recurrent), bits 3.. slot id
+};
+static_assert(sizeof(ItemHeader) == 16, "header is one 16-byte word");
+
+enum : uint32_t { kFlushNone = 0, kFlushDirect = 1, kFlushPartial = 2, kSrcRecurrent = 4, kSlotShift = 3 };
+enum { kMaxNk = 64, kItemAlign = 16 };
+
+struct Chunk {
+    uint32_t off16;    // offset of the chunk in the stream, in 16-byte units
+    uint32_t bytes;    // multiple of 16, <= stage_bytes
+};
+
+// Host image of one planned stream (before upload).
+struct StreamPlan {
+    std::vector<uint8_t> bytes;            // all chunks back to back
+    std::vector<Chunk> chunks;
+    std::vector<uint32_t> warp_chunk_begin; // [n_warps + 1]
+    std::vector<double> warp_cost;
+    int n_warps = 0;
+};
+
+// Planned product (SpMV / SpMM) on the device.
+struct ProductPlan {
+    int ctas = 0, warps = 0, stage_bytes = 0, stages = 0;
+    int x_in_smem = 0;
+    size_t smem_bytes = 0;
+    uint8_t* d_stream = nullptr;
+    Chunk* d_chunks = nullptr;
+    uint32_t* d_warp_chunk_begin = nullptr;
+    // partial block-row sums: slots [part_base[bi], part_base[bi] + part_count[bi]) belong to block-row bi
+    uint32_t* d_part_base = nullptr;
+    uint32_t* d_part_count = nullptr;
+    uint32_t* d_arrivals = nullptr;        // [nbr], zero between launches
+    float* d_partials = nullptr;           // [n_slots * block_r * max_batch_tile]
+    uint32_t n_slots = 0;
+    int n_warps = 0;                       // warps the stream was cut for
+    uint32_t* h_status = nullptr;          // mapped host word the kernels raise on a bounded-wait expiry
+    uint32_t* d_status = nullptr;
+    int64_t stream_bytes = 0;
+    double balance = 1.0;
+};
+
+struct Planner;                            // csb_plan.cpp
+struct RnnPlan;                            // csb_rnn.cu
+
+}  // namespace csb
+
+// The opaque handle of the C ABI.
+struct csb_matrix {
+    int64_t rows = 0, cols = 0;
+    int block_r = 0, block_c = 0;
+    int64_t nbr = 0, nbc = 0, nblk = 0, nnz = 0;
+    int val_dtype = CSB_F16;
+    int device = -1;
+    csb_plan_opts opts{};
+    // canonical arrays (Section 3.1.1 + offsets)
+    std::vector<uint16_t> m, n;
+    std::vector<uint8_t> row_idx, col_idx;
+    std::vector<uint64_t> val_off;
+    std::vector<uint32_t> ridx_off, cidx_off;
+    std::vector<uint8_t> val;              // nnz * (2 | 4) bytes
+    // device side
+    csb::ProductPlan product;
+    int sm_count = 0;
+    size_t smem_optin = 0;
+    uint64_t uid = 0;                      // identity for the recurrent-plan cache
+};
+
+namespace csb {
+
+inline int val_size(int dt) { return dt == CSB_F16 ? 2 : 4; }
+inline int rows_per_word(int dt) { return dt == CSB_F16 ? 2 : 1; }
+inline int max_item_rows(int dt) { return dt == CSB_F16 ? 64 : 32; }
+
+// csb_encode.cpp
+int encode_host(const float* dense, int64_t rows, int64_t cols, int64_t ld, int br, int bc,
+                const uint8_t* row_keep, const uint8_t* col_keep, int val_dtype, csb_matrix* A);
+int validate_host(const csb_matrix* A);
+
+// csb_plan.cpp -- one item source: (block, row subset, column range)
+struct ItemSpec {
+    int64_t block;       // canonical block id
+    int r0, r1;          // range [r0, r1) into the block's kept-row list
+    int k0, k1;          // range [k0, k1) into the block's kept-column list
+    uint32_t xbase, zbase;
+    int ridx_bias;       // subtracted from the in-block row index before it is stored
+    uint32_t tail;       // flush kind / source / slot, ready for the header
+};
+size_t item_bytes(const csb_matrix* A, const ItemSpec& it);
+void emit_item(const csb_matrix* A, const ItemSpec& it, std::vector<uint8_t>& out);
+// Cut per-warp item lists into chunks and lay them out back to back.
+void build_stream(const csb_matrix* A, const std::vector<std::vector<ItemSpec>>& per_warp,
+                  int stage_bytes, StreamPlan* out);
+void slice_block(const csb_matrix* A, int64_t b, int r0, int r1, int k0, int k1, int value_budget,
+                 ItemSpec proto, std::vector<ItemSpec>* out);
+struct ProductHostPlan {
+    StreamPlan stream;
+    std::vector<uint32_t> part_base, part_count;   // per block-row
+    uint32_t n_slots = 0;
+    double balance = 1.0;
+};
+int plan_product_host(const csb_matrix* A, int n_warps, int stage_bytes, ProductHostPlan* out);
+
+// csb_product.cu
+int plan_product(csb_matrix* A);           // plans, uploads, fills A->product
+void free_product(csb_matrix* A);
+int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy,
+                   void* stream);
+
+// csb_rnn.cu
+void drop_rnn_plans(const csb_matrix* A);  // forget cached time-loop plans that use A
+
+}  // namespace csb

@@ -1,0 +1,333 @@
+// CSB sparse product kernel (SpMV and the CUDA-core batched form) and its launch glue.
+//
+// What the paper's CSB-Engine does per block (Section 4.3.1) -- read the kept inputs
+// through ColIdx, multiply by the kernel matrix, accumulate into the outputs through
+// RowIdx, sum along the block-row -- is done here by independent warps of a persistent
+// grid.  Every warp owns one contiguous run of the planned item stream and pulls it
+// through its own shared-memory ring with bulk asynchronous copies, so global memory is
+// read once, in large aligned pieces, while the irregular indexing happens on chip.
+#include <algorithm>
+#include <cstdio>
+
+#include "csb_device.cuh"
+#include "csb_internal.hpp"
+
+namespace csb {
+
+struct ProductArgs {
+    const uint8_t* stream;
+    const Chunk* chunks;
+    const uint32_t* warp_chunk_begin;
+    const uint32_t* part_base;
+    const uint32_t* part_count;
+    uint32_t* arrivals;
+    float* partials;
+    const float* X;
+    float* Y;
+    long long ldx, ldy;
+    uint32_t* status;
+    int n_warps, nb, rows, cols, block_r, stage_bytes, stages, x_in_smem;
+};
+
+__host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t)15; }
+
+// Shared-memory carve-up, identical on host and device.
+struct ProductSmem {
+    size_t ring, bars, zs, xg, xs, total;
+    int zs_stride;
+    __host__ __device__ ProductSmem(int W, int stages, int stage_bytes, int block_r, int BT, int cols_in_smem) {
+        zs_stride = block_r * BT;
+        ring = 0;
+        bars = ring + (size_t)W * stages * stage_bytes;
+        zs = align16(bars + (size_t)W * stages * 8);
+        xg = align16(zs + (size_t)W * zs_stride * 4);
+        xs = align16(xg + (size_t)W * kMaxNk * BT * 4);
+        total = align16(xs + (size_t)cols_in_smem * 4);
+    }
+};
+
+template <typename T, int BT>
+__global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    constexpr int R = WordTraits<T>::kRows;
+    const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const ProductSmem L(W, a.stages, a.stage_bytes, a.block_r, BT, a.x_in_smem ? a.cols : 0);
+    uint8_t* ring = smem + L.ring + (size_t)warp * a.stages * a.stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.bars) + warp * a.stages;
+    float* zs = reinterpret_cast<float*>(smem + L.zs) + warp * L.zs_stride;
+    float* xg = reinterpret_cast<float*>(smem + L.xg) + warp * kMaxNk * BT;
+    const float* xs = reinterpret_cast<const float*>(smem + L.xs);
+
+    const int gw = blockIdx.x * W + warp;
+    uint32_t c0 = 0, c1 = 0;
+    if (gw < a.n_warps) { c0 = a.warp_chunk_begin[gw]; c1 = a.warp_chunk_begin[gw + 1]; }
+
+    if (lane == 0) {
+        for (int s = 0; s < a.stages; ++s) mbar_init(&bars[s], 1);
+        mbar_fence_init();
+        for (int s = 0; s < a.stages && c0 + s < c1; ++s) {
+            const Chunk ch = a.chunks[c0 + s];
+            mbar_expect_tx(&bars[s], ch.bytes);
+            bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)ch.off16 * 16, ch.bytes, &bars[s]);
+        }
+    }
+    for (int i = lane; i < L.zs_stride; i += 32) zs[i] = 0.f;
+    if (a.x_in_smem) {
+        float* xw = reinterpret_cast<float*>(smem + L.xs);
+        for (int i = threadIdx.x; i < a.cols; i += blockDim.x) xw[i] = __ldg(a.X + i);
+        __syncthreads();
+    } else {
+        __syncwarp();
+    }
+
+    bool dead = false;
+    Chunk cur = (c0 < c1) ? a.chunks[c0] : Chunk{0, 0};
+    for (uint32_t c = c0; c < c1; ++c) {
+        const int s = (int)((c - c0) % (uint32_t)a.stages);
+        const uint32_t parity = ((c - c0) / (uint32_t)a.stages) & 1u;
+        const Chunk nxt = (c + 1 < c1) ? a.chunks[c + 1] : Chunk{0, 0};
+        const Chunk refill = (c + a.stages < c1) ? a.chunks[c + a.stages] : Chunk{0, 0};
+        if (!mbar_wait_bounded(&bars[s], parity)) { dead = true; }
+        dead = __any_sync(0xffffffffu, dead);
+        if (dead) {
+            // report, then give the copies still in flight a bounded chance to land before leaving
+            if (lane == 0) {
+                *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout;
+                for (uint32_t j = c + 1; j < c1 && j < c + (uint32_t)a.stages; ++j)
+                    mbar_wait_bounded(&bars[(j - c0) % (uint32_t)a.stages], ((j - c0) / (uint32_t)a.stages) & 1u);
+            }
+            break;
+        }
+
+        const uint8_t* p = ring + (size_t)s * a.stage_bytes;
+        const uint8_t* end = p + cur.bytes;
+        while (p < end) {
+            const uint4 h = *reinterpret_cast<const uint4*>(p);
+            const int nk = (int)(h.x & 0xffffu), mr = (int)(h.x >> 16);
+            const uint32_t xbase = h.y, zbase = h.z, tail = h.w;
+            const uint8_t* cidx = p + 16;
+            const uint8_t* ridx = cidx + nk;
+            const int idx_bytes = (nk + mr + 3) & ~3;
+            const uint32_t* vals = reinterpret_cast<const uint32_t*>(p + 16 + idx_bytes);
+            const int RLw = (mr + R - 1) / R;
+            p += (16 + idx_bytes + nk * RLw * 4 + 15) & ~15;
+
+            if (nk > 0 && mr > 0) {
+                for (int k = lane; k < nk; k += 32) {
+                    const uint32_t col = xbase + cidx[k];
+#pragma unroll
+                    for (int bt = 0; bt < BT; ++bt) {
+                        float v = 0.f;
+                        if (BT == 1) v = a.x_in_smem ? xs[col] : __ldg(a.X + col);
+                        else if (bt < a.nb) v = __ldg(a.X + (long long)bt * a.ldx + col);
+                        xg[k * BT + bt] = v;
+                    }
+                }
+                __syncwarp();
+                const LaneMap lm = lane_map<R>(mr, lane);
+                float acc[R][BT];
+#pragma unroll
+                for (int q = 0; q < R; ++q)
+#pragma unroll
+                    for (int bt = 0; bt < BT; ++bt) acc[q][bt] = 0.f;
+                item_mac<T, BT>(vals, nk, lm, lane, xg, acc);
+                if (lane < lm.RL) {
+#pragma unroll
+                    for (int q = 0; q < R; ++q) {
+                        const int r = lane * R + q;
+                        if (r < mr) {
+                            float* z = zs + (int)ridx[r] * BT;
+#pragma unroll
+                            for (int bt = 0; bt < BT; ++bt) z[bt] += acc[q][bt];
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+
+            const uint32_t flush = tail & 3u;
+            if (flush != kFlushNone) {
+                const int nrows = min(a.block_r, a.rows - (int)zbase);
+                if (flush == kFlushDirect) {
+                    for (int i = lane; i < nrows * BT; i += 32) {
+                        const int r = i / BT, bt = i % BT;
+                        if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = zs[i];
+                        zs[i] = 0.f;
+                    }
+                } else {
+                    const uint32_t slot = tail >> kSlotShift;
+                    const uint32_t bi = zbase / (uint32_t)a.block_r;
+                    float* dst = a.partials + (size_t)slot * a.block_r * BT;
+                    for (int i = lane; i < nrows * BT; i += 32) { __stcg(dst + i, zs[i]); zs[i] = 0.f; }
+                    __threadfence();
+                    __syncwarp();
+                    int last = 0;
+                    if (lane == 0) last = (atomicAdd(&a.arrivals[bi], 1u) == a.part_count[bi] - 1u);
+                    last = __shfl_sync(0xffffffffu, last, 0);
+                    if (last) {
+                        // this warp saw every other contributor arrive: add the partial sums in slot
+                        // order (fixed, so the result does not depend on who came last)
+                        __threadfence();
+                        const uint32_t pb = a.part_base[bi], pc = a.part_count[bi];
+                        for (int i = lane; i < nrows * BT; i += 32) {
+                            float sum = 0.f;
+                            for (uint32_t q = 0; q < pc; ++q) sum += __ldcg(a.partials + ((size_t)(pb + q) * a.block_r) * BT + i);
+                            const int r = i / BT, bt = i % BT;
+                            if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = sum;
+                        }
+                        if (lane == 0) a.arrivals[bi] = 0u;      // ready for the next launch
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        __syncwarp();
+        if (lane == 0 && refill.bytes) {
+            mbar_expect_tx(&bars[s], refill.bytes);
+            bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)refill.off16 * 16, refill.bytes, &bars[s]);
+        }
+        cur = nxt;
+    }
+}
+
+
+#define CSB_CUDA(call)                                                                     \
+    do {                                                                                   \
+        cudaError_t e_ = (call);                                                           \
+        if (e_ != cudaSuccess) {                                                           \
+            set_error("%s failed: %s", #call, cudaGetErrorString(e_));                     \
+            return e_ == cudaErrorMemoryAllocation ? CSB_ERR_ALLOC : CSB_ERR_CUDA;         \
+        }                                                                                  \
+    } while (0)
+
+template <typename V>
+static int upload(const std::vector<V>& h, V** d) {
+    *d = nullptr;
+    const size_t bytes = std::max<size_t>(h.size(), 1) * sizeof(V);
+    CSB_CUDA(cudaMalloc((void**)d, bytes));
+    if (!h.empty()) CSB_CUDA(cudaMemcpy(*d, h.data(), h.size() * sizeof(V), cudaMemcpyHostToDevice));
+    return CSB_OK;
+}
+
+static const int kBatchTiles[] = {8, 4, 1};
+enum { kMaxBatchTile = 8 };
+
+// Largest warp count per CTA whose carve-up fits the opt-in shared memory.
+static int fit_warps(const csb_matrix* A, int want, int BT, int cols_in_smem, size_t* smem) {
+    const ProductPlan& P = A->product;
+    for (int W = want; W >= 1; --W) {
+        const ProductSmem L(W, P.stages, P.stage_bytes, A->block_r, BT, cols_in_smem);
+        if (L.total <= A->smem_optin) { *smem = L.total; return W; }
+    }
+    return 0;
+}
+
+int plan_product(csb_matrix* A) {
+    ProductPlan& P = A->product;
+    int dev_prev = 0;
+    CSB_CUDA(cudaGetDevice(&dev_prev));
+    CSB_CUDA(cudaSetDevice(A->device));
+    cudaDeviceProp prop{};
+    CSB_CUDA(cudaGetDeviceProperties(&prop, A->device));
+    if (prop.major < 10) { set_error("device %d is sm_%d%d; this library is built for sm_100a", A->device, prop.major, prop.minor); return CSB_ERR_UNSUPPORTED; }
+    A->sm_count = prop.multiProcessorCount;
+    A->smem_optin = prop.sharedMemPerBlockOptin;
+    const int ctas = A->opts.ctas > 0 ? A->opts.ctas : A->sm_count;
+    const int wpc = std::min(16, A->opts.warps_per_cta > 0 ? A->opts.warps_per_cta : 16);
+    P.stage_bytes = ((A->opts.stage_bytes > 0 ? A->opts.stage_bytes : 3072) + 15) & ~15;
+    P.stage_bytes = std::max(P.stage_bytes, 1024);
+    P.stages = std::min(8, std::max(1, A->opts.stages > 0 ? A->opts.stages : 3));
+    // small matrices: no more warps than there is work for (about 2 KB of stream each)
+    const int64_t approx = A->nnz * val_size(A->val_dtype) + (int64_t)A->ridx_off[A->nblk] + A->cidx_off[A->nblk] + 16 * A->nblk;
+    const int64_t useful = std::max<int64_t>(1, approx / 2048);
+    const int n_warps = (int)std::min<int64_t>((int64_t)ctas * wpc, useful);
+    ProductHostPlan H;
+    int rc = plan_product_host(A, n_warps, P.stage_bytes, &H);
+    if (rc != CSB_OK) return rc;
+    P.warps = std::max(1, (n_warps + ctas - 1) / ctas);
+    P.ctas = (n_warps + P.warps - 1) / P.warps;
+    P.n_slots = H.n_slots;
+    P.balance = H.balance;
+    P.stream_bytes = (int64_t)H.stream.bytes.size();
+    P.n_warps = n_warps;
+    if ((rc = upload(H.stream.bytes, &P.d_stream)) != CSB_OK) return rc;
+    if ((rc = upload(H.stream.chunks, &P.d_chunks)) != CSB_OK) return rc;
+    if ((rc = upload(H.stream.warp_chunk_begin, &P.d_warp_chunk_begin)) != CSB_OK) return rc;
+    if ((rc = upload(H.part_base, &P.d_part_base)) != CSB_OK) return rc;
+    if ((rc = upload(H.part_count, &P.d_part_count)) != CSB_OK) return rc;
+    CSB_CUDA(cudaMalloc((void**)&P.d_arrivals, std::max<size_t>(A->nbr, 1) * 4));
+    CSB_CUDA(cudaMemset(P.d_arrivals, 0, std::max<size_t>(A->nbr, 1) * 4));
+    CSB_CUDA(cudaMalloc((void**)&P.d_partials, std::max<size_t>((size_t)P.n_slots * A->block_r * kMaxBatchTile, 1) * 4));
+    CSB_CUDA(cudaHostAlloc((void**)&P.h_status, 4, cudaHostAllocMapped));
+    *P.h_status = 0;
+    CSB_CUDA(cudaHostGetDevicePointer((void**)&P.d_status, P.h_status, 0));
+    CSB_CUDA(cudaDeviceSynchronize());
+    CSB_CUDA(cudaSetDevice(dev_prev));
+    return CSB_OK;
+}
+
+void free_product(csb_matrix* A) {
+    ProductPlan& P = A->product;
+    if (A->device < 0) return;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(A->device);
+    cudaFree(P.d_stream); cudaFree(P.d_chunks); cudaFree(P.d_warp_chunk_begin); cudaFree(P.d_part_base);
+    cudaFree(P.d_part_count); cudaFree(P.d_arrivals); cudaFree(P.d_partials);
+    if (P.h_status) cudaFreeHost(P.h_status);
+    P = ProductPlan{};
+    cudaSetDevice(prev);
+}
+
+template <typename T, int BT>
+static int launch_tile(const csb_matrix* A, ProductArgs a, cudaStream_t st) {
+    const ProductPlan& P = A->product;
+    size_t smem = 0;
+    int cols_in_smem = 0;
+    if (BT == 1 && (size_t)A->cols * 4 <= 64 * 1024) {
+        size_t s2 = 0;
+        if (fit_warps(A, P.warps, 1, (int)A->cols, &s2) == P.warps) cols_in_smem = (int)A->cols;
+    }
+    const int W = fit_warps(A, P.warps, BT, cols_in_smem, &smem);
+    if (W == 0) { set_error("a single warp's shared-memory ring does not fit (%d stages of %d bytes)", P.stages, P.stage_bytes); return CSB_ERR_LAUNCH; }
+    a.x_in_smem = cols_in_smem > 0;
+    const int ctas = (P.n_warps + W - 1) / W;
+    static bool configured[64] = {};                   // per device; setting it twice is harmless
+    if (A->device >= 64 || !configured[A->device]) {
+        CSB_CUDA(cudaFuncSetAttribute(csb_product_kernel<T, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)A->smem_optin));
+        if (A->device < 64) configured[A->device] = true;
+    }
+    csb_product_kernel<T, BT><<<ctas, W * 32, smem, st>>>(a);
+    CSB_CUDA(cudaGetLastError());
+    return CSB_OK;
+}
+
+int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream) {
+    const ProductPlan& P = A->product;
+    if (P.h_status && *P.h_status != 0) { set_error("an earlier product on this handle gave up waiting on the device (code %u)", *P.h_status); return CSB_ERR_TIMEOUT; }
+    int prev = 0;
+    CSB_CUDA(cudaGetDevice(&prev));
+    if (prev != A->device) CSB_CUDA(cudaSetDevice(A->device));
+    ProductArgs a{};
+    a.stream = P.d_stream; a.chunks = P.d_chunks; a.warp_chunk_begin = P.d_warp_chunk_begin;
+    a.part_base = P.d_part_base; a.part_count = P.d_part_count; a.arrivals = P.d_arrivals; a.partials = P.d_partials;
+    a.ldx = ldx; a.ldy = ldy; a.status = P.d_status; a.n_warps = P.n_warps;
+    a.rows = (int)A->rows; a.cols = (int)A->cols; a.block_r = A->block_r; a.stage_bytes = P.stage_bytes; a.stages = P.stages;
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = CSB_OK;
+    for (int b0 = 0; b0 < batch && rc == CSB_OK;) {
+        int bt = 1;
+        for (int cand : kBatchTiles) if (batch - b0 >= cand || cand == 1) { bt = cand; break; }
+        if (batch - b0 > 1 && bt == 1) bt = 4;          // 2 or 3 left: one padded tile of 4
+        a.X = X + (int64_t)b0 * ldx; a.Y = Y + (int64_t)b0 * ldy; a.nb = std::min(bt, batch - b0);
+        const bool h = A->val_dtype == CSB_F16;
+        if (bt == 8) rc = h ? launch_tile<__half, 8>(A, a, st) : launch_tile<float, 8>(A, a, st);
+        else if (bt == 4) rc = h ? launch_tile<__half, 4>(A, a, st) : launch_tile<float, 4>(A, a, st);
+        else rc = h ? launch_tile<__half, 1>(A, a, st) : launch_tile<float, 1>(A, a, st);
+        b0 += a.nb;
+    }
+    if (prev != A->device) cudaSetDevice(prev);
+    return rc;
+}
+
+}  // namespace csb

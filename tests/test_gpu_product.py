@@ -1,0 +1,94 @@
+"""Parity of csb_spmv / csb_spmm (CUDA, through the C ABI) with the float64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from oracle import csb_oracle as O
+from paper_2005_05758_b200 import binding
+
+pytestmark = pytest.mark.gpu
+
+RTOL = {"f16": 2e-3, "f32": 1e-5}   # max relative error per output allowed for each storage type
+
+
+def check_product(got, want, scale, vd):
+    """|got - want| <= rtol * max(|want|, 1e-2 * sum|w||x|): relative error per output, with
+    the forward-error scale of the row as the floor where the exact output is near zero."""
+    got = got.astype(np.float64)
+    tol = RTOL[vd] * np.maximum(np.abs(want), 1e-2 * scale)
+    bad = np.abs(got - want) > tol
+    assert not bad.any(), "max excess %g at %s" % (np.max(np.abs(got - want) / np.maximum(tol, 1e-300)),
+                                                   np.argwhere(bad)[:4].tolist())
+    assert np.all(got[scale == 0] == 0.0)      # rows kept nowhere (or meeting only zeros) are exact zeros
+
+
+def run_case(mat, X, opts=None, repeat=2):
+    A = binding.csb_encode(mat.dense, mat.block_r, mat.block_c, mat.row_keep, mat.col_keep, mat.val_dtype, 0, opts)
+    Xd = torch.from_numpy(X).cuda()
+    B = X.shape[0]
+    outs = []
+    for _ in range(repeat):
+        Y = torch.full((B, mat.rows), float("nan"), device="cuda")
+        if B == 1:
+            binding.csb_spmv(A, Xd[0], Y[0])
+        else:
+            binding.csb_spmm(A, Xd, Y)
+        torch.cuda.synchronize()
+        outs.append(Y.cpu().numpy())
+    assert np.array_equal(outs[0], outs[1]), "two runs differ bitwise: summation order is not fixed"
+    args = (mat.dense, mat.block_r, mat.block_c, mat.row_keep, mat.col_keep, mat.val_dtype)
+    check_product(outs[0], O.spmm(*args, X), O.abs_scale(*args, X), mat.val_dtype)
+    info = A.info()
+    A.free()
+    return info
+
+
+@pytest.mark.parametrize("vd", ["f16", "f32"])
+@pytest.mark.parametrize("shape", [(4, 4, 2, 2, 1), (64, 64, 16, 16, 1), (50, 39, 16, 8, 3), (512, 192, 16, 16, 1),
+                                   (300, 1177, 32, 32, 1), (1024, 768, 64, 64, 8), (257, 513, 256, 256, 5),
+                                   (2048, 2048, 64, 64, 13), (96, 4096, 32, 128, 2)])
+def test_random_masks(shape, vd):
+    R, C, br, bc, B = shape
+    rng = np.random.default_rng(R + 7 * C + B)
+    nblk = -(-R // br) * -(-C // bc)
+    mat = workloads.MatrixSpec((rng.standard_normal((R, C)) * 0.1).astype(np.float32), br, bc,
+                               (rng.random(nblk * br) < 0.45).astype(np.uint8),
+                               (rng.random(nblk * bc) < 0.35).astype(np.uint8), vd)
+    run_case(mat, rng.standard_normal((B, C)).astype(np.float32))
+
+
+@pytest.mark.parametrize("law,kw", [("lognormal", dict(rate=16.0)), ("lognormal", dict(rate=4.0, diag_boost=4.0)),
+                                    ("uniform", dict(lo=0.0, hi=1.0)), ("exact", dict(count=64)),
+                                    ("exact", dict(count=0)), ("exact", dict(count=1))])
+def test_keep_laws_and_degenerate_blocks(law, kw):
+    w = workloads.make_spmv_workload(3, 1024, 1536, 64, 64, law, batch=1, w_std=0.05, **kw)
+    run_case(w.matrix, w.X)
+
+
+def test_rows_kept_nowhere_and_empty_block_rows():
+    rng = np.random.default_rng(9)
+    R, C, br, bc = 256, 256, 32, 32
+    rk = (rng.random(64 * br) < 0.5).astype(np.uint8).reshape(8, 8, br)
+    ck = (rng.random(64 * bc) < 0.5).astype(np.uint8).reshape(8, 8, bc)
+    rk[2] = 0                # a whole block-row without kept rows
+    ck[5] = 0                # a whole block-row without kept columns
+    rk[:, :, 3] = 0          # in-block row 3 kept nowhere
+    mat = workloads.MatrixSpec(rng.standard_normal((R, C)).astype(np.float32), br, bc, rk.reshape(-1), ck.reshape(-1), "f16")
+    run_case(mat, rng.standard_normal((4, C)).astype(np.float32))
+
+
+@pytest.mark.parametrize("opts", [dict(ctas=1, warps_per_cta=1), dict(ctas=3, warps_per_cta=5, stages=1),
+                                  dict(ctas=148, warps_per_cta=16, stage_bytes=1024, stages=2), dict(ctas=500)])
+def test_schedules_agree(opts):
+    w = workloads.make_spmv_workload(4, 768, 1024, 32, 32, "lognormal", rate=8.0, batch=2, w_std=0.05)
+    full = dict(ctas=0, warps_per_cta=0, stage_bytes=0, stages=0)
+    full.update(opts)
+    run_case(w.matrix, w.X, full)
+
+
+def test_cfg4_full_size_sampled():
+    # the benchmark's matrix: full parity on a sample of rows is implied by full comparison here
+    w = workloads.CONFIGS["cfg4"](rate=16.0, B=1)
+    info = run_case(w.matrix, w.X)
+    assert info["balance"] > 0.8
