@@ -172,6 +172,15 @@ int csb_gru_forward(int n_layers, const csb_matrix_t* const* W, const float* con
                     const float* x, int64_t T, int B, const float* h0, float* y, float* hT,
                     unsigned flags, void* stream);
 
+/*
+ * csb_test_barrier_hook -- testing aid for the give-up path of the time loop's grid barrier
+ * (the paper has no counterpart).  Makes every later recurrent call expect `extra_arrivals`
+ * arrivals that never come and bounds each barrier wait to `limit_ns` nanoseconds, so the
+ * kernel returns with CSB_ERR_TIMEOUT instead of completing; (0, 0) restores normal operation
+ * (no extra arrivals, 2 s bound).  Process-wide; not for production use.
+ */
+void csb_test_barrier_hook(unsigned int extra_arrivals, unsigned long long limit_ns);
+
 /* Short text for a status code; never NULL. */
 const char* csb_strerror(int status);
 

@@ -56,6 +56,8 @@ lib.csb_lstm_forward.argtypes = [C.c_int, C.POINTER(_P), C.POINTER(_P), _P, C.c_
                                  C.c_uint, _P]
 lib.csb_gru_forward.argtypes = [C.c_int, C.POINTER(_P), C.POINTER(_P), _P, C.c_int64, C.c_int, _P, _P, _P,
                                 C.c_uint, _P]
+lib.csb_test_barrier_hook.argtypes = [C.c_uint, C.c_ulonglong]
+lib.csb_test_barrier_hook.restype = None
 lib.csb_strerror.argtypes = [C.c_int]
 lib.csb_strerror.restype = C.c_char_p
 lib.csb_last_error.restype = C.c_char_p

@@ -117,4 +117,55 @@ __device__ __forceinline__ void item_mac(const uint32_t* __restrict__ vals, int 
     }
 }
 
+// Walk the items stored in [p, end) (shared memory).  For each item: gather the kept inputs
+// through the column indices (gather(col, tail, bt) returns input `col` of batch column bt),
+// multiply by the kernel matrix, add into zs[(zbase_local + row_idx) * BT + bt], then let
+// after(zbase, tail) act (flush of a finished block-row, or nothing).  zs_base(zbase) maps an
+// item's zbase to the index its rows are relative to inside zs.
+template <typename T, int BT, typename Gather, typename ZsBase, typename After>
+__device__ __forceinline__ void walk_items(const uint8_t* p, const uint8_t* end, int lane, float* __restrict__ xg,
+                                           float* __restrict__ zs, Gather gather, ZsBase zs_base, After after) {
+    constexpr int R = WordTraits<T>::kRows;
+    while (p < end) {
+        const uint4 h = *reinterpret_cast<const uint4*>(p);
+        const int nk = (int)(h.x & 0xffffu), mr = (int)(h.x >> 16);
+        const uint32_t xbase = h.y, zbase = h.z, tail = h.w;
+        const uint8_t* cidx = p + 16;
+        const uint8_t* ridx = cidx + nk;
+        const int idx_bytes = (nk + mr + 3) & ~3;
+        const uint32_t* vals = reinterpret_cast<const uint32_t*>(p + 16 + idx_bytes);
+        const int RLw = (mr + R - 1) / R;
+        p += (16 + idx_bytes + nk * RLw * 4 + 15) & ~15;
+        if (nk > 0 && mr > 0) {
+            for (int k = lane; k < nk; k += 32) {
+                const uint32_t col = xbase + cidx[k];
+#pragma unroll
+                for (int bt = 0; bt < BT; ++bt) xg[k * BT + bt] = gather(col, tail, bt);
+            }
+            __syncwarp();
+            const LaneMap lm = lane_map<R>(mr, lane);
+            float acc[R][BT];
+#pragma unroll
+            for (int q = 0; q < R; ++q)
+#pragma unroll
+                for (int bt = 0; bt < BT; ++bt) acc[q][bt] = 0.f;
+            item_mac<T, BT>(vals, nk, lm, lane, xg, acc);
+            if (lane < lm.RL) {
+                float* zrow = zs + zs_base(zbase) * BT;
+#pragma unroll
+                for (int q = 0; q < R; ++q) {
+                    const int r = lane * R + q;
+                    if (r < mr) {
+                        float* z = zrow + (int)ridx[r] * BT;
+#pragma unroll
+                        for (int bt = 0; bt < BT; ++bt) z[bt] += acc[q][bt];
+                    }
+                }
+            }
+            __syncwarp();
+        }
+        after(zbase, tail);
+    }
+}
+
 }  // namespace csb

@@ -140,6 +140,22 @@ struct ProductHostPlan {
 };
 int plan_product_host(const csb_matrix* A, int n_warps, int stage_bytes, ProductHostPlan* out);
 
+// Recurrent time loop: one descriptor per CTA.
+struct RnnCtaDesc {
+    int32_t layer, u0, U;      // hidden units [u0, u0 + U) of `layer`
+    uint32_t warp0;            // first of this CTA's warps in the stream's warp table
+};
+enum { kMaxTileUnits = 64, kMaxLayers = 8 };
+struct RnnHostPlan {
+    StreamPlan stream;
+    std::vector<RnnCtaDesc> ctas;
+    int warps = 0, max_U = 0;
+    size_t max_warp_bytes = 0;
+    double balance = 1.0;
+};
+int plan_rnn_host(int gates, int n_layers, const csb_matrix* const* Wm, const int* in_size, int H, int n_ctas,
+                  int warps, int stage_bytes, RnnHostPlan* out);
+
 // csb_product.cu
 int plan_product(csb_matrix* A);           // plans, uploads, fills A->product
 void free_product(csb_matrix* A);

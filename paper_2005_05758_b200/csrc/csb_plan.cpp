@@ -51,12 +51,12 @@ void emit_item(const csb_matrix* A, const ItemSpec& it, std::vector<uint8_t>& ou
 
 void build_stream(const csb_matrix* A, const std::vector<std::vector<ItemSpec>>& per_warp,
                   int stage_bytes, StreamPlan* out) {
-    out->n_warps = (int)per_warp.size();
-    out->warp_chunk_begin.assign(per_warp.size() + 1, 0);
-    out->warp_cost.assign(per_warp.size(), 0.0);
+    // appends: a stream may hold the warps of several matrices (stacked layers)
+    if (!out->warp_chunk_begin.empty()) out->warp_chunk_begin.pop_back();
     for (size_t w = 0; w < per_warp.size(); ++w) {
-        out->warp_chunk_begin[w] = (uint32_t)out->chunks.size();
+        out->warp_chunk_begin.push_back((uint32_t)out->chunks.size());
         size_t chunk_start = out->bytes.size();
+        double cost = 0;
         for (const ItemSpec& it : per_warp[w]) {
             const size_t ib = item_bytes(A, it);
             if (out->bytes.size() - chunk_start + ib > (size_t)stage_bytes && out->bytes.size() > chunk_start) {
@@ -64,12 +64,14 @@ void build_stream(const csb_matrix* A, const std::vector<std::vector<ItemSpec>>&
                 chunk_start = out->bytes.size();
             }
             emit_item(A, it, out->bytes);
-            out->warp_cost[w] += (double)ib + 48.0;
+            cost += (double)ib + 48.0;
         }
         if (out->bytes.size() > chunk_start)
             out->chunks.push_back({(uint32_t)(chunk_start / 16), (uint32_t)(out->bytes.size() - chunk_start)});
+        out->warp_cost.push_back(cost);
     }
-    out->warp_chunk_begin[per_warp.size()] = (uint32_t)out->chunks.size();
+    out->warp_chunk_begin.push_back((uint32_t)out->chunks.size());
+    out->n_warps = (int)out->warp_cost.size();
 }
 
 // Split one block (restricted to kept rows [r0, r1)) into items that respect the
@@ -156,6 +158,126 @@ int plan_product_host(const csb_matrix* A, int n_warps, int stage_bytes, Product
     double mx = 0, sum = 0;
     for (double c : out->stream.warp_cost) { mx = std::max(mx, c); sum += c; }
     out->balance = mx > 0 ? sum / n_warps / mx : 1.0;
+    return CSB_OK;
+}
+
+// Schedule for the recurrent time loop.  Every CTA owns a tile of hidden units of one layer
+// together with ALL gate rows of those units (rows u, H+u, 2H+u, ...), so the gate arithmetic
+// needs no data from other CTAs and one grid-wide barrier per step is enough.  CTAs are shared
+// out between the layers in proportion to their stored weights (the layers run as a
+// wavefront: layer l works on step t while layer l+1 works on step t-1); unit tiles and the
+// warps inside a CTA are cut by cost, not by count.
+int plan_rnn_host(int gates, int n_layers, const csb_matrix* const* Wm, const int* in_size, int H, int n_ctas,
+                  int warps, int stage_bytes, RnnHostPlan* out) {
+    out->warps = warps;
+    out->max_U = 0;
+    // CTAs per layer
+    // every layer gets enough CTAs for its tiles to stay under the unit limit; the rest are
+    // shared out by stored weights
+    const int floor_ctas = std::min(H, (H + 47) / 48);
+    std::vector<int> ncta(n_layers, floor_ctas);
+    {
+        if (floor_ctas * n_layers > n_ctas) {
+            set_error("%d layers of hidden size %d need %d CTAs, %d available", n_layers, H, floor_ctas * n_layers, n_ctas);
+            return CSB_ERR_UNSUPPORTED;
+        }
+        double tot = 0;
+        for (int l = 0; l < n_layers; ++l) tot += (double)Wm[l]->nnz + 1.0;
+        const int spare = n_ctas - floor_ctas * n_layers;
+        for (int l = 0; l < n_layers; ++l)
+            ncta[l] = std::min(H, floor_ctas + (int)((double)spare * ((double)Wm[l]->nnz + 1.0) / tot));
+    }
+    const int value_budget = std::max(256, std::min(2048, stage_bytes - 16 - 2 * kMaxNk - 64));
+    double cost_sum = 0, cost_max = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const csb_matrix* A = Wm[l];
+        const int I = in_size[l];
+        // cost of every matrix row = stored weights in it
+        std::vector<double> rowcost(A->rows, 0.0);
+        for (int64_t b = 0; b < A->nblk; ++b) {
+            const int64_t bi = b / A->nbc;
+            const uint8_t* ri = A->row_idx.data() + A->ridx_off[b];
+            for (int r = 0; r < A->m[b]; ++r) rowcost[bi * A->block_r + ri[r]] += A->n[b] + 2.0;
+        }
+        std::vector<double> ucost(H, 8.0);
+        for (int g = 0; g < gates; ++g)
+            for (int u = 0; u < H; ++u) ucost[u] += rowcost[(int64_t)g * H + u];
+        double tot = 0;
+        for (double c : ucost) tot += c;
+        // contiguous unit tiles of about equal cost
+        std::vector<int> cut(ncta[l] + 1, H);
+        cut[0] = 0;
+        {
+            double cum = 0;
+            int t = 1;
+            for (int u = 0; u < H && t < ncta[l]; ++u) {
+                cum += ucost[u];
+                const int left_units = H - (u + 1), left_tiles = ncta[l] - t;
+                const bool full = u + 1 - cut[t - 1] >= kMaxTileUnits;
+                if (cum >= tot * t / ncta[l] || left_units <= left_tiles || full) { cut[t++] = u + 1; }
+            }
+        }
+        for (int c = 0; c < ncta[l]; ++c) {
+            const int u0 = cut[c], u1 = cut[c + 1];
+            const int U = u1 - u0;
+            if (U > kMaxTileUnits) {
+                set_error("hidden size %d over %d CTAs gives tiles of %d units (limit %d)", H, ncta[l], U, kMaxTileUnits);
+                return CSB_ERR_UNSUPPORTED;
+            }
+            out->max_U = std::max(out->max_U, U);
+            std::vector<ItemSpec> items;
+            for (int g = 0; g < gates && U > 0; ++g) {
+                const int64_t row0 = (int64_t)g * H + u0, row1 = (int64_t)g * H + u1;
+                for (int64_t bi = row0 / A->block_r; bi <= (row1 - 1) / A->block_r; ++bi) {
+                    const int lo = (int)std::max<int64_t>(0, row0 - bi * A->block_r);
+                    const int hi = (int)std::min<int64_t>(A->block_r, row1 - bi * A->block_r);
+                    for (int64_t bj = 0; bj < A->nbc; ++bj) {
+                        const int64_t b = bi * A->nbc + bj;
+                        const uint8_t* ri = A->row_idx.data() + A->ridx_off[b];
+                        const uint8_t* ci = A->col_idx.data() + A->cidx_off[b];
+                        const int m = A->m[b], n = A->n[b];
+                        const int r0 = (int)(std::lower_bound(ri, ri + m, lo) - ri);
+                        const int r1 = (int)(std::lower_bound(ri, ri + m, hi) - ri);
+                        const int64_t split_col = (int64_t)I - bj * A->block_c;      // first recurrent column, block-local
+                        const int ks = split_col <= 0 ? 0 : split_col >= A->block_c ? n
+                                       : (int)(std::lower_bound(ci, ci + n, (int)split_col) - ci);
+                        ItemSpec proto{};
+                        proto.ridx_bias = (int)(row0 - bi * A->block_r);
+                        proto.xbase = (uint32_t)(bj * A->block_c);
+                        proto.zbase = (uint32_t)(g * U);
+                        slice_block(A, b, r0, r1, 0, ks, value_budget, proto, &items);
+                        proto.xbase = (uint32_t)(bj * A->block_c - I);                 // may wrap; col_idx brings it back
+                        proto.tail = kSrcRecurrent;
+                        if (gates == 3 && g == 2) proto.zbase = (uint32_t)(3 * U);     // GRU candidate gate, hidden part
+                        slice_block(A, b, r0, r1, ks, n, value_budget, proto, &items);
+                    }
+                }
+            }
+            // warps of this CTA: contiguous runs of about equal cost
+            std::vector<std::vector<ItemSpec>> per_warp(warps);
+            double total = 0;
+            std::vector<double> cost(items.size());
+            for (size_t i = 0; i < items.size(); ++i) { cost[i] = (double)item_bytes(A, items[i]) + 48.0; total += cost[i]; }
+            double cum = 0;
+            for (size_t i = 0; i < items.size(); ++i) {
+                int w = total > 0 ? (int)((cum + 0.5 * cost[i]) / (total / warps)) : 0;
+                per_warp[std::min(std::max(w, 0), warps - 1)].push_back(items[i]);
+                cum += cost[i];
+            }
+            RnnCtaDesc d{l, u0, U, (uint32_t)out->stream.n_warps};
+            build_stream(A, per_warp, stage_bytes, &out->stream);
+            out->ctas.push_back(d);
+            cost_sum += total;
+            cost_max = std::max(cost_max, total);
+        }
+    }
+    out->max_warp_bytes = 0;
+    for (int w = 0; w < out->stream.n_warps; ++w) {
+        size_t bytes = 0;
+        for (uint32_t c = out->stream.warp_chunk_begin[w]; c < out->stream.warp_chunk_begin[w + 1]; ++c) bytes += out->stream.chunks[c].bytes;
+        out->max_warp_bytes = std::max(out->max_warp_bytes, bytes);
+    }
+    out->balance = cost_max > 0 ? cost_sum / out->ctas.size() / cost_max : 1.0;
     return CSB_OK;
 }
 

@@ -46,6 +46,52 @@ struct ProductSmem {
     }
 };
 
+// A warp that holds only part of a block-row parks its sums in its own slot; the warp that
+// arrives last adds all slots of that block-row in slot order and writes y.
+template <int BT>
+__device__ __forceinline__ void flush_partial(const ProductArgs& a, float* zs, uint32_t zbase, uint32_t tail, int nrows, int lane) {
+                        const uint32_t slot = tail >> kSlotShift;
+                        const uint32_t bi = zbase / (uint32_t)a.block_r;
+                        float* dst = a.partials + (size_t)slot * a.block_r * BT;
+                        for (int i = lane; i < nrows * BT; i += 32) { __stcg(dst + i, zs[i]); zs[i] = 0.f; }
+                        __threadfence();
+                        __syncwarp();
+                        int last = 0;
+                        if (lane == 0) last = (atomicAdd(&a.arrivals[bi], 1u) == a.part_count[bi] - 1u);
+                        last = __shfl_sync(0xffffffffu, last, 0);
+                        if (last) {
+                            // this warp saw every other contributor arrive: add the partial sums in slot
+                            // order (fixed, so the result does not depend on who came last)
+                            __threadfence();
+                            const uint32_t pb = a.part_base[bi], pc = a.part_count[bi];
+                            const size_t pstride = (size_t)a.block_r * BT;
+                            for (int i = lane; i < nrows * BT; i += 32) {
+                                // eight loads in flight; the grouping is fixed, so the sum is reproducible
+                                const float* src = a.partials + (size_t)pb * pstride + i;
+                                float s[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                                uint32_t q = 0;
+                                for (; q + 8 <= pc; q += 8) {
+                                    float v[8];
+    #pragma unroll
+                                    for (int j = 0; j < 8; ++j) v[j] = __ldcg(src + (size_t)(q + j) * pstride);
+    #pragma unroll
+                                    for (int j = 0; j < 8; ++j) s[j] += v[j];
+                                }
+                                {
+                                    float v[8];
+    #pragma unroll
+                                    for (int j = 0; j < 8; ++j) v[j] = (q + j < pc) ? __ldcg(src + (size_t)(q + j) * pstride) : 0.f;
+    #pragma unroll
+                                    for (int j = 0; j < 8; ++j) s[j] += v[j];
+                                }
+                                const float sum = ((s[0] + s[1]) + (s[2] + s[3])) + ((s[4] + s[5]) + (s[6] + s[7]));
+                                const int r = i / BT, bt = i % BT;
+                                if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = sum;
+                            }
+                            if (lane == 0) a.arrivals[bi] = 0u;      // ready for the next launch
+                        }
+}
+
 template <typename T, int BT>
 __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -101,52 +147,16 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
 
         const uint8_t* p = ring + (size_t)s * a.stage_bytes;
         const uint8_t* end = p + cur.bytes;
-        while (p < end) {
-            const uint4 h = *reinterpret_cast<const uint4*>(p);
-            const int nk = (int)(h.x & 0xffffu), mr = (int)(h.x >> 16);
-            const uint32_t xbase = h.y, zbase = h.z, tail = h.w;
-            const uint8_t* cidx = p + 16;
-            const uint8_t* ridx = cidx + nk;
-            const int idx_bytes = (nk + mr + 3) & ~3;
-            const uint32_t* vals = reinterpret_cast<const uint32_t*>(p + 16 + idx_bytes);
-            const int RLw = (mr + R - 1) / R;
-            p += (16 + idx_bytes + nk * RLw * 4 + 15) & ~15;
-
-            if (nk > 0 && mr > 0) {
-                for (int k = lane; k < nk; k += 32) {
-                    const uint32_t col = xbase + cidx[k];
-#pragma unroll
-                    for (int bt = 0; bt < BT; ++bt) {
-                        float v = 0.f;
-                        if (BT == 1) v = a.x_in_smem ? xs[col] : __ldg(a.X + col);
-                        else if (bt < a.nb) v = __ldg(a.X + (long long)bt * a.ldx + col);
-                        xg[k * BT + bt] = v;
-                    }
-                }
-                __syncwarp();
-                const LaneMap lm = lane_map<R>(mr, lane);
-                float acc[R][BT];
-#pragma unroll
-                for (int q = 0; q < R; ++q)
-#pragma unroll
-                    for (int bt = 0; bt < BT; ++bt) acc[q][bt] = 0.f;
-                item_mac<T, BT>(vals, nk, lm, lane, xg, acc);
-                if (lane < lm.RL) {
-#pragma unroll
-                    for (int q = 0; q < R; ++q) {
-                        const int r = lane * R + q;
-                        if (r < mr) {
-                            float* z = zs + (int)ridx[r] * BT;
-#pragma unroll
-                            for (int bt = 0; bt < BT; ++bt) z[bt] += acc[q][bt];
-                        }
-                    }
-                }
-                __syncwarp();
-            }
-
-            const uint32_t flush = tail & 3u;
-            if (flush != kFlushNone) {
+        walk_items<T, BT>(
+            p, end, lane, xg, zs,
+            [&](uint32_t col, uint32_t, int bt) -> float {
+                if (BT == 1) return a.x_in_smem ? xs[col] : __ldg(a.X + col);
+                return bt < a.nb ? __ldg(a.X + (long long)bt * a.ldx + col) : 0.f;
+            },
+            [](uint32_t) { return 0; },
+            [&](uint32_t zbase, uint32_t tail) {
+                const uint32_t flush = tail & 3u;
+                if (flush == kFlushNone) return;
                 const int nrows = min(a.block_r, a.rows - (int)zbase);
                 if (flush == kFlushDirect) {
                     for (int i = lane; i < nrows * BT; i += 32) {
@@ -155,32 +165,10 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
                         zs[i] = 0.f;
                     }
                 } else {
-                    const uint32_t slot = tail >> kSlotShift;
-                    const uint32_t bi = zbase / (uint32_t)a.block_r;
-                    float* dst = a.partials + (size_t)slot * a.block_r * BT;
-                    for (int i = lane; i < nrows * BT; i += 32) { __stcg(dst + i, zs[i]); zs[i] = 0.f; }
-                    __threadfence();
-                    __syncwarp();
-                    int last = 0;
-                    if (lane == 0) last = (atomicAdd(&a.arrivals[bi], 1u) == a.part_count[bi] - 1u);
-                    last = __shfl_sync(0xffffffffu, last, 0);
-                    if (last) {
-                        // this warp saw every other contributor arrive: add the partial sums in slot
-                        // order (fixed, so the result does not depend on who came last)
-                        __threadfence();
-                        const uint32_t pb = a.part_base[bi], pc = a.part_count[bi];
-                        for (int i = lane; i < nrows * BT; i += 32) {
-                            float sum = 0.f;
-                            for (uint32_t q = 0; q < pc; ++q) sum += __ldcg(a.partials + ((size_t)(pb + q) * a.block_r) * BT + i);
-                            const int r = i / BT, bt = i % BT;
-                            if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = sum;
-                        }
-                        if (lane == 0) a.arrivals[bi] = 0u;      // ready for the next launch
-                    }
+                    flush_partial<BT>(a, zs, zbase, tail, nrows, lane);
                 }
                 __syncwarp();
-            }
-        }
+            });
         __syncwarp();
         if (lane == 0 && refill.bytes) {
             mbar_expect_tx(&bars[s], refill.bytes);

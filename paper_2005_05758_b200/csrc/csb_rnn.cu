@@ -1,9 +1,498 @@
+// Persistent LSTM / GRU time-loop kernel and its launch glue.
+//
+// One cooperative launch runs the whole sequence (Section 2.1 of the paper: per step one
+// CSB product with [u_t ; h_{t-1}] followed by the element-wise gate arithmetic, the c / h
+// "context link" feeding the next step).  A CTA owns a tile of hidden units with all gate
+// rows of those units; its compressed weights stay in shared memory for the whole sequence
+// when they fit (otherwise they are re-streamed from L2 through the same bulk-copy ring as
+// the bare product).  Only h_t crosses CTAs, through global memory and one bounded grid
+// barrier per step.  Stacked layers run as a wavefront: in tick k layer l does step k - l.
+#include <algorithm>
+#include <list>
+#include <memory>
+#include <mutex>
+
 #include "csb_device.cuh"
 #include "csb_internal.hpp"
-namespace csb { void drop_rnn_plans(const csb_matrix*) {} }
-extern "C" {
-int csb_lstm_forward(int, const csb_matrix_t* const*, const float* const*, const float*, int64_t, int, const float*,
-                     const float*, float*, float*, float*, unsigned, void*) { csb::set_error("not built yet"); return CSB_ERR_UNSUPPORTED; }
-int csb_gru_forward(int, const csb_matrix_t* const*, const float* const*, const float*, int64_t, int, const float*,
-                    float*, float*, unsigned, void*) { csb::set_error("not built yet"); return CSB_ERR_UNSUPPORTED; }
+
+namespace csb {
+
+struct RnnArgs {
+    const uint8_t* stream;
+    const Chunk* chunks;
+    const uint32_t* warp_chunk_begin;
+    const RnnCtaDesc* ctas;
+    const float* x;            // [T, B, I0]
+    float* y;                  // [T, B, H] or null
+    float* hbuf;               // [L][2][B][H]: h of step t lives in slot t & 1
+    float* cstate;             // [L][B][H], in: c0, out: cT
+    const float* bias[kMaxLayers];
+    int in_size[kMaxLayers];
+    unsigned int* barrier;     // zero at launch
+    uint32_t* status;
+    unsigned long long barrier_ns;
+    unsigned int barrier_extra;   // test hook: arrivals that never come
+    int T, B, H, L, gates, stage_bytes, stages, resident, max_warp_bytes, max_U, max_C;
+};
+
+struct RnnSmem {
+    size_t weights, bars, zs, xg, v, cs, flag, total;
+    int zs_stride;
+    __host__ __device__ RnnSmem(int W, int stages, int stage_bytes, int resident, int max_warp_bytes, int max_U, int BT,
+                                int B, int max_C) {
+        zs_stride = 4 * max_U * BT;
+        weights = 0;
+        const size_t per_warp = resident ? (size_t)max_warp_bytes : (size_t)stages * stage_bytes;
+        bars = weights + (size_t)W * per_warp;
+        zs = (bars + (size_t)W * (resident ? 1 : stages) * 8 + 15) & ~(size_t)15;
+        xg = (zs + (size_t)W * zs_stride * 4 + 15) & ~(size_t)15;
+        v = (xg + (size_t)W * kMaxNk * BT * 4 + 15) & ~(size_t)15;
+        cs = (v + (BT == 1 ? (size_t)max_C * 4 : 0) + 15) & ~(size_t)15;
+        flag = (cs + (size_t)max_U * B * 4 + 15) & ~(size_t)15;
+        total = flag + 16;
+    }
+};
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
+
+// All CTAs arrive, then wait until `target` arrivals are visible.  The wait is bounded in
+// wall-clock time; on expiry the status word is raised and every thread gets `false`.
+__device__ __forceinline__ bool grid_barrier(const RnnArgs& a, unsigned int target, volatile int* s_flag) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(a.barrier, 1u);
+        bool ok = true;
+        unsigned long long t0 = 0;
+        unsigned int spins = 0;
+        while (ld_acquire_u32(a.barrier) < target) {
+            if ((++spins & 63u) == 0) {
+                const unsigned long long now = global_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > a.barrier_ns) { ok = false; break; }
+            }
+        }
+        if (!ok) *(volatile uint32_t*)a.status = (uint32_t)kDevBarrierTimeout;
+        *s_flag = ok ? 1 : 0;
+    }
+    __syncthreads();
+    return *s_flag != 0;
+}
+
+__device__ __forceinline__ float sigmoidf_acc(float a) { return 1.f / (1.f + expf(-a)); }
+
+template <typename T, int BT>
+__global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const RnnSmem S(W, a.stages, a.stage_bytes, a.resident, a.max_warp_bytes, a.max_U, BT, a.B, a.max_C);
+    const RnnCtaDesc me = a.ctas[blockIdx.x];
+    const int layer = me.layer, U = me.U, u0 = me.u0, H = a.H, B = a.B;
+    const int I = a.in_size[layer], C = I + H;
+    const size_t per_warp = a.resident ? (size_t)a.max_warp_bytes : (size_t)a.stages * a.stage_bytes;
+    uint8_t* wbuf = smem + S.weights + warp * per_warp;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S.bars) + warp * (a.resident ? 1 : a.stages);
+    float* zs_all = reinterpret_cast<float*>(smem + S.zs);
+    float* zs = zs_all + warp * S.zs_stride;
+    float* xg = reinterpret_cast<float*>(smem + S.xg) + warp * kMaxNk * BT;
+    float* vs = reinterpret_cast<float*>(smem + S.v);
+    float* cs = reinterpret_cast<float*>(smem + S.cs);
+    volatile int* s_flag = reinterpret_cast<volatile int*>(smem + S.flag);
+
+    const uint32_t c0 = a.warp_chunk_begin[me.warp0 + warp], c1 = a.warp_chunk_begin[me.warp0 + warp + 1];
+    const uint32_t nchunks = c1 - c0;
+    const uint8_t* wsrc = a.stream + (size_t)(nchunks ? a.chunks[c0].off16 : 0) * 16;
+    uint32_t wbytes = 0;
+    bool alive = true;
+
+    // ---- weights: load once (resident) or prime the ring (streaming) ----
+    // streaming: every step walks the ring once per batch tile; chunk sequence numbers keep counting
+    unsigned long long n_done = 0;
+    const unsigned long long n_total = (unsigned long long)a.T * ((B + BT - 1) / BT) * nchunks;
+    if (a.resident) {
+        for (uint32_t c = c0; c < c1; ++c) wbytes += a.chunks[c].bytes;   // chunks of a warp are contiguous
+        if (lane == 0) {
+            mbar_init(&bars[0], 1);
+            mbar_fence_init();
+            if (wbytes) {
+                mbar_expect_tx(&bars[0], wbytes);
+                for (uint32_t off = 0; off < wbytes; off += 16384u)
+                    bulk_g2s(wbuf + off, wsrc + off, min(16384u, wbytes - off), &bars[0]);
+            }
+        }
+        __syncwarp();
+        if (wbytes && !mbar_wait_bounded(&bars[0], 0)) alive = false;
+    } else {
+        if (lane == 0) {
+            for (int s = 0; s < a.stages; ++s) mbar_init(&bars[s], 1);
+            mbar_fence_init();
+            for (unsigned long long n_issued = 0; n_issued < (unsigned long long)a.stages && n_issued < n_total; ++n_issued) {
+                const Chunk ch = a.chunks[c0 + (uint32_t)(n_issued % nchunks)];
+                const int s = (int)(n_issued % (unsigned)a.stages);
+                mbar_expect_tx(&bars[s], ch.bytes);
+                bulk_g2s(wbuf + (size_t)s * a.stage_bytes, a.stream + (size_t)ch.off16 * 16, ch.bytes, &bars[s]);
+            }
+        }
+        __syncwarp();
+    }
+    // cell state of this tile
+    for (int i = threadIdx.x; i < U * B; i += blockDim.x) {
+        const int b = i / U, u = i % U;
+        cs[b * a.max_U + u] = a.gates == 4 ? a.cstate[((size_t)layer * B + b) * H + u0 + u] : 0.f;
+    }
+    if (threadIdx.x == 0) *s_flag = 1;
+    __syncthreads();
+
+    const float* bias = a.bias[layer];
+    const int n_ticks = a.T + a.L - 1;
+    for (int tick = 0; tick < n_ticks; ++tick) {
+        const int t = tick - layer;
+        const bool active = t >= 0 && t < a.T;
+        if (active) {
+            const float* in_src = layer == 0 ? a.x + (size_t)t * B * I
+                                             : a.hbuf + ((size_t)(layer - 1) * 2 + (t & 1)) * B * H;
+            const float* rec_src = a.hbuf + ((size_t)layer * 2 + ((t + 1) & 1)) * B * H;   // slot of step t-1
+            float* h_dst = a.hbuf + ((size_t)layer * 2 + (t & 1)) * B * H;
+            const int in_ld = layer == 0 ? I : H;
+            if (BT == 1) {
+                for (int i = threadIdx.x; i < C; i += blockDim.x)
+                    vs[i] = i < I ? (layer == 0 ? __ldg(in_src + i) : __ldcg(in_src + i)) : __ldcg(rec_src + (i - I));
+                __syncthreads();
+            }
+            for (int b0 = 0; b0 < B; b0 += BT) {
+                const int nb = min(BT, B - b0);
+                for (int i = lane; i < S.zs_stride; i += 32) zs[i] = 0.f;
+                __syncwarp();
+                auto gather = [&](uint32_t col, uint32_t tail, int bt) -> float {
+                    if (BT == 1) return vs[(tail & kSrcRecurrent) ? col + I : col];
+                    if (bt >= nb) return 0.f;
+                    return (tail & kSrcRecurrent) ? __ldcg(rec_src + (size_t)(b0 + bt) * H + col)
+                                                  : __ldcg(in_src + (size_t)(b0 + bt) * in_ld + col);
+                };
+                auto zs_base = [](uint32_t zbase) { return (int)zbase; };
+                auto after = [](uint32_t, uint32_t) {};
+                if (a.resident) {
+                    if (alive) walk_items<T, BT>(wbuf, wbuf + wbytes, lane, xg, zs, gather, zs_base, after);
+                } else {
+                    for (uint32_t c = 0; c < nchunks && alive; ++c) {
+                        const int s = (int)(n_done % (unsigned)a.stages);
+                        const uint32_t parity = (uint32_t)((n_done / (unsigned)a.stages) & 1u);
+                        const Chunk ch = a.chunks[c0 + c];
+                        if (!mbar_wait_bounded(&bars[s], parity)) alive = false;
+                        alive = !__any_sync(0xffffffffu, !alive);
+                        if (!alive) {
+                            if (lane == 0)        // bounded drain of the copies still in flight
+                                for (unsigned long long n = n_done + 1; n < n_done + a.stages && n < n_total; ++n)
+                                    mbar_wait_bounded(&bars[n % (unsigned)a.stages], (uint32_t)((n / (unsigned)a.stages) & 1u));
+                            break;
+                        }
+                        const uint8_t* p = wbuf + (size_t)s * a.stage_bytes;
+                        walk_items<T, BT>(p, p + ch.bytes, lane, xg, zs, gather, zs_base, after);
+                        __syncwarp();
+                        ++n_done;
+                        if (lane == 0 && n_done + a.stages - 1 < n_total) {
+                            const unsigned long long n = n_done + a.stages - 1;
+                            const Chunk nx = a.chunks[c0 + (uint32_t)(n % nchunks)];
+                            mbar_expect_tx(&bars[s], nx.bytes);
+                            bulk_g2s(wbuf + (size_t)s * a.stage_bytes, a.stream + (size_t)nx.off16 * 16, nx.bytes, &bars[s]);
+                        }
+                    }
+                }
+                __syncthreads();
+                // ---- gate arithmetic for this batch tile ----
+                for (int i = threadIdx.x; i < U * nb; i += blockDim.x) {
+                    const int bt = i / U, u = i % U, b = b0 + bt;
+                    float z[4] = {0.f, 0.f, 0.f, 0.f};
+                    for (int w = 0; w < W; ++w) {
+                        const float* zw = zs_all + w * S.zs_stride;
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) z[g] += zw[(g * U + u) * BT + bt];
+                    }
+                    float h;
+                    if (a.gates == 4) {
+                        if (bias) {
+#pragma unroll
+                            for (int g = 0; g < 4; ++g) z[g] += __ldg(bias + g * H + u0 + u);
+                        }
+                        const float c = sigmoidf_acc(z[1]) * cs[b * a.max_U + u] + sigmoidf_acc(z[0]) * tanhf(z[2]);
+                        cs[b * a.max_U + u] = c;
+                        h = sigmoidf_acc(z[3]) * tanhf(c);
+                        if (t == a.T - 1) a.cstate[((size_t)layer * B + b) * H + u0 + u] = c;
+                    } else {
+                        float br = 0.f, bz = 0.f, bin = 0.f, bhn = 0.f;
+                        if (bias) {
+                            br = __ldg(bias + u0 + u); bz = __ldg(bias + H + u0 + u);
+                            bin = __ldg(bias + 2 * H + u0 + u); bhn = __ldg(bias + 3 * H + u0 + u);
+                        }
+                        const float r = sigmoidf_acc(z[0] + br), zg = sigmoidf_acc(z[1] + bz);
+                        const float n = tanhf(z[2] + bin + r * (z[3] + bhn));
+                        const float hp = __ldcg(rec_src + (size_t)b * H + u0 + u);
+                        h = (1.f - zg) * n + zg * hp;
+                    }
+                    h_dst[(size_t)b * H + u0 + u] = h;
+                    if (layer == a.L - 1 && a.y) a.y[((size_t)t * B + b) * H + u0 + u] = h;
+                }
+                __syncthreads();
+            }
+        }
+        if (tick + 1 < n_ticks) {
+            if (!grid_barrier(a, (unsigned)(tick + 1) * (gridDim.x + a.barrier_extra), s_flag)) break;
+        }
+    }
+    if (!alive && lane == 0) *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout;
+}
+
+
+#define CSB_CUDA(call)                                                                     \
+    do {                                                                                   \
+        cudaError_t e_ = (call);                                                           \
+        if (e_ != cudaSuccess) {                                                           \
+            set_error("%s failed: %s", #call, cudaGetErrorString(e_));                     \
+            return e_ == cudaErrorMemoryAllocation ? CSB_ERR_ALLOC : CSB_ERR_CUDA;         \
+        }                                                                                  \
+    } while (0)
+
+// Everything one (cell, layer stack, batch) combination needs on the device; built on first
+// use and kept until one of its matrices is freed.
+struct RnnPlan {
+    int gates = 0, L = 0, B = 0, H = 0, device = 0, val_dtype = 0;
+    std::vector<uint64_t> uids;
+    int in_size[kMaxLayers] = {};
+    int n_ctas = 0, warps = 0, BT = 1, resident = 0, stages = 0, stage_bytes = 0, max_warp_bytes = 0, max_U = 0, max_C = 0;
+    size_t smem = 0;
+    double balance = 1.0;
+    int64_t stream_bytes = 0;
+    uint8_t* d_stream = nullptr; Chunk* d_chunks = nullptr; uint32_t* d_wcb = nullptr; RnnCtaDesc* d_ctas = nullptr;
+    float* d_hbuf = nullptr; float* d_cstate = nullptr; unsigned int* d_barrier = nullptr;
+    uint32_t* h_status = nullptr; uint32_t* d_status = nullptr;
+    float* d_stage = nullptr; size_t stage_cap = 0;      // host-I/O staging: x, y, states
+    ~RnnPlan() {
+        cudaFree(d_stream); cudaFree(d_chunks); cudaFree(d_wcb); cudaFree(d_ctas); cudaFree(d_hbuf);
+        cudaFree(d_cstate); cudaFree(d_barrier); cudaFree(d_stage);
+        if (h_status) cudaFreeHost(h_status);
+    }
+};
+
+static std::mutex g_rnn_mu;
+static std::list<std::unique_ptr<RnnPlan>> g_rnn_plans;
+static unsigned long long g_barrier_ns = 2000ull * 1000ull * 1000ull;
+static unsigned int g_barrier_extra = 0;
+
+void drop_rnn_plans(const csb_matrix* A) {
+    std::lock_guard<std::mutex> lk(g_rnn_mu);
+    int prev = 0;
+    cudaGetDevice(&prev);
+    for (auto it = g_rnn_plans.begin(); it != g_rnn_plans.end();) {
+        if (std::find((*it)->uids.begin(), (*it)->uids.end(), A->uid) != (*it)->uids.end()) {
+            cudaSetDevice((*it)->device);
+            it = g_rnn_plans.erase(it);
+        } else ++it;
+    }
+    cudaSetDevice(prev);
+}
+
+template <typename V>
+static int upload_vec(const std::vector<V>& h, V** d) {
+    const size_t bytes = std::max<size_t>(h.size(), 1) * sizeof(V);
+    CSB_CUDA(cudaMalloc((void**)d, bytes));
+    if (!h.empty()) CSB_CUDA(cudaMemcpy(*d, h.data(), h.size() * sizeof(V), cudaMemcpyHostToDevice));
+    return CSB_OK;
+}
+
+static int env_int(const char* name, int dflt) {
+    const char* v = getenv(name);
+    return v && *v ? atoi(v) : dflt;
+}
+
+static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, int H, const int* in_size, RnnPlan* P) {
+    const csb_matrix* A0 = W[0];
+    P->gates = gates; P->L = L; P->B = B; P->H = H; P->device = A0->device; P->val_dtype = A0->val_dtype;
+    for (int l = 0; l < L; ++l) { P->uids.push_back(W[l]->uid); P->in_size[l] = in_size[l]; P->max_C = std::max(P->max_C, in_size[l] + H); }
+    P->BT = B == 1 ? 1 : (B <= 4 ? 4 : 8);
+    P->warps = std::min(16, std::max(1, env_int("CSB_RNN_WARPS", 16)));
+    P->stage_bytes = 3072; P->stages = 3;
+    int64_t approx = 0;
+    for (int l = 0; l < L; ++l) approx += W[l]->nnz * val_size(W[l]->val_dtype) + 32 * W[l]->nblk;
+    int want = (int)std::min<int64_t>(A0->sm_count, std::max<int64_t>(L, approx / (24 * 1024)));
+    want = std::max(want, L * ((H + 47) / 48));        // tiles are cut by cost; leave room under the 64-unit limit
+    want = env_int("CSB_RNN_CTAS", want);
+    want = std::min(std::max(want, L), A0->sm_count);
+    RnnHostPlan Hp;
+    int rc = plan_rnn_host(gates, L, W, in_size, H, want, P->warps, P->stage_bytes, &Hp);
+    if (rc != CSB_OK) return rc;
+    P->n_ctas = (int)Hp.ctas.size();
+    P->max_U = Hp.max_U; P->max_warp_bytes = (int)Hp.max_warp_bytes; P->balance = Hp.balance;
+    P->stream_bytes = (int64_t)Hp.stream.bytes.size();
+    const RnnSmem res(P->warps, P->stages, P->stage_bytes, 1, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
+    const RnnSmem str(P->warps, P->stages, P->stage_bytes, 0, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
+    if (res.total <= A0->smem_optin && !env_int("CSB_RNN_STREAM", 0)) { P->resident = 1; P->smem = res.total; }
+    else if (str.total <= A0->smem_optin) { P->resident = 0; P->smem = str.total; }
+    else { set_error("time-loop kernel needs %zu bytes of shared memory per CTA, device offers %zu", str.total, A0->smem_optin); return CSB_ERR_LAUNCH; }
+    if ((rc = upload_vec(Hp.stream.bytes, &P->d_stream)) != CSB_OK) return rc;
+    if ((rc = upload_vec(Hp.stream.chunks, &P->d_chunks)) != CSB_OK) return rc;
+    if ((rc = upload_vec(Hp.stream.warp_chunk_begin, &P->d_wcb)) != CSB_OK) return rc;
+    if ((rc = upload_vec(Hp.ctas, &P->d_ctas)) != CSB_OK) return rc;
+    CSB_CUDA(cudaMalloc((void**)&P->d_hbuf, (size_t)L * 2 * B * H * 4));
+    CSB_CUDA(cudaMalloc((void**)&P->d_cstate, (size_t)L * B * H * 4));
+    CSB_CUDA(cudaMalloc((void**)&P->d_barrier, 4));
+    CSB_CUDA(cudaHostAlloc((void**)&P->h_status, 4, cudaHostAllocMapped));
+    *P->h_status = 0;
+    CSB_CUDA(cudaHostGetDevicePointer((void**)&P->d_status, P->h_status, 0));
+    return CSB_OK;
+}
+
+template <typename T, int BT>
+static int launch_rnn(const RnnPlan* P, RnnArgs& a, cudaStream_t st) {
+    CSB_CUDA(cudaFuncSetAttribute(csb_rnn_kernel<T, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem));
+    int occ = 0;
+    CSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, csb_rnn_kernel<T, BT>, P->warps * 32, P->smem));
+    int sms = 0;
+    CSB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, P->device));
+    if (occ < 1 || P->n_ctas > occ * sms) {
+        set_error("grid of %d CTAs cannot be co-resident (%d per SM x %d SMs)", P->n_ctas, occ, sms);
+        return CSB_ERR_LAUNCH;
+    }
+    void* params[] = {(void*)&a};
+    const cudaError_t e = cudaLaunchCooperativeKernel((const void*)csb_rnn_kernel<T, BT>, dim3(P->n_ctas), dim3(P->warps * 32),
+                                                      params, P->smem, st);
+    if (e == cudaErrorCooperativeLaunchTooLarge) { set_error("cooperative launch too large"); return CSB_ERR_LAUNCH; }
+    CSB_CUDA(e);
+    return CSB_OK;
+}
+
+static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const float* const* bias, const float* x, int64_t T,
+                       int B, const float* h0, const float* c0, float* y, float* hT, float* cT, unsigned flags, void* stream) {
+    clear_error();
+    if (L < 1 || L > kMaxLayers || !W) { set_error("n_layers %d (1..%d) or W is NULL", L, (int)kMaxLayers); return CSB_ERR_INVALID_ARG; }
+    if (T < 0 || B < 0 || T > 0x7fffffff) { set_error("T=%lld B=%d", (long long)T, B); return CSB_ERR_INVALID_ARG; }
+    for (int l = 0; l < L; ++l) if (!W[l]) { set_error("W[%d] is NULL", l); return CSB_ERR_INVALID_ARG; }
+    if (W[0]->rows % gates) { set_error("W[0] has %lld rows, not a multiple of %d gates", (long long)W[0]->rows, gates); return CSB_ERR_SHAPE; }
+    const int H = (int)(W[0]->rows / gates);
+    int in_size[kMaxLayers];
+    for (int l = 0; l < L; ++l) {
+        in_size[l] = (int)(W[l]->cols - H);
+        if (W[l]->rows != (int64_t)gates * H || in_size[l] <= 0 || (l > 0 && in_size[l] != H)) {
+            set_error("layer %d: weight is %lld x %lld, expected %d x (%s + %d)", l, (long long)W[l]->rows, (long long)W[l]->cols,
+                      gates * H, l ? "H" : "I", H);
+            return CSB_ERR_SHAPE;
+        }
+        if (W[l]->device < 0) { set_error("layer %d was encoded host-only", l); return CSB_ERR_UNSUPPORTED; }
+        if (W[l]->device != W[0]->device || W[l]->val_dtype != W[0]->val_dtype) {
+            set_error("layers must share device and value type");
+            return CSB_ERR_UNSUPPORTED;
+        }
+    }
+    if (T == 0 || B == 0) return CSB_OK;
+    if (!x) { set_error("x is NULL"); return CSB_ERR_INVALID_ARG; }
+    const int I0 = in_size[0];
+    int prev = 0;
+    CSB_CUDA(cudaGetDevice(&prev));
+    CSB_CUDA(cudaSetDevice(W[0]->device));
+    struct Restore { int d; ~Restore() { cudaSetDevice(d); } } restore{prev};
+
+    RnnPlan* P = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(g_rnn_mu);
+        for (auto& p : g_rnn_plans) {
+            if (p->gates != gates || p->L != L || p->B != B) continue;
+            bool same = true;
+            for (int l = 0; l < L; ++l) same = same && p->uids[l] == W[l]->uid;
+            if (same) { P = p.get(); break; }
+        }
+        if (!P) {
+            std::unique_ptr<RnnPlan> np(new RnnPlan());
+            int rc = CSB_OK;
+            try { rc = build_rnn_plan(gates, L, W, B, H, in_size, np.get()); }
+            catch (const std::bad_alloc&) { set_error("out of host memory while planning the time loop"); rc = CSB_ERR_ALLOC; }
+            if (rc != CSB_OK) return rc;
+            CSB_CUDA(cudaDeviceSynchronize());
+            P = np.get();
+            g_rnn_plans.push_back(std::move(np));
+        }
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool host_io = (flags & CSB_FLAG_HOST_IO) != 0;
+    const size_t nx = (size_t)T * B * I0, ny = (size_t)T * B * H, ns = (size_t)L * B * H;
+    const float* dx = x;
+    float* dy = y;
+    if (host_io) {
+        const size_t need = nx + (y ? ny : 0);
+        if (need > P->stage_cap) {
+            CSB_CUDA(cudaStreamSynchronize(st));
+            cudaFree(P->d_stage); P->d_stage = nullptr; P->stage_cap = 0;
+            CSB_CUDA(cudaMalloc((void**)&P->d_stage, need * 4));
+            P->stage_cap = need;
+        }
+        CSB_CUDA(cudaMemcpyAsync(P->d_stage, x, nx * 4, cudaMemcpyHostToDevice, st));
+        dx = P->d_stage;
+        dy = y ? P->d_stage + nx : nullptr;
+    }
+    const cudaMemcpyKind in_kind = host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
+    const cudaMemcpyKind out_kind = host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice;
+    const size_t row = (size_t)B * H * 4;
+    // h0 goes to slot 1 of every layer (the slot of "step -1"), c0 to the cell-state buffer
+    if (h0) CSB_CUDA(cudaMemcpy2DAsync(P->d_hbuf + (size_t)B * H, 2 * row, h0, row, row, L, in_kind, st));
+    else CSB_CUDA(cudaMemsetAsync(P->d_hbuf, 0, 2 * row * L, st));
+    if (gates == 4) {
+        if (c0) CSB_CUDA(cudaMemcpyAsync(P->d_cstate, c0, ns * 4, in_kind, st));
+        else CSB_CUDA(cudaMemsetAsync(P->d_cstate, 0, ns * 4, st));
+    }
+    CSB_CUDA(cudaMemsetAsync(P->d_barrier, 0, 4, st));
+    *P->h_status = 0;
+
+    RnnArgs a{};
+    a.stream = P->d_stream; a.chunks = P->d_chunks; a.warp_chunk_begin = P->d_wcb; a.ctas = P->d_ctas;
+    a.x = dx; a.y = dy; a.hbuf = P->d_hbuf; a.cstate = P->d_cstate;
+    for (int l = 0; l < L; ++l) { a.bias[l] = bias ? bias[l] : nullptr; a.in_size[l] = in_size[l]; }
+    a.barrier = P->d_barrier; a.status = P->d_status; a.barrier_ns = g_barrier_ns; a.barrier_extra = g_barrier_extra;
+    a.T = (int)T; a.B = B; a.H = H; a.L = L; a.gates = gates; a.stage_bytes = P->stage_bytes; a.stages = P->stages;
+    a.resident = P->resident; a.max_warp_bytes = P->max_warp_bytes; a.max_U = P->max_U; a.max_C = P->max_C;
+    int rc;
+    const bool half = P->val_dtype == CSB_F16;
+    if (P->BT == 1) rc = half ? launch_rnn<__half, 1>(P, a, st) : launch_rnn<float, 1>(P, a, st);
+    else if (P->BT == 4) rc = half ? launch_rnn<__half, 4>(P, a, st) : launch_rnn<float, 4>(P, a, st);
+    else rc = half ? launch_rnn<__half, 8>(P, a, st) : launch_rnn<float, 8>(P, a, st);
+    if (rc != CSB_OK) return rc;
+    const int last_slot = (int)((T - 1) & 1);
+    if (hT) CSB_CUDA(cudaMemcpy2DAsync(hT, row, P->d_hbuf + (size_t)last_slot * B * H, 2 * row, row, L, out_kind, st));
+    if (cT && gates == 4) CSB_CUDA(cudaMemcpyAsync(cT, P->d_cstate, ns * 4, out_kind, st));
+    if (host_io && y) CSB_CUDA(cudaMemcpyAsync(y, dy, ny * 4, cudaMemcpyDeviceToHost, st));
+    if (host_io || !(flags & CSB_FLAG_ASYNC)) {
+        CSB_CUDA(cudaStreamSynchronize(st));
+        if (*P->h_status != 0) {
+            set_error("the time-loop kernel gave up a bounded wait (code %u: %s)", *P->h_status,
+                      *P->h_status == kDevBarrierTimeout ? "grid barrier" : "bulk copy");
+            return CSB_ERR_TIMEOUT;
+        }
+    }
+    return CSB_OK;
+}
+
+void set_barrier_test_hook(unsigned int extra, unsigned long long ns) {
+    g_barrier_extra = extra;
+    g_barrier_ns = ns ? ns : 2000ull * 1000ull * 1000ull;
+}
+
+}  // namespace csb
+
+extern "C" {
+
+int csb_lstm_forward(int n_layers, const csb_matrix_t* const* W, const float* const* bias, const float* x, int64_t T, int B,
+                     const float* h0, const float* c0, float* y, float* hT, float* cT, unsigned flags, void* stream) {
+    return csb::rnn_forward(4, n_layers, W, bias, x, T, B, h0, c0, y, hT, cT, flags, stream);
+}
+
+int csb_gru_forward(int n_layers, const csb_matrix_t* const* W, const float* const* bias, const float* x, int64_t T, int B,
+                    const float* h0, float* y, float* hT, unsigned flags, void* stream) {
+    return csb::rnn_forward(3, n_layers, W, bias, x, T, B, h0, nullptr, y, hT, nullptr, flags, stream);
+}
+
+void csb_test_barrier_hook(unsigned int extra_arrivals, unsigned long long limit_ns) {
+    csb::set_barrier_test_hook(extra_arrivals, limit_ns);
+}
+
+}  // extern "C"
