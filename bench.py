@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the CSB-RNN hot path on B200.
+
+A step is one pass of the whole path over one batch of synthetic input: one
+csb_lstm_forward call over the full sequence of the largest recurrent workload
+(two stacked LSTM layers, 8192x4096 CSB weights with 64x64 blocks at ~10x pruning,
+512 steps, batch 1).  The headline value is microseconds per timestep.  Beside it
+the JSON line carries the roofline of the time-loop kernel, the bare CSB-SpMV sweep
+against the HBM roofline, microseconds per timestep of the other workloads, an
+end-to-end figure with host buffers, and the float64 oracle timed on the host.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    torchrun ... bench.py --gpus N ...     (N > 1: independent replicas, no collective)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+METRIC = "us_per_timestep_batch1"
+UNIT = "us/timestep"
+WORKLOAD = "cfg5: 2-layer LSTM, I=H=2048, 8192x4096 CSB weights, 64x64 blocks, ~10x pruning, T=512, B=1, fp16 values / fp32 accumulate"
+
+
+def peaks():
+    """Measured HBM copy bandwidth of this machine's B200 (generated file), else the fallback."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def layer_tuples(w):
+    return [(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype) for m in w.layers]
+
+
+# ----------------------------------------------------------------------------------------
+# CPU oracle arm
+# ----------------------------------------------------------------------------------------
+def oracle_us_per_step(w, t_short=2, t_long=10):
+    """Per-step cost of the oracle recurrence as it stands: the slope between two calls of
+    different length, so that building the masked dense matrix (done once per call) drops out."""
+    from oracle import rnn_oracle as R
+    fn = R.lstm_forward if w.cell == "lstm" else R.gru_forward
+    args = (layer_tuples(w), w.bias)
+
+    def run(n):
+        t0 = time.perf_counter()
+        if w.cell == "lstm":
+            fn(*args, w.x[:n], w.h0, w.c0)
+        else:
+            fn(*args, w.x[:n], w.h0)
+        return time.perf_counter() - t0
+
+    a, b = run(t_short), run(t_long)
+    return max(b - a, 1e-9) / (t_long - t_short) * 1e6
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def reference_arm(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    w = workloads.CONFIGS["cfg5"](T=12)
+    vals = []
+    for _ in range(args.warmup):
+        oracle_us_per_step(w, 1, 2)
+    for _ in range(args.steps):
+        vals.append(oracle_us_per_step(w, 2, 10))
+    v = float(np.mean(vals))
+    sample = "slope of the float64 oracle recurrence between 2 and 10 timesteps of cfg5 (numpy BLAS), per step"
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": v * 512 / 1e3, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ----------------------------------------------------------------------------------------
+# GPU arm
+# ----------------------------------------------------------------------------------------
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.lines, self.proc = [], None
+        try:
+            cmd = ["nvidia-smi", "--query-gpu=" + self.Q, "--format=csv,noheader,nounits", "-lms", "200"]
+            if uuid:
+                cmd += ["-i", uuid]
+            self.proc = subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def rnn_alg_bytes_per_step(w, infos):
+    """Bytes the method itself must move per timestep: packed values, index lists and 6-byte block
+    headers of every layer, the input and state vectors read, the states written, the bias."""
+    B, H = w.B, w.hidden_size
+    total = 0
+    for l, info in enumerate(infos):
+        in_l = w.input_size if l == 0 else H
+        total += info["algorithmic_bytes"] + (in_l + H) * B * 4 + 4 * H * B * 4
+        if w.bias[l] is not None:
+            total += 4 * H * 4
+    return total
+
+
+def encode_layers(binding, w, dev):
+    return [binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, dev) for m in w.layers]
+
+
+def make_runner(binding, torch, w, mats, host_io=False):
+    """Returns a zero-argument callable that performs one forward call, plus its I/O byte counts."""
+    L, B, H, T = len(w.layers), w.B, w.hidden_size, w.T
+    if host_io:
+        x = torch.from_numpy(w.x).pin_memory()
+        y = torch.empty((T, B, H), dtype=torch.float32).pin_memory()
+        hT = torch.empty((L, B, H), dtype=torch.float32).pin_memory()
+        cT = torch.empty((L, B, H), dtype=torch.float32).pin_memory()
+        flags = binding.CSB_FLAG_HOST_IO
+    else:
+        x = torch.from_numpy(w.x).cuda()
+        y = torch.empty((T, B, H), device="cuda")
+        hT = torch.empty((L, B, H), device="cuda")
+        cT = torch.empty((L, B, H), device="cuda")
+        flags = binding.CSB_FLAG_ASYNC
+    if w.cell == "lstm":
+        fn = lambda: binding.csb_lstm_forward(mats, None, x, None, None, y, hT, cT, flags)
+        d2h = (y.numel() + hT.numel() + cT.numel()) * 4
+    else:
+        fn = lambda: binding.csb_gru_forward(mats, None, x, None, y, hT, flags)
+        d2h = (y.numel() + hT.numel()) * 4
+    return fn, x.numel() * 4, d2h, (x, y, hT, cT)
+
+
+def time_calls(torch, fn, steps, warmup, flush):
+    """Mean milliseconds per call over `steps` calls, CUDA events on the current stream around each
+    call, an L2 flush (untimed) before each."""
+    for _ in range(warmup):
+        flush()
+        fn()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in ev:
+        flush()
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in ev]
+
+
+def spmv_sweep(binding, torch, dev, rates, batch, reps=10):
+    """Bare CSB-SpMV on the 8192x8192 / 64x64 matrix, cold: launches rotate through enough encoded
+    copies of the matrix to exceed L2, captured in one CUDA graph, timed with events."""
+    hbm, _ = peaks()
+    out = []
+    for rate in rates:
+        w = workloads.CONFIGS["cfg4"](rate=rate, B=batch)
+        m = w.matrix
+        A0 = binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, dev)
+        info = A0.info()
+        ncopy = max(2, int(160e6 // max(info["device_stream_bytes"], 1)) + 1)
+        As = [A0] + [binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, dev)
+                     for _ in range(ncopy - 1)]
+        X = torch.from_numpy(w.X).cuda()
+        Y = torch.empty((batch, m.rows), device="cuda")
+
+        def run(n):
+            for i in range(n):
+                if batch == 1:
+                    binding.csb_spmv(As[i % ncopy], X[0], Y[0])
+                else:
+                    binding.csb_spmm(As[i % ncopy], X, Y)
+        run(ncopy)
+        torch.cuda.synchronize()
+        n = 8 * ncopy
+        g = torch.cuda.CUDAGraph()
+        st = torch.cuda.Stream()
+        with torch.cuda.stream(st):
+            with torch.cuda.graph(g, stream=st):
+                run(n)
+        g.replay()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); g.replay(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) / n * 1e3)
+        us = float(np.median(ts))
+        alg = info["algorithmic_bytes"] + (m.cols + m.rows) * 4 * batch
+        out.append({"rate": rate, "batch": batch, "nnz": info["nnz"], "us": round(us, 3), "algorithmic_bytes": alg,
+                    "GBps": round(alg / us / 1e3, 1), "frac_hbm_measured": round(alg / us / 1e3 / hbm, 4),
+                    "frac_hbm_8TBps": round(alg / us / 1e3 / 8000.0, 4), "GFLOPs": round(2 * info["nnz"] * batch / us / 1e3, 1),
+                    "balance": round(info["balance"], 3), "copies": ncopy})
+        for a in As:
+            a.free()
+        del g
+    return out
+
+
+def other_configs(binding, torch, dev, flush, quick):
+    """Microseconds per timestep of the remaining recurrent workloads (device-resident inputs)."""
+    out = {}
+    cases = [("cfg1", dict()), ("cfg2", dict()), ("cfg3", dict(B=1)), ("cfg3", dict(B=8)), ("cfg5", dict(B=32, T=64))]
+    for name, kw in cases:
+        w = workloads.CONFIGS[name](**kw)
+        mats = encode_layers(binding, w, dev)
+        infos = [m.info() for m in mats]
+        fn, _, _, keep = make_runner(binding, torch, w, mats)
+        ms = time_calls(torch, fn, 3 if quick else 10, 3, flush)
+        us = float(np.median(ms)) * 1e3 / w.T
+        out["%s_B%d" % (name, w.B)] = {"us_per_timestep": round(us, 3), "T": w.T, "B": w.B,
+                                       "algorithmic_bytes_per_step": rnn_alg_bytes_per_step(w, infos),
+                                       "GFLOPs": round(2 * sum(i["nnz"] for i in infos) * w.B / us / 1e3, 1)}
+        for m in mats:
+            m.free()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sections", default="rnn,e2e,spmv,configs,cpu",
+                    help="comma list of: rnn (always), e2e, spmv, configs, cpu")
+    ap.add_argument("--seq-len", type=int, default=512)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        return reference_arm(args)
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the library")
+    from paper_2005_05758_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    sections = set(args.sections.split(",")) | {"rnn"}
+    if rank != 0:
+        sections &= {"rnn", "e2e"}
+    hbm, peak_kind = peaks()
+
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush = lambda: flush_buf.zero_()
+
+    w = workloads.CONFIGS["cfg5"](T=args.seq_len)
+    mats = encode_layers(binding, w, local)
+    infos = [m.info() for m in mats]
+    fn, _, _, keep = make_runner(binding, torch, w, mats)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    uuid = str(torch.cuda.get_device_properties(local).uuid)
+    uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+    for _ in range(args.warmup):
+        flush(); fn()
+    barrier()
+    sampler = ClockSampler(uuid) if rank == 0 else None
+    wall0 = time.perf_counter()
+    ms = time_calls(torch, fn, args.steps, 0, flush)
+    barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.stop() if sampler else None
+    mean_ms = float(np.mean(ms))
+    if dist is not None:
+        t = torch.tensor([mean_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        mean_ms = float(t.item())
+    us_step = mean_ms * 1e3 / (w.T * world)          # all replicas' timesteps over the slowest replica's time
+
+    line = {"metric": METRIC, "value": round(us_step, 4), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(mean_ms, 4), "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "seq_len": w.T, "batch": 1, "replicas": world,
+                       "l2": "flushed (256 MiB written) before every timed call; weights then stay on chip for the sequence",
+                       "paper_context": "0.79-6.58 us per frame on the paper's FPGA (other models, int16): not comparable"},
+            "gpu_launches": args.steps, "clocks": clocks, "wall_s_timed_region": round(wall, 3)}
+    alg_step = rnn_alg_bytes_per_step(w, infos)
+    achieved = alg_step * w.T / (mean_ms * 1e-3) / 1e9
+    line["roofline"] = {"kernel": "csb_rnn_kernel<half,1>", "bound": "hbm", "achieved": round(achieved, 1), "peak": hbm,
+                        "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / hbm, 4), "traffic": None,
+                        "algorithmic_bytes_per_launch": alg_step * w.T,
+                        "note": "weights are shared-memory resident, so DRAM traffic is far below the algorithmic bytes; "
+                                "the fraction compares the per-step compressed bytes with what HBM could stream"}
+    if "e2e" in sections:
+        fn_h, h2d, d2h, keep_h = make_runner(binding, torch, w, mats, host_io=True)
+        for _ in range(3):
+            fn_h()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            fn_h()                                     # synchronous: copies in, kernel, copies out
+        barrier()
+        e2e_ms = (time.perf_counter() - t0) / args.steps * 1e3
+        if dist is not None:
+            t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        line["e2e"] = {"value": round(e2e_ms * 1e3 / (w.T * world), 4), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                       "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4)}
+    for m in mats:
+        m.free()
+    if rank == 0 and "spmv" in sections:
+        line["spmv"] = spmv_sweep(binding, torch, local, [4.0, 8.0, 16.0, 25.0], 1)
+        best = max(line["spmv"], key=lambda r: r["frac_hbm_measured"])
+        line["roofline_spmv"] = {"kernel": "csb_product_kernel<half,1>", "bound": "hbm", "achieved": best["GBps"], "peak": hbm,
+                                 "peak_kind": peak_kind, "unit": "GB/s", "frac": best["frac_hbm_measured"], "traffic": None,
+                                 "workload": "cfg4 8192x8192, 64x64 blocks, rate %gx, batch 1, cold (rotating copies > L2)" % best["rate"]}
+    if rank == 0 and "configs" in sections:
+        line["configs"] = other_configs(binding, torch, local, flush, quick=False)
+    if rank == 0 and "cpu" in sections:
+        wc = workloads.CONFIGS["cfg5"](T=12)
+        v = oracle_us_per_step(wc, 2, 10)
+        line["cpu_baseline"] = {"value": round(v, 1), "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                "sample": "slope of the float64 oracle recurrence between 2 and 10 timesteps of cfg5"}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

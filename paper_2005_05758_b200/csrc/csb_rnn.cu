@@ -321,17 +321,27 @@ static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, i
     want = std::max(want, L * ((H + 47) / 48));        // tiles are cut by cost; leave room under the 64-unit limit
     want = env_int("CSB_RNN_CTAS", want);
     want = std::min(std::max(want, L), A0->sm_count);
+    // fewer warps per CTA shrink the per-warp accumulators and rings until the carve-up fits
     RnnHostPlan Hp;
-    int rc = plan_rnn_host(gates, L, W, in_size, H, want, P->warps, P->stage_bytes, &Hp);
-    if (rc != CSB_OK) return rc;
+    int rc = CSB_OK;
+    const int first = P->warps;
+    bool fits = false;
+    for (int wtry : {first, 12, 8, 6, 4, 2, 1}) {
+        if (wtry > first) continue;
+        Hp = RnnHostPlan();
+        rc = plan_rnn_host(gates, L, W, in_size, H, want, wtry, P->stage_bytes, &Hp);
+        if (rc != CSB_OK) return rc;
+        P->warps = wtry;
+        P->max_U = Hp.max_U; P->max_warp_bytes = (int)Hp.max_warp_bytes;
+        const RnnSmem res(wtry, P->stages, P->stage_bytes, 1, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
+        const RnnSmem str(wtry, P->stages, P->stage_bytes, 0, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
+        if (res.total <= A0->smem_optin && !env_int("CSB_RNN_STREAM", 0)) { P->resident = 1; P->smem = res.total; fits = true; break; }
+        if (str.total <= A0->smem_optin) { P->resident = 0; P->smem = str.total; fits = true; break; }
+    }
+    if (!fits) { set_error("time-loop kernel does not fit the %zu bytes of shared memory per CTA", A0->smem_optin); return CSB_ERR_LAUNCH; }
     P->n_ctas = (int)Hp.ctas.size();
-    P->max_U = Hp.max_U; P->max_warp_bytes = (int)Hp.max_warp_bytes; P->balance = Hp.balance;
+    P->balance = Hp.balance;
     P->stream_bytes = (int64_t)Hp.stream.bytes.size();
-    const RnnSmem res(P->warps, P->stages, P->stage_bytes, 1, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
-    const RnnSmem str(P->warps, P->stages, P->stage_bytes, 0, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
-    if (res.total <= A0->smem_optin && !env_int("CSB_RNN_STREAM", 0)) { P->resident = 1; P->smem = res.total; }
-    else if (str.total <= A0->smem_optin) { P->resident = 0; P->smem = str.total; }
-    else { set_error("time-loop kernel needs %zu bytes of shared memory per CTA, device offers %zu", str.total, A0->smem_optin); return CSB_ERR_LAUNCH; }
     if ((rc = upload_vec(Hp.stream.bytes, &P->d_stream)) != CSB_OK) return rc;
     if ((rc = upload_vec(Hp.stream.chunks, &P->d_chunks)) != CSB_OK) return rc;
     if ((rc = upload_vec(Hp.stream.warp_chunk_begin, &P->d_wcb)) != CSB_OK) return rc;
