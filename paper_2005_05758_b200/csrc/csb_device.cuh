@@ -67,104 +67,112 @@ template <> struct WordTraits<float> {
     __device__ static __forceinline__ void unpack(uint32_t w, float (&v)[1]) { v[0] = __uint_as_float(w); }
 };
 
-// Lane mapping of one item.  A word is kRows consecutive kept rows of one kept column; the
-// kernel matrix is stored column-major in words, RL words per column.  The warp is cut into
-// S = 32 / RL lane groups; group kg takes columns kg, kg + S, ...; inside a group lane rl owns
-// word rl of each column, i.e. the same output rows for the whole item.  A = S * RL lanes are
-// active and in step s they read words s*A .. s*A + A-1: consecutive, conflict-free.
-struct LaneMap {
-    int RL, S, A, kg;
-};
-template <int kRows>
-__device__ __forceinline__ LaneMap lane_map(int mr, int lane) {
-    LaneMap m;
-    m.RL = (mr + kRows - 1) / kRows;
-    m.S = 32 / m.RL;
-    m.A = m.S * m.RL;
-    m.kg = lane / m.RL;
-    return m;
+template <int N> struct Log2;
+template <> struct Log2<8> { static constexpr int v = 3; };
+template <> struct Log2<16> { static constexpr int v = 4; };
+template <> struct Log2<32> { static constexpr int v = 5; };
+
+// Size in bytes of a chunk, from its header (sum of the sub-stream sizes plus the header).
+__device__ __forceinline__ uint32_t chunk_bytes(const uint4& ch) {
+    return 16u + 16u * ((ch.x & 0xffffu) + (ch.x >> 16) + (ch.y & 0xffffu) + (ch.y >> 16));
 }
 
-// acc[q][bt] += sum over this lane's columns of value(row word, q) * xg[k][bt].
-template <typename T, int BT>
-__device__ __forceinline__ void item_mac(const uint32_t* __restrict__ vals, int nk, const LaneMap& lm, int lane,
-                                         const float* __restrict__ xg, float (&acc)[WordTraits<T>::kRows][BT]) {
+// Work through one chunk held in shared memory.  The warp is cut into G = 32 / GW lane groups;
+// group g walks sub-stream g, so G items are in flight and share every instruction.
+//
+// Lane mapping inside a group, per item: a word is kRows consecutive kept rows of one kept
+// column; the kernel matrix is stored column-major in words, RL words per column.  The group is
+// cut into S = GW / RL sub-groups; sub-group kg takes columns kg, kg + S, ...; lane rl of a
+// sub-group owns word rl of each column, i.e. the same output rows for the whole item.  The
+// A = S * RL active lanes read words s*A .. s*A + A-1 in step s: consecutive, conflict-free.
+//
+// Per item: gather the kept inputs through the column indices (gather(col, flags, bt) returns
+// input `col` of batch column bt) into xg, multiply, fold the sub-groups, and add into
+// zs[(zbase + row_idx) * BT + bt] of this group's private accumulators.
+//   xg_w: per warp, G * kMaxNk * BT floats;  zs_w: per warp, G * zs_stride floats.
+template <typename T, int BT, int GW, typename Gather>
+__device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch, int lane, float* __restrict__ xg_w,
+                                           float* __restrict__ zs_w, int zs_stride, Gather gather) {
     constexpr int R = WordTraits<T>::kRows;
-    if (lane < lm.A) {
-        const int nwords = nk * lm.RL;
-        int k = lm.kg;
-#pragma unroll 4
-        for (int w = lane; w < nwords; w += lm.A, k += lm.S) {
-            float v[R];
-            WordTraits<T>::unpack(vals[w], v);
+    const int g = lane / GW, gl = lane % GW;
+    const uint32_t sz[4] = {ch.x & 0xffffu, ch.x >> 16, ch.y & 0xffffu, ch.y >> 16};
+    uint32_t before = 0, mine = 0;
 #pragma unroll
-            for (int bt = 0; bt < BT; ++bt) {
-                const float xv = xg[k * BT + bt];
-#pragma unroll
-                for (int q = 0; q < R; ++q) acc[q][bt] = fmaf(v[q], xv, acc[q][bt]);
-            }
+    for (int j = 0; j < 32 / GW; ++j) {
+        if (j < g) before += sz[j];
+        if (j == g) mine = sz[j];
+    }
+    const uint8_t* p = chunk + 16 + 16 * before;
+    const uint8_t* end = p + 16 * mine;
+    float* xg = xg_w + g * (kMaxNk * BT);
+    float* zs = zs_w + g * zs_stride;
+    while (__any_sync(0xffffffffu, p < end)) {
+        int nk = 0, mr = 0, RL = 1, S = 1;
+        uint32_t xbase = 0, zbase = 0, magic = 1024, flags = 0;
+        if (p < end) {
+            const uint4 h = *reinterpret_cast<const uint4*>(p);
+            nk = (int)(h.x & 0xffu); mr = (int)((h.x >> 8) & 0xffu); RL = (int)((h.x >> 16) & 0xffu); S = (int)(h.x >> 24);
+            xbase = h.y; zbase = h.z; magic = h.w & 0xffffu; flags = h.w >> 16;
         }
-    }
-    // fold the lane groups onto group 0 (a tree over groups; S need not be a power of two)
-    for (int off = lm.RL; off < lm.A; off <<= 1) {
-#pragma unroll
-        for (int q = 0; q < R; ++q)
-#pragma unroll
-            for (int bt = 0; bt < BT; ++bt) {
-                const float o = __shfl_down_sync(0xffffffffu, acc[q][bt], off);
-                if (lane + off < lm.A) acc[q][bt] += o;
-            }
-    }
-}
-
-// Walk the items stored in [p, end) (shared memory).  For each item: gather the kept inputs
-// through the column indices (gather(col, tail, bt) returns input `col` of batch column bt),
-// multiply by the kernel matrix, add into zs[(zbase_local + row_idx) * BT + bt], then let
-// after(zbase, tail) act (flush of a finished block-row, or nothing).  zs_base(zbase) maps an
-// item's zbase to the index its rows are relative to inside zs.
-template <typename T, int BT, typename Gather, typename ZsBase, typename After>
-__device__ __forceinline__ void walk_items(const uint8_t* p, const uint8_t* end, int lane, float* __restrict__ xg,
-                                           float* __restrict__ zs, Gather gather, ZsBase zs_base, After after) {
-    constexpr int R = WordTraits<T>::kRows;
-    while (p < end) {
-        const uint4 h = *reinterpret_cast<const uint4*>(p);
-        const int nk = (int)(h.x & 0xffffu), mr = (int)(h.x >> 16);
-        const uint32_t xbase = h.y, zbase = h.z, tail = h.w;
         const uint8_t* cidx = p + 16;
         const uint8_t* ridx = cidx + nk;
         const int idx_bytes = (nk + mr + 3) & ~3;
         const uint32_t* vals = reinterpret_cast<const uint32_t*>(p + 16 + idx_bytes);
-        const int RLw = (mr + R - 1) / R;
-        p += (16 + idx_bytes + nk * RLw * 4 + 15) & ~15;
-        if (nk > 0 && mr > 0) {
-            for (int k = lane; k < nk; k += 32) {
-                const uint32_t col = xbase + cidx[k];
+        const int nwords = nk * RL;
+        if (p < end) p += (16 + idx_bytes + nwords * 4 + 15) & ~15;
+
+        for (int k = gl; k < nk; k += GW) {
+            const uint32_t col = xbase + cidx[k];
 #pragma unroll
-                for (int bt = 0; bt < BT; ++bt) xg[k * BT + bt] = gather(col, tail, bt);
+            for (int bt = 0; bt < BT; ++bt) xg[k * BT + bt] = gather(col, flags, bt);
+        }
+        __syncwarp();
+        const int kg = (int)(((uint32_t)gl * magic) >> 10);
+        const int A = S * RL;
+        float acc[R][BT];
+#pragma unroll
+        for (int q = 0; q < R; ++q)
+#pragma unroll
+            for (int bt = 0; bt < BT; ++bt) acc[q][bt] = 0.f;
+        if (gl < A) {
+            int k = kg;
+#pragma unroll 4
+            for (int w = gl; w < nwords; w += A, k += S) {
+                float v[R];
+                WordTraits<T>::unpack(vals[w], v);
+#pragma unroll
+                for (int bt = 0; bt < BT; ++bt) {
+                    const float xv = xg[k * BT + bt];
+#pragma unroll
+                    for (int q = 0; q < R; ++q) acc[q][bt] = fmaf(v[q], xv, acc[q][bt]);
+                }
             }
-            __syncwarp();
-            const LaneMap lm = lane_map<R>(mr, lane);
-            float acc[R][BT];
+        }
+        // fold the sub-groups onto sub-group 0: a tree over kg (S need not be a power of two)
+#pragma unroll
+        for (int r = 0; r < Log2<GW>::v; ++r) {
+            const int off = RL << r;
+            const bool take = off < A && gl + off < A;
 #pragma unroll
             for (int q = 0; q < R; ++q)
 #pragma unroll
-                for (int bt = 0; bt < BT; ++bt) acc[q][bt] = 0.f;
-            item_mac<T, BT>(vals, nk, lm, lane, xg, acc);
-            if (lane < lm.RL) {
-                float* zrow = zs + zs_base(zbase) * BT;
+                for (int bt = 0; bt < BT; ++bt) {
+                    const float o = __shfl_down_sync(0xffffffffu, acc[q][bt], off < GW ? off : 0, GW);
+                    if (take) acc[q][bt] += o;
+                }
+        }
+        if (gl < RL) {
 #pragma unroll
-                for (int q = 0; q < R; ++q) {
-                    const int r = lane * R + q;
-                    if (r < mr) {
-                        float* z = zrow + (int)ridx[r] * BT;
+            for (int q = 0; q < R; ++q) {
+                const int r = gl * R + q;
+                if (r < mr) {
+                    float* z = zs + ((int)zbase + (int)ridx[r]) * BT;
 #pragma unroll
-                        for (int bt = 0; bt < BT; ++bt) z[bt] += acc[q][bt];
-                    }
+                    for (int bt = 0; bt < BT; ++bt) z[bt] += acc[q][bt];
                 }
             }
-            __syncwarp();
         }
-        after(zbase, tail);
+        __syncwarp();
     }
 }
 

@@ -18,30 +18,45 @@ void clear_error();
 
 // ---- device stream format -------------------------------------------------
 // The private device layout is a byte stream per warp, cut into chunks that one
-// bulk copy moves into a shared-memory ring stage.  A chunk holds whole items;
-// an item is one block (or a slice of one) of the CSB matrix:
+// bulk copy moves into shared memory.  A warp is split into G = 32 / GW lane
+// groups of GW lanes (GW is fixed per stream); every group works through its own
+// list of items, so G items are in flight per warp.
 //
-//   ItemHeader (16 B)
-//   col_idx[nk]  uint8   gather indices, relative to xbase
-//   row_idx[mr]  uint8   scatter indices, relative to zbase      (padded to 4 B)
-//   values       nk columns of RL "row words" each, column-major (k-major):
-//                  f16: a word is two consecutive kept rows (half2), RL = ceil(mr/2)
-//                  f32: a word is one kept row, RL = mr
-//                padding rows inside the last word are zero      (item padded to 16 B)
+//   chunk  = ChunkHeader (16 B), then the G sub-streams back to back
+//   sub-stream g = the items of lane group g, each aligned to 16 B
+//   item   = ItemHeader (16 B)
+//            col_idx[nk]  uint8   gather indices, relative to xbase
+//            row_idx[mr]  uint8   scatter indices, relative to zbase   (padded to 4 B)
+//            values       nk columns of RL "row words" each, column-major:
+//                           f16: a word is two consecutive kept rows (half2), RL = ceil(mr/2)
+//                           f32: a word is one kept row, RL = mr
+//                         padding rows inside the last word are zero  (item padded to 16 B)
 //
-// Column-major kernel matrices let one lane own a pair of output rows for the
-// whole item, so products need no cross-lane reduction except across the few
-// lane groups that split the columns.
+// An item is one block of the CSB matrix or a slice of it (a range of its kept
+// rows and of its kept columns).  Column-major kernel matrices let one lane own
+// the same output rows for the whole item, so a product needs no cross-lane
+// reduction except across the S = GW / RL lane sub-groups that split the columns.
 struct ItemHeader {
-    uint16_t nk;       // kept columns in this item (<= kMaxNk)
-    uint16_t mr;       // kept rows in this item (<= 64 for f16, <= 32 for f32)
+    uint8_t nk;        // kept columns in this item (<= kMaxNk)
+    uint8_t mr;        // kept rows in this item (<= GW * rows per word)
+    uint8_t RL;        // row words per column
+    uint8_t S;         // column sub-groups, GW / RL
     uint32_t xbase;    // first column of the block in the gathered vector
-    uint32_t zbase;    // first accumulator slot / matrix row of the block
-    uint32_t tail;     // bits 0..1 flush kind, bit 2 source select (recurrent), bits 3.. slot id
+    uint32_t zbase;    // first accumulator slot of the block's rows
+    uint16_t magic;    // ceil(1024 / RL): lane / RL == (lane * magic) >> 10 for lane < 32
+    uint16_t flags;    // bit 0: columns index the recurrent (h) vector
 };
 static_assert(sizeof(ItemHeader) == 16, "header is one 16-byte word");
 
-enum : uint32_t { kFlushNone = 0, kFlushDirect = 1, kFlushPartial = 2, kSrcRecurrent = 4, kSlotShift = 3 };
+struct ChunkHeader {
+    uint16_t sub16[4]; // size of each lane group's sub-stream in 16-byte units
+    uint32_t zbase;    // product: first matrix row of the block-row this chunk belongs to
+    uint32_t tail;     // bits 0..1 flush kind, bits 3.. partial-sum slot
+};
+static_assert(sizeof(ChunkHeader) == 16, "header is one 16-byte word");
+
+enum : uint32_t { kFlushNone = 0, kFlushDirect = 1, kFlushPartial = 2, kSlotShift = 3 };
+enum : uint16_t { kItemRecurrent = 1 };
 enum { kMaxNk = 64, kItemAlign = 16 };
 
 struct Chunk {
@@ -56,11 +71,12 @@ struct StreamPlan {
     std::vector<uint32_t> warp_chunk_begin; // [n_warps + 1]
     std::vector<double> warp_cost;
     int n_warps = 0;
+    int group_width = 32;                  // GW
 };
 
 // Planned product (SpMV / SpMM) on the device.
 struct ProductPlan {
-    int ctas = 0, warps = 0, stage_bytes = 0, stages = 0;
+    int ctas = 0, warps = 0, stage_bytes = 0, stages = 0, group_width = 32;
     int x_in_smem = 0;
     size_t smem_bytes = 0;
     uint8_t* d_stream = nullptr;
@@ -123,15 +139,23 @@ struct ItemSpec {
     int k0, k1;          // range [k0, k1) into the block's kept-column list
     uint32_t xbase, zbase;
     int ridx_bias;       // subtracted from the in-block row index before it is stored
-    uint32_t tail;       // flush kind / source / slot, ready for the header
+    uint16_t flags;
+};
+// A run of items of one warp that ends in one action (flush of a block-row, or nothing).
+struct Segment {
+    std::vector<ItemSpec> items;
+    uint32_t zbase = 0, tail = 0;
 };
 size_t item_bytes(const csb_matrix* A, const ItemSpec& it);
-void emit_item(const csb_matrix* A, const ItemSpec& it, std::vector<uint8_t>& out);
-// Cut per-warp item lists into chunks and lay them out back to back.
-void build_stream(const csb_matrix* A, const std::vector<std::vector<ItemSpec>>& per_warp,
-                  int stage_bytes, StreamPlan* out);
-void slice_block(const csb_matrix* A, int64_t b, int r0, int r1, int k0, int k1, int value_budget,
+int item_steps(const csb_matrix* A, const ItemSpec& it, int gw);
+void emit_item(const csb_matrix* A, const ItemSpec& it, int gw, std::vector<uint8_t>& out);
+// Cut per-warp segment lists into chunks and append them to the stream.
+void build_stream(const csb_matrix* A, const std::vector<std::vector<Segment>>& per_warp, int stage_bytes,
+                  StreamPlan* out);
+void slice_block(const csb_matrix* A, int64_t b, int r0, int r1, int k0, int k1, int max_rows, int value_budget,
                  ItemSpec proto, std::vector<ItemSpec>* out);
+int item_value_budget(int stage_bytes, int gw);
+int pick_group_width(const std::vector<int>& item_row_words);
 struct ProductHostPlan {
     StreamPlan stream;
     std::vector<uint32_t> part_base, part_count;   // per block-row
@@ -147,7 +171,7 @@ struct RnnCtaDesc {
 };
 enum { kMaxTileUnits = 64, kMaxLayers = 8 };
 struct RnnHostPlan {
-    StreamPlan stream;
+    StreamPlan stream;                 // stream.group_width is chosen by the planner
     std::vector<RnnCtaDesc> ctas;
     int warps = 0, max_U = 0;
     size_t max_warp_bytes = 0;

@@ -9,8 +9,8 @@
 #include <algorithm>
 #include <cstdio>
 
-#include "csb_device.cuh"
 #include "csb_internal.hpp"
+#include "csb_device.cuh"
 
 namespace csb {
 
@@ -34,74 +34,78 @@ __host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t
 // Shared-memory carve-up, identical on host and device.
 struct ProductSmem {
     size_t ring, bars, zs, xg, xs, total;
-    int zs_stride;
-    __host__ __device__ ProductSmem(int W, int stages, int stage_bytes, int block_r, int BT, int cols_in_smem) {
+    int zs_stride;                                     // floats per lane group
+    __host__ __device__ ProductSmem(int W, int G, int stages, int stage_bytes, int block_r, int BT, int cols_in_smem) {
         zs_stride = block_r * BT;
         ring = 0;
         bars = ring + (size_t)W * stages * stage_bytes;
         zs = align16(bars + (size_t)W * stages * 8);
-        xg = align16(zs + (size_t)W * zs_stride * 4);
-        xs = align16(xg + (size_t)W * kMaxNk * BT * 4);
+        xg = align16(zs + (size_t)W * G * zs_stride * 4);
+        xs = align16(xg + (size_t)W * G * kMaxNk * BT * 4);
         total = align16(xs + (size_t)cols_in_smem * 4);
     }
 };
 
-// A warp that holds only part of a block-row parks its sums in its own slot; the warp that
-// arrives last adds all slots of that block-row in slot order and writes y.
-template <int BT>
-__device__ __forceinline__ void flush_partial(const ProductArgs& a, float* zs, uint32_t zbase, uint32_t tail, int nrows, int lane) {
-                        const uint32_t slot = tail >> kSlotShift;
-                        const uint32_t bi = zbase / (uint32_t)a.block_r;
-                        float* dst = a.partials + (size_t)slot * a.block_r * BT;
-                        for (int i = lane; i < nrows * BT; i += 32) { __stcg(dst + i, zs[i]); zs[i] = 0.f; }
-                        __threadfence();
-                        __syncwarp();
-                        int last = 0;
-                        if (lane == 0) last = (atomicAdd(&a.arrivals[bi], 1u) == a.part_count[bi] - 1u);
-                        last = __shfl_sync(0xffffffffu, last, 0);
-                        if (last) {
-                            // this warp saw every other contributor arrive: add the partial sums in slot
-                            // order (fixed, so the result does not depend on who came last)
-                            __threadfence();
-                            const uint32_t pb = a.part_base[bi], pc = a.part_count[bi];
-                            const size_t pstride = (size_t)a.block_r * BT;
-                            for (int i = lane; i < nrows * BT; i += 32) {
-                                // eight loads in flight; the grouping is fixed, so the sum is reproducible
-                                const float* src = a.partials + (size_t)pb * pstride + i;
-                                float s[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                                uint32_t q = 0;
-                                for (; q + 8 <= pc; q += 8) {
-                                    float v[8];
-    #pragma unroll
-                                    for (int j = 0; j < 8; ++j) v[j] = __ldcg(src + (size_t)(q + j) * pstride);
-    #pragma unroll
-                                    for (int j = 0; j < 8; ++j) s[j] += v[j];
-                                }
-                                {
-                                    float v[8];
-    #pragma unroll
-                                    for (int j = 0; j < 8; ++j) v[j] = (q + j < pc) ? __ldcg(src + (size_t)(q + j) * pstride) : 0.f;
-    #pragma unroll
-                                    for (int j = 0; j < 8; ++j) s[j] += v[j];
-                                }
-                                const float sum = ((s[0] + s[1]) + (s[2] + s[3])) + ((s[4] + s[5]) + (s[6] + s[7]));
-                                const int r = i / BT, bt = i % BT;
-                                if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = sum;
-                            }
-                            if (lane == 0) a.arrivals[bi] = 0u;      // ready for the next launch
-                        }
+// End of a block-row inside a warp: add the lane groups' private sums in group order, then
+// either store to y (the warp owned the whole block-row) or park the sums in the warp's slot;
+// the warp that arrives last adds all slots of that block-row in slot order and writes y.
+template <int BT, int G>
+__device__ __forceinline__ void flush_block_row(const ProductArgs& a, float* zs, int zs_stride, uint32_t zbase, uint32_t tail,
+                                                int lane) {
+    const int nrows = min(a.block_r, a.rows - (int)zbase);
+    const bool direct = (tail & 3u) == kFlushDirect;
+    float* dst = a.partials + (size_t)(tail >> kSlotShift) * a.block_r * BT;
+    for (int i = lane; i < nrows * BT; i += 32) {
+        float v = zs[i];
+        zs[i] = 0.f;
+#pragma unroll
+        for (int g = 1; g < G; ++g) { v += zs[g * zs_stride + i]; zs[g * zs_stride + i] = 0.f; }
+        if (direct) {
+            const int r = i / BT, bt = i % BT;
+            if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = v;
+        } else {
+            __stcg(dst + i, v);
+        }
+    }
+    if (direct) return;
+    const uint32_t bi = zbase / (uint32_t)a.block_r;
+    __threadfence();
+    __syncwarp();
+    int last = 0;
+    if (lane == 0) last = (atomicAdd(&a.arrivals[bi], 1u) == a.part_count[bi] - 1u);
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (!last) return;
+    __threadfence();
+    const uint32_t pb = a.part_base[bi], pc = a.part_count[bi];
+    const size_t pstride = (size_t)a.block_r * BT;
+    for (int i = lane; i < nrows * BT; i += 32) {
+        // eight loads in flight; the grouping is fixed, so the sum is reproducible
+        const float* src = a.partials + (size_t)pb * pstride + i;
+        float s[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (uint32_t q = 0; q < pc; q += 8) {
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = (q + j < pc) ? __ldcg(src + (size_t)(q + j) * pstride) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s[j] += v[j];
+        }
+        const float sum = ((s[0] + s[1]) + (s[2] + s[3])) + ((s[4] + s[5]) + (s[6] + s[7]));
+        const int r = i / BT, bt = i % BT;
+        if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = sum;
+    }
+    if (lane == 0) a.arrivals[bi] = 0u;                // ready for the next launch
 }
 
-template <typename T, int BT>
+template <typename T, int BT, int GW>
 __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a) {
     extern __shared__ __align__(128) uint8_t smem[];
-    constexpr int R = WordTraits<T>::kRows;
+    constexpr int G = 32 / GW;
     const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const ProductSmem L(W, a.stages, a.stage_bytes, a.block_r, BT, a.x_in_smem ? a.cols : 0);
+    const ProductSmem L(W, G, a.stages, a.stage_bytes, a.block_r, BT, a.x_in_smem ? a.cols : 0);
     uint8_t* ring = smem + L.ring + (size_t)warp * a.stages * a.stage_bytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.bars) + warp * a.stages;
-    float* zs = reinterpret_cast<float*>(smem + L.zs) + warp * L.zs_stride;
-    float* xg = reinterpret_cast<float*>(smem + L.xg) + warp * kMaxNk * BT;
+    float* zs = reinterpret_cast<float*>(smem + L.zs) + warp * G * L.zs_stride;
+    float* xg = reinterpret_cast<float*>(smem + L.xg) + warp * G * kMaxNk * BT;
     const float* xs = reinterpret_cast<const float*>(smem + L.xs);
 
     const int gw = blockIdx.x * W + warp;
@@ -117,23 +121,26 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
             bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)ch.off16 * 16, ch.bytes, &bars[s]);
         }
     }
-    for (int i = lane; i < L.zs_stride; i += 32) zs[i] = 0.f;
+    for (int i = lane; i < G * L.zs_stride; i += 32) zs[i] = 0.f;
     if (a.x_in_smem) {
         float* xw = reinterpret_cast<float*>(smem + L.xs);
-        for (int i = threadIdx.x; i < a.cols; i += blockDim.x) xw[i] = __ldg(a.X + i);
+        if ((reinterpret_cast<uintptr_t>(a.X) & 15) == 0) {
+            const float4* x4 = reinterpret_cast<const float4*>(a.X);
+            for (int i = threadIdx.x; i < a.cols / 4; i += blockDim.x) reinterpret_cast<float4*>(xw)[i] = __ldg(x4 + i);
+            for (int i = (a.cols & ~3) + threadIdx.x; i < a.cols; i += blockDim.x) xw[i] = __ldg(a.X + i);
+        } else {
+            for (int i = threadIdx.x; i < a.cols; i += blockDim.x) xw[i] = __ldg(a.X + i);
+        }
         __syncthreads();
     } else {
         __syncwarp();
     }
 
-    bool dead = false;
-    Chunk cur = (c0 < c1) ? a.chunks[c0] : Chunk{0, 0};
     for (uint32_t c = c0; c < c1; ++c) {
         const int s = (int)((c - c0) % (uint32_t)a.stages);
         const uint32_t parity = ((c - c0) / (uint32_t)a.stages) & 1u;
-        const Chunk nxt = (c + 1 < c1) ? a.chunks[c + 1] : Chunk{0, 0};
         const Chunk refill = (c + a.stages < c1) ? a.chunks[c + a.stages] : Chunk{0, 0};
-        if (!mbar_wait_bounded(&bars[s], parity)) { dead = true; }
+        bool dead = !mbar_wait_bounded(&bars[s], parity);
         dead = __any_sync(0xffffffffu, dead);
         if (dead) {
             // report, then give the copies still in flight a bounded chance to land before leaving
@@ -144,40 +151,22 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
             }
             break;
         }
-
         const uint8_t* p = ring + (size_t)s * a.stage_bytes;
-        const uint8_t* end = p + cur.bytes;
-        walk_items<T, BT>(
-            p, end, lane, xg, zs,
-            [&](uint32_t col, uint32_t, int bt) -> float {
-                if (BT == 1) return a.x_in_smem ? xs[col] : __ldg(a.X + col);
-                return bt < a.nb ? __ldg(a.X + (long long)bt * a.ldx + col) : 0.f;
-            },
-            [](uint32_t) { return 0; },
-            [&](uint32_t zbase, uint32_t tail) {
-                const uint32_t flush = tail & 3u;
-                if (flush == kFlushNone) return;
-                const int nrows = min(a.block_r, a.rows - (int)zbase);
-                if (flush == kFlushDirect) {
-                    for (int i = lane; i < nrows * BT; i += 32) {
-                        const int r = i / BT, bt = i % BT;
-                        if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = zs[i];
-                        zs[i] = 0.f;
-                    }
-                } else {
-                    flush_partial<BT>(a, zs, zbase, tail, nrows, lane);
-                }
-                __syncwarp();
-            });
-        __syncwarp();
+        const uint4 ch = *reinterpret_cast<const uint4*>(p);
+        walk_chunk<T, BT, GW>(p, ch, lane, xg, zs, L.zs_stride, [&](uint32_t col, uint32_t, int bt) -> float {
+            if (BT == 1) return a.x_in_smem ? xs[col] : __ldg(a.X + col);
+            return bt < a.nb ? __ldg(a.X + (long long)bt * a.ldx + col) : 0.f;
+        });
+        if ((ch.w & 3u) != kFlushNone) {
+            flush_block_row<BT, G>(a, zs, L.zs_stride, ch.z, ch.w, lane);
+            __syncwarp();
+        }
         if (lane == 0 && refill.bytes) {
             mbar_expect_tx(&bars[s], refill.bytes);
             bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)refill.off16 * 16, refill.bytes, &bars[s]);
         }
-        cur = nxt;
     }
 }
-
 
 #define CSB_CUDA(call)                                                                     \
     do {                                                                                   \
@@ -204,7 +193,7 @@ enum { kMaxBatchTile = 8 };
 static int fit_warps(const csb_matrix* A, int want, int BT, int cols_in_smem, size_t* smem) {
     const ProductPlan& P = A->product;
     for (int W = want; W >= 1; --W) {
-        const ProductSmem L(W, P.stages, P.stage_bytes, A->block_r, BT, cols_in_smem);
+        const ProductSmem L(W, 32 / P.group_width, P.stages, P.stage_bytes, A->block_r, BT, cols_in_smem);
         if (L.total <= A->smem_optin) { *smem = L.total; return W; }
     }
     return 0;
@@ -222,9 +211,9 @@ int plan_product(csb_matrix* A) {
     A->smem_optin = prop.sharedMemPerBlockOptin;
     const int ctas = A->opts.ctas > 0 ? A->opts.ctas : A->sm_count;
     const int wpc = std::min(16, A->opts.warps_per_cta > 0 ? A->opts.warps_per_cta : 16);
-    P.stage_bytes = ((A->opts.stage_bytes > 0 ? A->opts.stage_bytes : 3072) + 15) & ~15;
+    P.stage_bytes = ((A->opts.stage_bytes > 0 ? A->opts.stage_bytes : 4096) + 15) & ~15;
     P.stage_bytes = std::max(P.stage_bytes, 1024);
-    P.stages = std::min(8, std::max(1, A->opts.stages > 0 ? A->opts.stages : 3));
+    P.stages = std::min(8, std::max(1, A->opts.stages > 0 ? A->opts.stages : 2));
     // small matrices: no more warps than there is work for (about 2 KB of stream each)
     const int64_t approx = A->nnz * val_size(A->val_dtype) + (int64_t)A->ridx_off[A->nblk] + A->cidx_off[A->nblk] + 16 * A->nblk;
     const int64_t useful = std::max<int64_t>(1, approx / 2048);
@@ -235,6 +224,7 @@ int plan_product(csb_matrix* A) {
     P.warps = std::max(1, (n_warps + ctas - 1) / ctas);
     P.ctas = (n_warps + P.warps - 1) / P.warps;
     P.n_slots = H.n_slots;
+    P.group_width = H.stream.group_width;
     P.balance = H.balance;
     P.stream_bytes = (int64_t)H.stream.bytes.size();
     P.n_warps = n_warps;
@@ -267,7 +257,7 @@ void free_product(csb_matrix* A) {
     cudaSetDevice(prev);
 }
 
-template <typename T, int BT>
+template <typename T, int BT, int GW>
 static int launch_tile(const csb_matrix* A, ProductArgs a, cudaStream_t st) {
     const ProductPlan& P = A->product;
     size_t smem = 0;
@@ -282,12 +272,28 @@ static int launch_tile(const csb_matrix* A, ProductArgs a, cudaStream_t st) {
     const int ctas = (P.n_warps + W - 1) / W;
     static bool configured[64] = {};                   // per device; setting it twice is harmless
     if (A->device >= 64 || !configured[A->device]) {
-        CSB_CUDA(cudaFuncSetAttribute(csb_product_kernel<T, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)A->smem_optin));
+        CSB_CUDA(cudaFuncSetAttribute(csb_product_kernel<T, BT, GW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)A->smem_optin));
         if (A->device < 64) configured[A->device] = true;
     }
-    csb_product_kernel<T, BT><<<ctas, W * 32, smem, st>>>(a);
+    csb_product_kernel<T, BT, GW><<<ctas, W * 32, smem, st>>>(a);
     CSB_CUDA(cudaGetLastError());
     return CSB_OK;
+}
+
+template <typename T, int BT>
+static int dispatch_gw(const csb_matrix* A, const ProductArgs& a, cudaStream_t st) {
+    switch (A->product.group_width) {
+        case 8: return launch_tile<T, BT, 8>(A, a, st);
+        case 16: return launch_tile<T, BT, 16>(A, a, st);
+        default: return launch_tile<T, BT, 32>(A, a, st);
+    }
+}
+
+static int dispatch_tile(const csb_matrix* A, const ProductArgs& a, cudaStream_t st, int bt) {
+    const bool h = A->val_dtype == CSB_F16;
+    if (bt == 8) return h ? dispatch_gw<__half, 8>(A, a, st) : dispatch_gw<float, 8>(A, a, st);
+    if (bt == 4) return h ? dispatch_gw<__half, 4>(A, a, st) : dispatch_gw<float, 4>(A, a, st);
+    return h ? dispatch_gw<__half, 1>(A, a, st) : dispatch_gw<float, 1>(A, a, st);
 }
 
 int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream) {
@@ -308,10 +314,7 @@ int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, 
         for (int cand : kBatchTiles) if (batch - b0 >= cand || cand == 1) { bt = cand; break; }
         if (batch - b0 > 1 && bt == 1) bt = 4;          // 2 or 3 left: one padded tile of 4
         a.X = X + (int64_t)b0 * ldx; a.Y = Y + (int64_t)b0 * ldy; a.nb = std::min(bt, batch - b0);
-        const bool h = A->val_dtype == CSB_F16;
-        if (bt == 8) rc = h ? launch_tile<__half, 8>(A, a, st) : launch_tile<float, 8>(A, a, st);
-        else if (bt == 4) rc = h ? launch_tile<__half, 4>(A, a, st) : launch_tile<float, 4>(A, a, st);
-        else rc = h ? launch_tile<__half, 1>(A, a, st) : launch_tile<float, 1>(A, a, st);
+        rc = dispatch_tile(A, a, st, bt);
         b0 += a.nb;
     }
     if (prev != A->device) cudaSetDevice(prev);

@@ -12,8 +12,8 @@
 #include <memory>
 #include <mutex>
 
-#include "csb_device.cuh"
 #include "csb_internal.hpp"
+#include "csb_device.cuh"
 
 namespace csb {
 
@@ -38,15 +38,15 @@ struct RnnArgs {
 struct RnnSmem {
     size_t weights, bars, zs, xg, v, cs, flag, total;
     int zs_stride;
-    __host__ __device__ RnnSmem(int W, int stages, int stage_bytes, int resident, int max_warp_bytes, int max_U, int BT,
+    __host__ __device__ RnnSmem(int W, int G, int stages, int stage_bytes, int resident, int max_warp_bytes, int max_U, int BT,
                                 int B, int max_C) {
-        zs_stride = 4 * max_U * BT;
+        zs_stride = 4 * max_U * BT;                    // floats per lane group
         weights = 0;
         const size_t per_warp = resident ? (size_t)max_warp_bytes : (size_t)stages * stage_bytes;
         bars = weights + (size_t)W * per_warp;
         zs = (bars + (size_t)W * (resident ? 1 : stages) * 8 + 15) & ~(size_t)15;
-        xg = (zs + (size_t)W * zs_stride * 4 + 15) & ~(size_t)15;
-        v = (xg + (size_t)W * kMaxNk * BT * 4 + 15) & ~(size_t)15;
+        xg = (zs + (size_t)W * G * zs_stride * 4 + 15) & ~(size_t)15;
+        v = (xg + (size_t)W * G * kMaxNk * BT * 4 + 15) & ~(size_t)15;
         cs = (v + (BT == 1 ? (size_t)max_C * 4 : 0) + 15) & ~(size_t)15;
         flag = (cs + (size_t)max_U * B * 4 + 15) & ~(size_t)15;
         total = flag + 16;
@@ -85,11 +85,12 @@ __device__ __forceinline__ bool grid_barrier(const RnnArgs& a, unsigned int targ
 
 __device__ __forceinline__ float sigmoidf_acc(float a) { return 1.f / (1.f + expf(-a)); }
 
-template <typename T, int BT>
+template <typename T, int BT, int GW>
 __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     extern __shared__ __align__(128) uint8_t smem[];
+    constexpr int G = 32 / GW;
     const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const RnnSmem S(W, a.stages, a.stage_bytes, a.resident, a.max_warp_bytes, a.max_U, BT, a.B, a.max_C);
+    const RnnSmem S(W, G, a.stages, a.stage_bytes, a.resident, a.max_warp_bytes, a.max_U, BT, a.B, a.max_C);
     const RnnCtaDesc me = a.ctas[blockIdx.x];
     const int layer = me.layer, U = me.U, u0 = me.u0, H = a.H, B = a.B;
     const int I = a.in_size[layer], C = I + H;
@@ -97,8 +98,8 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     uint8_t* wbuf = smem + S.weights + warp * per_warp;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S.bars) + warp * (a.resident ? 1 : a.stages);
     float* zs_all = reinterpret_cast<float*>(smem + S.zs);
-    float* zs = zs_all + warp * S.zs_stride;
-    float* xg = reinterpret_cast<float*>(smem + S.xg) + warp * kMaxNk * BT;
+    float* zs = zs_all + warp * G * S.zs_stride;
+    float* xg = reinterpret_cast<float*>(smem + S.xg) + warp * G * kMaxNk * BT;
     float* vs = reinterpret_cast<float*>(smem + S.v);
     float* cs = reinterpret_cast<float*>(smem + S.cs);
     volatile int* s_flag = reinterpret_cast<volatile int*>(smem + S.flag);
@@ -159,29 +160,31 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
             float* h_dst = a.hbuf + ((size_t)layer * 2 + (t & 1)) * B * H;
             const int in_ld = layer == 0 ? I : H;
             if (BT == 1) {
-                for (int i = threadIdx.x; i < C; i += blockDim.x)
-                    vs[i] = i < I ? (layer == 0 ? __ldg(in_src + i) : __ldcg(in_src + i)) : __ldcg(rec_src + (i - I));
+#pragma unroll 8
+                for (int i = threadIdx.x; i < C; i += blockDim.x) vs[i] = __ldcg(i < I ? in_src + i : rec_src + (i - I));
                 __syncthreads();
             }
             for (int b0 = 0; b0 < B; b0 += BT) {
                 const int nb = min(BT, B - b0);
-                for (int i = lane; i < S.zs_stride; i += 32) zs[i] = 0.f;
+                for (int i = lane; i < G * S.zs_stride; i += 32) zs[i] = 0.f;
                 __syncwarp();
-                auto gather = [&](uint32_t col, uint32_t tail, int bt) -> float {
-                    if (BT == 1) return vs[(tail & kSrcRecurrent) ? col + I : col];
+                auto gather = [&](uint32_t col, uint32_t flags, int bt) -> float {
+                    if (BT == 1) return vs[(flags & kItemRecurrent) ? col + I : col];
                     if (bt >= nb) return 0.f;
-                    return (tail & kSrcRecurrent) ? __ldcg(rec_src + (size_t)(b0 + bt) * H + col)
-                                                  : __ldcg(in_src + (size_t)(b0 + bt) * in_ld + col);
+                    return (flags & kItemRecurrent) ? __ldcg(rec_src + (size_t)(b0 + bt) * H + col)
+                                                    : __ldcg(in_src + (size_t)(b0 + bt) * in_ld + col);
                 };
-                auto zs_base = [](uint32_t zbase) { return (int)zbase; };
-                auto after = [](uint32_t, uint32_t) {};
                 if (a.resident) {
-                    if (alive) walk_items<T, BT>(wbuf, wbuf + wbytes, lane, xg, zs, gather, zs_base, after);
+                    if (alive)
+                        for (const uint8_t* p = wbuf; p < wbuf + wbytes;) {
+                            const uint4 ch = *reinterpret_cast<const uint4*>(p);
+                            walk_chunk<T, BT, GW>(p, ch, lane, xg, zs, S.zs_stride, gather);
+                            p += chunk_bytes(ch);
+                        }
                 } else {
                     for (uint32_t c = 0; c < nchunks && alive; ++c) {
                         const int s = (int)(n_done % (unsigned)a.stages);
                         const uint32_t parity = (uint32_t)((n_done / (unsigned)a.stages) & 1u);
-                        const Chunk ch = a.chunks[c0 + c];
                         if (!mbar_wait_bounded(&bars[s], parity)) alive = false;
                         alive = !__any_sync(0xffffffffu, !alive);
                         if (!alive) {
@@ -191,7 +194,8 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                             break;
                         }
                         const uint8_t* p = wbuf + (size_t)s * a.stage_bytes;
-                        walk_items<T, BT>(p, p + ch.bytes, lane, xg, zs, gather, zs_base, after);
+                        const uint4 ch = *reinterpret_cast<const uint4*>(p);
+                        walk_chunk<T, BT, GW>(p, ch, lane, xg, zs, S.zs_stride, gather);
                         __syncwarp();
                         ++n_done;
                         if (lane == 0 && n_done + a.stages - 1 < n_total) {
@@ -207,7 +211,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                 for (int i = threadIdx.x; i < U * nb; i += blockDim.x) {
                     const int bt = i / U, u = i % U, b = b0 + bt;
                     float z[4] = {0.f, 0.f, 0.f, 0.f};
-                    for (int w = 0; w < W; ++w) {
+                    for (int w = 0; w < W * G; ++w) {           // warps, then lane groups: a fixed order
                         const float* zw = zs_all + w * S.zs_stride;
 #pragma unroll
                         for (int g = 0; g < 4; ++g) z[g] += zw[(g * U + u) * BT + bt];
@@ -262,7 +266,7 @@ struct RnnPlan {
     int gates = 0, L = 0, B = 0, H = 0, device = 0, val_dtype = 0;
     std::vector<uint64_t> uids;
     int in_size[kMaxLayers] = {};
-    int n_ctas = 0, warps = 0, BT = 1, resident = 0, stages = 0, stage_bytes = 0, max_warp_bytes = 0, max_U = 0, max_C = 0;
+    int n_ctas = 0, warps = 0, BT = 1, GW = 32, resident = 0, stages = 0, stage_bytes = 0, max_warp_bytes = 0, max_U = 0, max_C = 0;
     size_t smem = 0;
     double balance = 1.0;
     int64_t stream_bytes = 0;
@@ -332,9 +336,10 @@ static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, i
         rc = plan_rnn_host(gates, L, W, in_size, H, want, wtry, P->stage_bytes, &Hp);
         if (rc != CSB_OK) return rc;
         P->warps = wtry;
-        P->max_U = Hp.max_U; P->max_warp_bytes = (int)Hp.max_warp_bytes;
-        const RnnSmem res(wtry, P->stages, P->stage_bytes, 1, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
-        const RnnSmem str(wtry, P->stages, P->stage_bytes, 0, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
+        P->max_U = Hp.max_U; P->max_warp_bytes = (int)Hp.max_warp_bytes; P->GW = Hp.stream.group_width;
+        const int G = 32 / P->GW;
+        const RnnSmem res(wtry, G, P->stages, P->stage_bytes, 1, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
+        const RnnSmem str(wtry, G, P->stages, P->stage_bytes, 0, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
         if (res.total <= A0->smem_optin && !env_int("CSB_RNN_STREAM", 0)) { P->resident = 1; P->smem = res.total; fits = true; break; }
         if (str.total <= A0->smem_optin) { P->resident = 0; P->smem = str.total; fits = true; break; }
     }
@@ -355,11 +360,11 @@ static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, i
     return CSB_OK;
 }
 
-template <typename T, int BT>
+template <typename T, int BT, int GW>
 static int launch_rnn(const RnnPlan* P, RnnArgs& a, cudaStream_t st) {
-    CSB_CUDA(cudaFuncSetAttribute(csb_rnn_kernel<T, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem));
+    CSB_CUDA(cudaFuncSetAttribute(csb_rnn_kernel<T, BT, GW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem));
     int occ = 0;
-    CSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, csb_rnn_kernel<T, BT>, P->warps * 32, P->smem));
+    CSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, csb_rnn_kernel<T, BT, GW>, P->warps * 32, P->smem));
     int sms = 0;
     CSB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, P->device));
     if (occ < 1 || P->n_ctas > occ * sms) {
@@ -367,11 +372,20 @@ static int launch_rnn(const RnnPlan* P, RnnArgs& a, cudaStream_t st) {
         return CSB_ERR_LAUNCH;
     }
     void* params[] = {(void*)&a};
-    const cudaError_t e = cudaLaunchCooperativeKernel((const void*)csb_rnn_kernel<T, BT>, dim3(P->n_ctas), dim3(P->warps * 32),
+    const cudaError_t e = cudaLaunchCooperativeKernel((const void*)csb_rnn_kernel<T, BT, GW>, dim3(P->n_ctas), dim3(P->warps * 32),
                                                       params, P->smem, st);
     if (e == cudaErrorCooperativeLaunchTooLarge) { set_error("cooperative launch too large"); return CSB_ERR_LAUNCH; }
     CSB_CUDA(e);
     return CSB_OK;
+}
+
+template <typename T, int BT>
+static int dispatch_rnn_gw(const RnnPlan* P, RnnArgs& a, cudaStream_t st) {
+    switch (P->GW) {
+        case 8: return launch_rnn<T, BT, 8>(P, a, st);
+        case 16: return launch_rnn<T, BT, 16>(P, a, st);
+        default: return launch_rnn<T, BT, 32>(P, a, st);
+    }
 }
 
 static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const float* const* bias, const float* x, int64_t T,
@@ -463,9 +477,9 @@ static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const flo
     a.resident = P->resident; a.max_warp_bytes = P->max_warp_bytes; a.max_U = P->max_U; a.max_C = P->max_C;
     int rc;
     const bool half = P->val_dtype == CSB_F16;
-    if (P->BT == 1) rc = half ? launch_rnn<__half, 1>(P, a, st) : launch_rnn<float, 1>(P, a, st);
-    else if (P->BT == 4) rc = half ? launch_rnn<__half, 4>(P, a, st) : launch_rnn<float, 4>(P, a, st);
-    else rc = half ? launch_rnn<__half, 8>(P, a, st) : launch_rnn<float, 8>(P, a, st);
+    if (P->BT == 1) rc = half ? dispatch_rnn_gw<__half, 1>(P, a, st) : dispatch_rnn_gw<float, 1>(P, a, st);
+    else if (P->BT == 4) rc = half ? dispatch_rnn_gw<__half, 4>(P, a, st) : dispatch_rnn_gw<float, 4>(P, a, st);
+    else rc = half ? dispatch_rnn_gw<__half, 8>(P, a, st) : dispatch_rnn_gw<float, 8>(P, a, st);
     if (rc != CSB_OK) return rc;
     const int last_slot = (int)((T - 1) & 1);
     if (hT) CSB_CUDA(cudaMemcpy2DAsync(hT, row, P->d_hbuf + (size_t)last_slot * B * H, 2 * row, row, L, out_kind, st));

@@ -1,0 +1,217 @@
+// Block -> warp schedules for the two kernels (host side, run once per matrix / stack).
+#include <algorithm>
+#include <cstdlib>
+
+#include "csb_internal.hpp"
+
+namespace csb {
+
+static int env_gw() {
+    const char* v = getenv("CSB_GROUP_WIDTH");
+    const int g = v && *v ? atoi(v) : 0;
+    return (g == 8 || g == 16 || g == 32) ? g : 0;
+}
+
+// Schedule for the bare product: walk the blocks in row-major order, give every warp of
+// the persistent grid one contiguous, equal-cost run of items, and mark the end of each
+// block-row inside a warp with how its accumulators leave the warp: straight to y when the
+// warp owns the whole block-row, else as a partial sum in its own slot.
+int plan_product_host(const csb_matrix* A, int n_warps, int stage_bytes, ProductHostPlan* out) {
+    const int rpw = rows_per_word(A->val_dtype);
+    std::vector<int> rl;
+    rl.reserve(A->nblk);
+    for (int64_t b = 0; b < A->nblk; ++b)
+        if (A->m[b] && A->n[b]) rl.push_back((A->m[b] + rpw - 1) / rpw);
+    const int gw = env_gw() ? env_gw() : pick_group_width(rl);
+    out->stream.group_width = gw;
+    const int value_budget = item_value_budget(stage_bytes, gw);
+    std::vector<ItemSpec> items;
+    std::vector<int64_t> item_row;                      // block-row of each item; -1 items are placeholders
+    std::vector<char> placeholder;
+    for (int64_t bi = 0; bi < A->nbr; ++bi) {
+        const size_t before = items.size();
+        for (int64_t bj = 0; bj < A->nbc; ++bj) {
+            const int64_t b = bi * A->nbc + bj;
+            ItemSpec proto{};
+            proto.xbase = (uint32_t)(bj * A->block_c);
+            slice_block(A, b, 0, A->m[b], 0, A->n[b], gw * rpw, value_budget, proto, &items);
+        }
+        const bool empty = items.size() == before;
+        if (empty) items.push_back(ItemSpec{});         // nothing kept: the block-row still owes zeros to y
+        item_row.resize(items.size(), bi);
+        placeholder.resize(items.size(), empty ? 1 : 0);
+    }
+    std::vector<double> cost(items.size());
+    double total = 0;
+    for (size_t i = 0; i < items.size(); ++i) { cost[i] = placeholder[i] ? 4.0 : (double)item_steps(A, items[i], gw); total += cost[i]; }
+    std::vector<std::vector<Segment>> per_warp(n_warps);
+    const double target = total / n_warps;
+    double cum = 0;
+    for (size_t i = 0; i < items.size(); ++i) {
+        int w = (int)((cum + 0.5 * cost[i]) / target);
+        w = std::min(std::max(w, 0), n_warps - 1);
+        std::vector<Segment>& segs = per_warp[w];
+        const uint32_t zb = (uint32_t)(item_row[i] * A->block_r);
+        if (segs.empty() || segs.back().zbase != zb) { segs.emplace_back(); segs.back().zbase = zb; }
+        if (!placeholder[i]) segs.back().items.push_back(items[i]);
+        cum += cost[i];
+    }
+    // contributors per block-row, in warp order
+    out->part_base.assign(A->nbr, 0);
+    out->part_count.assign(A->nbr, 0);
+    std::vector<uint32_t> contributors(A->nbr, 0);
+    for (auto& segs : per_warp)
+        for (auto& sg : segs) contributors[sg.zbase / A->block_r]++;
+    uint32_t slots = 0;
+    for (int64_t bi = 0; bi < A->nbr; ++bi)
+        if (contributors[bi] > 1) { out->part_base[bi] = slots; out->part_count[bi] = contributors[bi]; slots += contributors[bi]; }
+    out->n_slots = slots;
+    std::vector<uint32_t> next_slot(out->part_base);
+    for (auto& segs : per_warp)
+        for (auto& sg : segs) {
+            const int64_t bi = sg.zbase / A->block_r;
+            sg.tail = contributors[bi] > 1 ? (kFlushPartial | (next_slot[bi]++ << kSlotShift)) : (uint32_t)kFlushDirect;
+        }
+    build_stream(A, per_warp, stage_bytes, &out->stream);
+    double mx = 0, sum = 0;
+    for (double c : out->stream.warp_cost) { mx = std::max(mx, c); sum += c; }
+    out->balance = mx > 0 ? sum / n_warps / mx : 1.0;
+    return CSB_OK;
+}
+
+// Schedule for the recurrent time loop.  Every CTA owns a tile of hidden units of one layer
+// together with ALL gate rows of those units (rows u, H+u, 2H+u, ...), so the gate arithmetic
+// needs no data from other CTAs and one grid-wide barrier per step is enough.  CTAs are shared
+// out between the layers in proportion to their stored weights (the layers run as a
+// wavefront: layer l works on step t while layer l+1 works on step t-1); unit tiles and the
+// warps inside a CTA are cut by cost, not by count.
+int plan_rnn_host(int gates, int n_layers, const csb_matrix* const* Wm, const int* in_size, int H, int n_ctas,
+                  int warps, int stage_bytes, RnnHostPlan* out) {
+    out->warps = warps;
+    out->max_U = 0;
+    // every layer gets enough CTAs for its tiles to stay under the unit limit; the rest are
+    // shared out by stored weights
+    const int floor_ctas = std::min(H, (H + 47) / 48);
+    std::vector<int> ncta(n_layers, floor_ctas);
+    {
+        if (floor_ctas * n_layers > n_ctas) {
+            set_error("%d layers of hidden size %d need %d CTAs, %d available", n_layers, H, floor_ctas * n_layers, n_ctas);
+            return CSB_ERR_UNSUPPORTED;
+        }
+        double tot = 0;
+        for (int l = 0; l < n_layers; ++l) tot += (double)Wm[l]->nnz + 1.0;
+        const int spare = n_ctas - floor_ctas * n_layers;
+        for (int l = 0; l < n_layers; ++l)
+            ncta[l] = std::min(H, floor_ctas + (int)((double)spare * ((double)Wm[l]->nnz + 1.0) / tot));
+    }
+    // unit tiles per layer: contiguous, about equal stored weights
+    std::vector<std::vector<int>> cuts(n_layers);
+    for (int l = 0; l < n_layers; ++l) {
+        const csb_matrix* A = Wm[l];
+        std::vector<double> rowcost(A->rows, 0.0);
+        for (int64_t b = 0; b < A->nblk; ++b) {
+            const int64_t bi = b / A->nbc;
+            const uint8_t* ri = A->row_idx.data() + A->ridx_off[b];
+            for (int r = 0; r < A->m[b]; ++r) rowcost[bi * A->block_r + ri[r]] += A->n[b] + 2.0;
+        }
+        std::vector<double> ucost(H, 8.0);
+        for (int g = 0; g < gates; ++g)
+            for (int u = 0; u < H; ++u) ucost[u] += rowcost[(int64_t)g * H + u];
+        double tot = 0;
+        for (double c : ucost) tot += c;
+        std::vector<int>& cut = cuts[l];
+        cut.assign(ncta[l] + 1, H);
+        cut[0] = 0;
+        double cum = 0;
+        int t = 1;
+        for (int u = 0; u < H && t < ncta[l]; ++u) {
+            cum += ucost[u];
+            const int left_units = H - (u + 1), left_tiles = ncta[l] - t;
+            const bool full = u + 1 - cut[t - 1] >= kMaxTileUnits;
+            if (cum >= tot * t / ncta[l] || left_units <= left_tiles || full) cut[t++] = u + 1;
+        }
+        for (int c = 0; c < ncta[l]; ++c) {
+            const int U = cut[c + 1] - cut[c];
+            if (U > kMaxTileUnits) {
+                set_error("hidden size %d over %d CTAs gives tiles of %d units (limit %d)", H, ncta[l], U, (int)kMaxTileUnits);
+                return CSB_ERR_UNSUPPORTED;
+            }
+            out->max_U = std::max(out->max_U, U);
+        }
+    }
+    // items of one CTA (layer l, units [u0, u1)) for a given lane-group width
+    auto tile_items = [&](int l, int u0, int u1, int gw, std::vector<ItemSpec>* items, std::vector<int>* rl) {
+        const csb_matrix* A = Wm[l];
+        const int I = in_size[l], U = u1 - u0, rpw = rows_per_word(A->val_dtype);
+        const int max_rows = gw * rpw, value_budget = item_value_budget(stage_bytes, gw);
+        for (int g = 0; g < gates; ++g) {
+            const int64_t row0 = (int64_t)g * H + u0, row1 = (int64_t)g * H + u1;
+            for (int64_t bi = row0 / A->block_r; bi <= (row1 - 1) / A->block_r; ++bi) {
+                const int lo = (int)std::max<int64_t>(0, row0 - bi * A->block_r);
+                const int hi = (int)std::min<int64_t>(A->block_r, row1 - bi * A->block_r);
+                for (int64_t bj = 0; bj < A->nbc; ++bj) {
+                    const int64_t b = bi * A->nbc + bj;
+                    const uint8_t* ri = A->row_idx.data() + A->ridx_off[b];
+                    const uint8_t* ci = A->col_idx.data() + A->cidx_off[b];
+                    const int m = A->m[b], n = A->n[b];
+                    const int r0 = (int)(std::lower_bound(ri, ri + m, lo) - ri);
+                    const int r1 = (int)(std::lower_bound(ri, ri + m, hi) - ri);
+                    if (rl) { if (r1 > r0 && n) rl->push_back((r1 - r0 + rpw - 1) / rpw); continue; }
+                    const int64_t split_col = (int64_t)I - bj * A->block_c;      // first recurrent column, block-local
+                    const int ks = split_col <= 0 ? 0 : split_col >= A->block_c ? n
+                                   : (int)(std::lower_bound(ci, ci + n, (int)split_col) - ci);
+                    ItemSpec proto{};
+                    proto.ridx_bias = (int)(row0 - bi * A->block_r);
+                    proto.xbase = (uint32_t)(bj * A->block_c);
+                    proto.zbase = (uint32_t)(g * U);
+                    slice_block(A, b, r0, r1, 0, ks, max_rows, value_budget, proto, items);
+                    proto.xbase = (uint32_t)(bj * A->block_c - I);                 // may wrap; col_idx brings it back
+                    proto.flags = kItemRecurrent;
+                    if (gates == 3 && g == 2) proto.zbase = (uint32_t)(3 * U);     // GRU candidate gate, hidden part
+                    slice_block(A, b, r0, r1, ks, n, max_rows, value_budget, proto, items);
+                }
+            }
+        }
+    };
+    // lane-group width from the row counts the tiles actually see
+    std::vector<int> rl;
+    for (int l = 0; l < n_layers; ++l)
+        for (int c = 0; c < ncta[l]; c += std::max(1, ncta[l] / 8)) tile_items(l, cuts[l][c], cuts[l][c + 1], 32, nullptr, &rl);
+    const int gw = env_gw() ? env_gw() : pick_group_width(rl);
+    out->stream.group_width = gw;
+    double cost_sum = 0, cost_max = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const csb_matrix* A = Wm[l];
+        for (int c = 0; c < ncta[l]; ++c) {
+            const int u0 = cuts[l][c], u1 = cuts[l][c + 1];
+            std::vector<ItemSpec> items;
+            tile_items(l, u0, u1, gw, &items, nullptr);
+            // warps of this CTA: contiguous runs of about equal cost
+            std::vector<std::vector<Segment>> per_warp(warps, std::vector<Segment>(1));
+            double total = 0;
+            std::vector<double> cost(items.size());
+            for (size_t i = 0; i < items.size(); ++i) { cost[i] = (double)item_steps(A, items[i], gw); total += cost[i]; }
+            double cum = 0;
+            for (size_t i = 0; i < items.size(); ++i) {
+                const int w = total > 0 ? (int)((cum + 0.5 * cost[i]) / (total / warps)) : 0;
+                per_warp[std::min(std::max(w, 0), warps - 1)][0].items.push_back(items[i]);
+                cum += cost[i];
+            }
+            RnnCtaDesc d{l, u0, u1 - u0, (uint32_t)out->stream.n_warps};
+            build_stream(A, per_warp, stage_bytes, &out->stream);
+            out->ctas.push_back(d);
+            cost_sum += total;
+            cost_max = std::max(cost_max, total);
+        }
+    }
+    out->max_warp_bytes = 0;
+    for (int w = 0; w < out->stream.n_warps; ++w) {
+        size_t bytes = 0;
+        for (uint32_t c = out->stream.warp_chunk_begin[w]; c < out->stream.warp_chunk_begin[w + 1]; ++c) bytes += out->stream.chunks[c].bytes;
+        out->max_warp_bytes = std::max(out->max_warp_bytes, bytes);
+    }
+    out->balance = cost_max > 0 ? cost_sum / out->ctas.size() / cost_max : 1.0;
+    return CSB_OK;
+}
+
+}  // namespace csb
