@@ -67,6 +67,17 @@ template <> struct WordTraits<float> {
     __device__ static __forceinline__ void unpack(uint32_t w, float (&v)[1]) { v[0] = __uint_as_float(w); }
 };
 
+// Per-group buffers are spaced so that the lane groups of a warp, which run in lock-step and
+// tend to touch the same index at the same time, fall into different shared-memory banks.
+__host__ __device__ constexpr int group_pad(int gw) { return gw == 32 ? 0 : gw; }
+__host__ __device__ constexpr int xg_stride(int gw, int bt) { return kMaxNk * bt + group_pad(gw); }
+
+#ifdef CSB_PHASE_CLOCKS
+// instrumented build only: per-thread lap counters of walk_chunk (header, gather, multiply, fold, scatter, rounds)
+static __device__ long long csb_walk_prof_dummy;
+#define csb_walk_prof csb_walk_prof_local
+#endif
+
 template <int N> struct Log2;
 template <> struct Log2<8> { static constexpr int v = 3; };
 template <> struct Log2<16> { static constexpr int v = 4; };
@@ -86,13 +97,17 @@ __device__ __forceinline__ uint32_t chunk_bytes(const uint4& ch) {
 // sub-group owns word rl of each column, i.e. the same output rows for the whole item.  The
 // A = S * RL active lanes read words s*A .. s*A + A-1 in step s: consecutive, conflict-free.
 //
-// Per item: gather the kept inputs through the column indices (gather(col, flags, bt) returns
-// input `col` of batch column bt) into xg, multiply, fold the sub-groups, and add into
+// Per item: gather the kept inputs through the column indices (gather4(xbase, c4, flags, left,
+// dst) resolves four packed indices, `left` of them real, and writes dst[j * BT + bt]) into xg, multiply, fold the sub-groups, and add into
 // zs[(zbase + row_idx) * BT + bt] of this group's private accumulators.
-//   xg_w: per warp, G * kMaxNk * BT floats;  zs_w: per warp, G * zs_stride floats.
+//   xg_w: per warp, G * xg_stride(GW, BT) floats;  zs_w: per warp, G * zs_stride floats.
 template <typename T, int BT, int GW, typename Gather>
 __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch, int lane, float* __restrict__ xg_w,
-                                           float* __restrict__ zs_w, int zs_stride, Gather gather) {
+                                           float* __restrict__ zs_w, int zs_stride, Gather gather4
+#ifdef CSB_PHASE_CLOCKS
+                                           , long long* csb_walk_prof_local = &csb_walk_prof_dummy
+#endif
+                                           ) {
     constexpr int R = WordTraits<T>::kRows;
     const int g = lane / GW, gl = lane % GW;
     const uint32_t sz[4] = {ch.x & 0xffffu, ch.x >> 16, ch.y & 0xffffu, ch.y >> 16};
@@ -104,29 +119,36 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
     }
     const uint8_t* p = chunk + 16 + 16 * before;
     const uint8_t* end = p + 16 * mine;
-    float* xg = xg_w + g * (kMaxNk * BT);
+    float* xg = xg_w + g * xg_stride(GW, BT);
     float* zs = zs_w + g * zs_stride;
+#ifdef CSB_PHASE_CLOCKS
+    long long tq = clock64();
+#define CSB_WALK_LAP(i) do { const long long n_ = clock64(); csb_walk_prof[i] += n_ - tq; tq = n_; } while (0)
+#else
+#define CSB_WALK_LAP(i) do { } while (0)
+#endif
     while (__any_sync(0xffffffffu, p < end)) {
-        int nk = 0, mr = 0, RL = 1, S = 1;
-        uint32_t xbase = 0, zbase = 0, magic = 1024, flags = 0;
-        if (p < end) {
-            const uint4 h = *reinterpret_cast<const uint4*>(p);
-            nk = (int)(h.x & 0xffu); mr = (int)((h.x >> 8) & 0xffu); RL = (int)((h.x >> 16) & 0xffu); S = (int)(h.x >> 24);
-            xbase = h.y; zbase = h.z; magic = h.w & 0xffffu; flags = h.w >> 16;
-        }
+        // ---- header: a finished group reads zeros, which turns every step below into a no-op
+        uint4 h = make_uint4(0u, 0u, 0u, 0u);
+        if (p < end) h = *reinterpret_cast<const uint4*>(p);
+        const int nk = (int)(h.x & 0xffu), mr = (int)((h.x >> 8) & 0xffu), RL = (int)((h.x >> 16) & 0xffu), S = (int)(h.x >> 24);
+        const uint32_t xbase = h.y, zbase = h.z, magic = h.w & 0xffffu, flags = h.w >> 16;
         const uint8_t* cidx = p + 16;
-        const uint8_t* ridx = cidx + nk;
-        const int idx_bytes = (nk + mr + 3) & ~3;
-        const uint32_t* vals = reinterpret_cast<const uint32_t*>(p + 16 + idx_bytes);
+        const int cidx_bytes = (nk + 3) & ~3, ridx_bytes = (mr + 3) & ~3;
+        const uint8_t* ridx = cidx + cidx_bytes;
+        const uint32_t* vals = reinterpret_cast<const uint32_t*>(ridx + ridx_bytes);
         const int nwords = nk * RL;
-        if (p < end) p += (16 + idx_bytes + nwords * 4 + 15) & ~15;
+        if (p < end) p += (16 + cidx_bytes + ridx_bytes + nwords * 4 + 15) & ~15;     // items are 16-byte aligned
+        CSB_WALK_LAP(0);
 
-        for (int k = gl; k < nk; k += GW) {
-            const uint32_t col = xbase + cidx[k];
-#pragma unroll
-            for (int bt = 0; bt < BT; ++bt) xg[k * BT + bt] = gather(col, flags, bt);
-        }
+        // ---- gather: each lane resolves four column indices at a time; indices past nk are
+        // padding zeros, gather4 decides whether they may be dereferenced
+        for (int k4 = gl * 4; k4 < nk; k4 += 4 * GW)
+            gather4(xbase, *reinterpret_cast<const uint32_t*>(cidx + k4), flags, nk - k4, xg + k4 * BT);
         __syncwarp();
+        CSB_WALK_LAP(1);
+
+        // ---- multiply: lane gl reads words gl, gl + A, ... and walks columns kg, kg + S, ...
         const int kg = (int)(((uint32_t)gl * magic) >> 10);
         const int A = S * RL;
         float acc[R][BT];
@@ -135,22 +157,43 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
 #pragma unroll
             for (int bt = 0; bt < BT; ++bt) acc[q][bt] = 0.f;
         if (gl < A) {
-            int k = kg;
-#pragma unroll 4
-            for (int w = gl; w < nwords; w += A, k += S) {
+            const uint32_t* vp = vals + gl;
+            const uint32_t* vend = vals + nwords;
+            const float* xp = xg + kg * BT;
+            const int xs = S * BT;
+            for (; vp + 3 * A < vend; vp += 4 * A, xp += 4 * xs) {
+                uint32_t w[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) w[j] = vp[j * A];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float v[R];
+                    WordTraits<T>::unpack(w[j], v);
+#pragma unroll
+                    for (int bt = 0; bt < BT; ++bt) {
+                        const float xv = xp[j * xs + bt];
+#pragma unroll
+                        for (int q = 0; q < R; ++q) acc[q][bt] = fmaf(v[q], xv, acc[q][bt]);
+                    }
+                }
+            }
+            for (; vp < vend; vp += A, xp += xs) {
                 float v[R];
-                WordTraits<T>::unpack(vals[w], v);
+                WordTraits<T>::unpack(*vp, v);
 #pragma unroll
                 for (int bt = 0; bt < BT; ++bt) {
-                    const float xv = xg[k * BT + bt];
+                    const float xv = xp[bt];
 #pragma unroll
                     for (int q = 0; q < R; ++q) acc[q][bt] = fmaf(v[q], xv, acc[q][bt]);
                 }
             }
         }
-        // fold the sub-groups onto sub-group 0: a tree over kg (S need not be a power of two)
-#pragma unroll
-        for (int r = 0; r < Log2<GW>::v; ++r) {
+        CSB_WALK_LAP(2);
+
+        // ---- fold the sub-groups onto sub-group 0: a tree over kg (S need not be a power of
+        // two); the number of rounds is the same for the whole warp
+        const int smax = (int)__reduce_max_sync(0xffffffffu, (unsigned)S);
+        for (int r = 0; (1 << r) < smax; ++r) {
             const int off = RL << r;
             const bool take = off < A && gl + off < A;
 #pragma unroll
@@ -161,18 +204,32 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
                     if (take) acc[q][bt] += o;
                 }
         }
+        CSB_WALK_LAP(3);
+
+        // ---- scatter-add through the row indices (distinct within an item: loads first, stores last)
         if (gl < RL) {
+            const int r0 = gl * R;
+            float* zr[R];
+            float cur[R][BT];
 #pragma unroll
             for (int q = 0; q < R; ++q) {
-                const int r = gl * R + q;
-                if (r < mr) {
-                    float* z = zs + ((int)zbase + (int)ridx[r]) * BT;
+                const int ri = (r0 + q < mr) ? (int)ridx[r0 + q] : (int)ridx[r0];
+                zr[q] = zs + ((int)zbase + ri) * BT;
 #pragma unroll
-                    for (int bt = 0; bt < BT; ++bt) z[bt] += acc[q][bt];
-                }
+                for (int bt = 0; bt < BT; ++bt) cur[q][bt] = zr[q][bt];
             }
+#pragma unroll
+            for (int q = 0; q < R; ++q)
+                if (r0 + q < mr) {
+#pragma unroll
+                    for (int bt = 0; bt < BT; ++bt) zr[q][bt] = cur[q][bt] + acc[q][bt];
+                }
         }
         __syncwarp();
+        CSB_WALK_LAP(4);
+#ifdef CSB_PHASE_CLOCKS
+        csb_walk_prof[5] += 1;
+#endif
     }
 }
 

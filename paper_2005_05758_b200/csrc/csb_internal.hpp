@@ -25,8 +25,8 @@ void clear_error();
 //   chunk  = ChunkHeader (16 B), then the G sub-streams back to back
 //   sub-stream g = the items of lane group g, each aligned to 16 B
 //   item   = ItemHeader (16 B)
-//            col_idx[nk]  uint8   gather indices, relative to xbase
-//            row_idx[mr]  uint8   scatter indices, relative to zbase   (padded to 4 B)
+//            col_idx[nk]  uint8   gather indices, relative to xbase     (padded to 4 B)
+//            row_idx[mr]  uint8   scatter indices, relative to zbase    (padded to 4 B)
 //            values       nk columns of RL "row words" each, column-major:
 //                           f16: a word is two consecutive kept rows (half2), RL = ceil(mr/2)
 //                           f32: a word is one kept row, RL = mr
@@ -81,7 +81,7 @@ struct ProductPlan {
     size_t smem_bytes = 0;
     uint8_t* d_stream = nullptr;
     Chunk* d_chunks = nullptr;
-    uint32_t* d_warp_chunk_begin = nullptr;
+    void* d_warp_desc = nullptr;           // uint4 per warp: first chunk, end chunk, first chunk's off16 and bytes
     // partial block-row sums: slots [part_base[bi], part_base[bi] + part_count[bi]) belong to block-row bi
     uint32_t* d_part_base = nullptr;
     uint32_t* d_part_count = nullptr;

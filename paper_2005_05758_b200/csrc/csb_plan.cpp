@@ -24,7 +24,7 @@ static inline int row_words(const csb_matrix* A, int mr) {
 
 size_t item_bytes(const csb_matrix* A, const ItemSpec& it) {
     const int nk = it.k1 - it.k0, mr = it.r1 - it.r0;
-    return pad_to(sizeof(ItemHeader) + pad_to((size_t)nk + mr, 4) + (size_t)nk * row_words(A, mr) * 4, kItemAlign);
+    return pad_to(sizeof(ItemHeader) + pad_to((size_t)nk, 4) + pad_to((size_t)mr, 4) + (size_t)nk * row_words(A, mr) * 4, kItemAlign);
 }
 
 // Lock-step cost of an item for a lane group of width gw: column steps plus a fixed part
@@ -50,8 +50,9 @@ void emit_item(const csb_matrix* A, const ItemSpec& it, int gw, std::vector<uint
     const uint8_t* ci = A->col_idx.data() + A->cidx_off[it.block];
     const uint8_t* ri = A->row_idx.data() + A->ridx_off[it.block];
     for (int k = 0; k < nk; ++k) p[k] = ci[it.k0 + k];
-    for (int r = 0; r < mr; ++r) p[nk + r] = (uint8_t)(ri[it.r0 + r] - it.ridx_bias);
-    p += pad_to((size_t)nk + mr, 4);
+    p += pad_to((size_t)nk, 4);
+    for (int r = 0; r < mr; ++r) p[r] = (uint8_t)(ri[it.r0 + r] - it.ridx_bias);
+    p += pad_to((size_t)mr, 4);
     const int n = A->n[it.block];
     const uint8_t* v = A->val.data() + A->val_off[it.block] * vs;
     for (int k = 0; k < nk; ++k)

@@ -17,7 +17,7 @@ namespace csb {
 struct ProductArgs {
     const uint8_t* stream;
     const Chunk* chunks;
-    const uint32_t* warp_chunk_begin;
+    const uint4* warp_desc;    // per warp: first chunk, end chunk, first chunk's off16 and bytes
     const uint32_t* part_base;
     const uint32_t* part_count;
     uint32_t* arrivals;
@@ -27,7 +27,20 @@ struct ProductArgs {
     long long ldx, ldy;
     uint32_t* status;
     int n_warps, nb, rows, cols, block_r, stage_bytes, stages, x_in_smem;
+#ifdef CSB_PHASE_CLOCKS
+    long long* clocks;         // [n_warps][6] cycle stamps: start, staged, first chunk, walked, flushed, end
+#endif
 };
+
+#ifdef CSB_PHASE_CLOCKS
+#define CSB_STAMP(i) do { if (lane == 0 && gw < a.n_warps) a.clocks[(size_t)gw * 6 + (i)] = clock64(); } while (0)
+#define CSB_ADD(i, v) do { if (lane == 0 && gw < a.n_warps) a.clocks[(size_t)gw * 6 + (i)] += (v); } while (0)
+#else
+#define CSB_STAMP(i) do { } while (0)
+#define CSB_ADD(i, v) do { } while (0)
+#endif
+
+constexpr int kXRegs = 4;      // float4 registers per thread used to stage x (covers 8192 columns at 512 threads)
 
 __host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t)15; }
 
@@ -36,12 +49,12 @@ struct ProductSmem {
     size_t ring, bars, zs, xg, xs, total;
     int zs_stride;                                     // floats per lane group
     __host__ __device__ ProductSmem(int W, int G, int stages, int stage_bytes, int block_r, int BT, int cols_in_smem) {
-        zs_stride = block_r * BT;
+        zs_stride = block_r * BT + group_pad(32 / G);
         ring = 0;
         bars = ring + (size_t)W * stages * stage_bytes;
         zs = align16(bars + (size_t)W * stages * 8);
         xg = align16(zs + (size_t)W * G * zs_stride * 4);
-        xs = align16(xg + (size_t)W * G * kMaxNk * BT * 4);
+        xs = align16(xg + (size_t)W * G * xg_stride(32 / G, BT) * 4);
         total = align16(xs + (size_t)cols_in_smem * 4);
     }
 };
@@ -105,17 +118,38 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
     uint8_t* ring = smem + L.ring + (size_t)warp * a.stages * a.stage_bytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.bars) + warp * a.stages;
     float* zs = reinterpret_cast<float*>(smem + L.zs) + warp * G * L.zs_stride;
-    float* xg = reinterpret_cast<float*>(smem + L.xg) + warp * G * kMaxNk * BT;
+    float* xg = reinterpret_cast<float*>(smem + L.xg) + warp * G * xg_stride(GW, BT);
     const float* xs = reinterpret_cast<const float*>(smem + L.xs);
 
     const int gw = blockIdx.x * W + warp;
-    uint32_t c0 = 0, c1 = 0;
-    if (gw < a.n_warps) { c0 = a.warp_chunk_begin[gw]; c1 = a.warp_chunk_begin[gw + 1]; }
-
+    CSB_STAMP(0);
+#ifdef CSB_PHASE_CLOCKS
+    if (lane == 0 && gw < a.n_warps) { a.clocks[(size_t)gw * 6 + 2] = 0; a.clocks[(size_t)gw * 6 + 3] = 0; a.clocks[(size_t)gw * 6 + 4] = 0; }
+#endif
+    // One 16-byte descriptor per warp (first chunk index, end chunk index, first chunk's place
+    // and size) starts the pipeline with a single round trip; the loads of x are issued before
+    // anything waits on it.
+    uint4 wd = make_uint4(0u, 0u, 0u, 0u);
+    if (gw < a.n_warps) wd = __ldg(a.warp_desc + gw);
+    const uint32_t c0 = wd.x, c1 = wd.y;
+    float4 xr[kXRegs];
+    const bool x_vec = a.x_in_smem && (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && a.cols <= (int)blockDim.x * 4 * kXRegs;
+    if (x_vec) {
+        const float4* x4 = reinterpret_cast<const float4*>(a.X);
+#pragma unroll
+        for (int j = 0; j < kXRegs; ++j) {
+            const int i = threadIdx.x + j * blockDim.x;
+            xr[j] = i < a.cols / 4 ? __ldg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
     if (lane == 0) {
         for (int s = 0; s < a.stages; ++s) mbar_init(&bars[s], 1);
         mbar_fence_init();
-        for (int s = 0; s < a.stages && c0 + s < c1; ++s) {
+        if (c0 < c1) {
+            mbar_expect_tx(&bars[0], wd.w);
+            bulk_g2s(ring, a.stream + (size_t)wd.z * 16, wd.w, &bars[0]);
+        }
+        for (int s = 1; s < a.stages && c0 + s < c1; ++s) {
             const Chunk ch = a.chunks[c0 + s];
             mbar_expect_tx(&bars[s], ch.bytes);
             bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)ch.off16 * 16, ch.bytes, &bars[s]);
@@ -124,9 +158,12 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
     for (int i = lane; i < G * L.zs_stride; i += 32) zs[i] = 0.f;
     if (a.x_in_smem) {
         float* xw = reinterpret_cast<float*>(smem + L.xs);
-        if ((reinterpret_cast<uintptr_t>(a.X) & 15) == 0) {
-            const float4* x4 = reinterpret_cast<const float4*>(a.X);
-            for (int i = threadIdx.x; i < a.cols / 4; i += blockDim.x) reinterpret_cast<float4*>(xw)[i] = __ldg(x4 + i);
+        if (x_vec) {
+#pragma unroll
+            for (int j = 0; j < kXRegs; ++j) {
+                const int i = threadIdx.x + j * blockDim.x;
+                if (i < a.cols / 4) reinterpret_cast<float4*>(xw)[i] = xr[j];
+            }
             for (int i = (a.cols & ~3) + threadIdx.x; i < a.cols; i += blockDim.x) xw[i] = __ldg(a.X + i);
         } else {
             for (int i = threadIdx.x; i < a.cols; i += blockDim.x) xw[i] = __ldg(a.X + i);
@@ -136,7 +173,14 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
         __syncwarp();
     }
 
+    CSB_STAMP(1);
+#ifdef CSB_PHASE_CLOCKS
+    long long wprof[6] = {0, 0, 0, 0, 0, 0};
+#endif
     for (uint32_t c = c0; c < c1; ++c) {
+#ifdef CSB_PHASE_CLOCKS
+        const long long tc0 = clock64();
+#endif
         const int s = (int)((c - c0) % (uint32_t)a.stages);
         const uint32_t parity = ((c - c0) / (uint32_t)a.stages) & 1u;
         const Chunk refill = (c + a.stages < c1) ? a.chunks[c + a.stages] : Chunk{0, 0};
@@ -151,21 +195,58 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
             }
             break;
         }
+#ifdef CSB_PHASE_CLOCKS
+        const long long tc1 = clock64();
+        CSB_ADD(2, tc1 - tc0);
+#endif
         const uint8_t* p = ring + (size_t)s * a.stage_bytes;
         const uint4 ch = *reinterpret_cast<const uint4*>(p);
-        walk_chunk<T, BT, GW>(p, ch, lane, xg, zs, L.zs_stride, [&](uint32_t col, uint32_t, int bt) -> float {
-            if (BT == 1) return a.x_in_smem ? xs[col] : __ldg(a.X + col);
-            return bt < a.nb ? __ldg(a.X + (long long)bt * a.ldx + col) : 0.f;
-        });
+        walk_chunk<T, BT, GW>(p, ch, lane, xg, zs, L.zs_stride,
+                              [&](uint32_t xbase, uint32_t c4, uint32_t, int left, float* dst) {
+            if (BT == 1) {
+                // index 0 of the block is always a valid column, so padding indices may be read
+                float4 v;
+                if (a.x_in_smem) {
+                    v.x = xs[xbase + (c4 & 0xffu)]; v.y = xs[xbase + ((c4 >> 8) & 0xffu)];
+                    v.z = xs[xbase + ((c4 >> 16) & 0xffu)]; v.w = xs[xbase + (c4 >> 24)];
+                } else {
+                    v.x = __ldg(a.X + xbase + (c4 & 0xffu)); v.y = __ldg(a.X + xbase + ((c4 >> 8) & 0xffu));
+                    v.z = __ldg(a.X + xbase + ((c4 >> 16) & 0xffu)); v.w = __ldg(a.X + xbase + (c4 >> 24));
+                }
+                *reinterpret_cast<float4*>(dst) = v;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float* src = a.X + xbase + ((c4 >> (8 * j)) & 0xffu);
+#pragma unroll
+                    for (int bt = 0; bt < BT; ++bt) dst[j * BT + bt] = bt < a.nb ? __ldg(src + (long long)bt * a.ldx) : 0.f;
+                }
+            }
+        }
+#ifdef CSB_PHASE_CLOCKS
+        , wprof
+#endif
+        );
+#ifdef CSB_PHASE_CLOCKS
+        const long long tc2 = clock64();
+        CSB_ADD(3, tc2 - tc1);
+#endif
         if ((ch.w & 3u) != kFlushNone) {
             flush_block_row<BT, G>(a, zs, L.zs_stride, ch.z, ch.w, lane);
             __syncwarp();
         }
+#ifdef CSB_PHASE_CLOCKS
+        CSB_ADD(4, clock64() - tc2);
+#endif
         if (lane == 0 && refill.bytes) {
             mbar_expect_tx(&bars[s], refill.bytes);
             bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)refill.off16 * 16, refill.bytes, &bars[s]);
         }
     }
+    CSB_STAMP(5);
+#ifdef CSB_PHASE_CLOCKS
+    if (lane == 0 && gw < a.n_warps) for (int i = 0; i < 6; ++i) a.clocks[(size_t)(a.n_warps + gw) * 6 + i] = wprof[i];
+#endif
 }
 
 #define CSB_CUDA(call)                                                                     \
@@ -230,7 +311,12 @@ int plan_product(csb_matrix* A) {
     P.n_warps = n_warps;
     if ((rc = upload(H.stream.bytes, &P.d_stream)) != CSB_OK) return rc;
     if ((rc = upload(H.stream.chunks, &P.d_chunks)) != CSB_OK) return rc;
-    if ((rc = upload(H.stream.warp_chunk_begin, &P.d_warp_chunk_begin)) != CSB_OK) return rc;
+    std::vector<uint4> wdesc(n_warps);
+    for (int w = 0; w < n_warps; ++w) {
+        const uint32_t c0 = H.stream.warp_chunk_begin[w], c1 = H.stream.warp_chunk_begin[w + 1];
+        wdesc[w] = make_uint4(c0, c1, c0 < c1 ? H.stream.chunks[c0].off16 : 0u, c0 < c1 ? H.stream.chunks[c0].bytes : 0u);
+    }
+    if ((rc = upload(wdesc, (uint4**)&P.d_warp_desc)) != CSB_OK) return rc;
     if ((rc = upload(H.part_base, &P.d_part_base)) != CSB_OK) return rc;
     if ((rc = upload(H.part_count, &P.d_part_count)) != CSB_OK) return rc;
     CSB_CUDA(cudaMalloc((void**)&P.d_arrivals, std::max<size_t>(A->nbr, 1) * 4));
@@ -250,7 +336,7 @@ void free_product(csb_matrix* A) {
     int prev = 0;
     cudaGetDevice(&prev);
     cudaSetDevice(A->device);
-    cudaFree(P.d_stream); cudaFree(P.d_chunks); cudaFree(P.d_warp_chunk_begin); cudaFree(P.d_part_base);
+    cudaFree(P.d_stream); cudaFree(P.d_chunks); cudaFree(P.d_warp_desc); cudaFree(P.d_part_base);
     cudaFree(P.d_part_count); cudaFree(P.d_arrivals); cudaFree(P.d_partials);
     if (P.h_status) cudaFreeHost(P.h_status);
     P = ProductPlan{};
@@ -296,6 +382,13 @@ static int dispatch_tile(const csb_matrix* A, const ProductArgs& a, cudaStream_t
     return h ? dispatch_gw<__half, 1>(A, a, st) : dispatch_gw<float, 1>(A, a, st);
 }
 
+#ifdef CSB_PHASE_CLOCKS
+long long* g_phase_clocks = nullptr;
+extern "C" int csb_debug_phase_clocks(long long* host_out, int n_warps) {
+    return (int)cudaMemcpy(host_out, g_phase_clocks, (size_t)n_warps * 6 * 8, cudaMemcpyDeviceToHost);
+}
+#endif
+
 int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream) {
     const ProductPlan& P = A->product;
     if (P.h_status && *P.h_status != 0) { set_error("an earlier product on this handle gave up waiting on the device (code %u)", *P.h_status); return CSB_ERR_TIMEOUT; }
@@ -303,10 +396,16 @@ int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, 
     CSB_CUDA(cudaGetDevice(&prev));
     if (prev != A->device) CSB_CUDA(cudaSetDevice(A->device));
     ProductArgs a{};
-    a.stream = P.d_stream; a.chunks = P.d_chunks; a.warp_chunk_begin = P.d_warp_chunk_begin;
+    a.stream = P.d_stream; a.chunks = P.d_chunks; a.warp_desc = (const uint4*)P.d_warp_desc;
     a.part_base = P.d_part_base; a.part_count = P.d_part_count; a.arrivals = P.d_arrivals; a.partials = P.d_partials;
     a.ldx = ldx; a.ldy = ldy; a.status = P.d_status; a.n_warps = P.n_warps;
     a.rows = (int)A->rows; a.cols = (int)A->cols; a.block_r = A->block_r; a.stage_bytes = P.stage_bytes; a.stages = P.stages;
+#ifdef CSB_PHASE_CLOCKS
+    static long long* d_clocks = nullptr;
+    if (!d_clocks) cudaMalloc((void**)&d_clocks, (size_t)1 << 22);
+    a.clocks = d_clocks;
+    g_phase_clocks = d_clocks;
+#endif
     cudaStream_t st = (cudaStream_t)stream;
     int rc = CSB_OK;
     for (int b0 = 0; b0 < batch && rc == CSB_OK;) {

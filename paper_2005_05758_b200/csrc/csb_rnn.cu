@@ -40,13 +40,13 @@ struct RnnSmem {
     int zs_stride;
     __host__ __device__ RnnSmem(int W, int G, int stages, int stage_bytes, int resident, int max_warp_bytes, int max_U, int BT,
                                 int B, int max_C) {
-        zs_stride = 4 * max_U * BT;                    // floats per lane group
+        zs_stride = 4 * max_U * BT + group_pad(32 / G);   // floats per lane group
         weights = 0;
         const size_t per_warp = resident ? (size_t)max_warp_bytes : (size_t)stages * stage_bytes;
         bars = weights + (size_t)W * per_warp;
         zs = (bars + (size_t)W * (resident ? 1 : stages) * 8 + 15) & ~(size_t)15;
         xg = (zs + (size_t)W * G * zs_stride * 4 + 15) & ~(size_t)15;
-        v = (xg + (size_t)W * G * kMaxNk * BT * 4 + 15) & ~(size_t)15;
+        v = (xg + (size_t)W * G * xg_stride(32 / G, BT) * 4 + 15) & ~(size_t)15;
         cs = (v + (BT == 1 ? (size_t)max_C * 4 : 0) + 15) & ~(size_t)15;
         flag = (cs + (size_t)max_U * B * 4 + 15) & ~(size_t)15;
         total = flag + 16;
@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S.bars) + warp * (a.resident ? 1 : a.stages);
     float* zs_all = reinterpret_cast<float*>(smem + S.zs);
     float* zs = zs_all + warp * G * S.zs_stride;
-    float* xg = reinterpret_cast<float*>(smem + S.xg) + warp * G * kMaxNk * BT;
+    float* xg = reinterpret_cast<float*>(smem + S.xg) + warp * G * xg_stride(GW, BT);
     float* vs = reinterpret_cast<float*>(smem + S.v);
     float* cs = reinterpret_cast<float*>(smem + S.cs);
     volatile int* s_flag = reinterpret_cast<volatile int*>(smem + S.flag);
@@ -168,11 +168,28 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                 const int nb = min(BT, B - b0);
                 for (int i = lane; i < G * S.zs_stride; i += 32) zs[i] = 0.f;
                 __syncwarp();
-                auto gather = [&](uint32_t col, uint32_t flags, int bt) -> float {
-                    if (BT == 1) return vs[(flags & kItemRecurrent) ? col + I : col];
-                    if (bt >= nb) return 0.f;
-                    return (flags & kItemRecurrent) ? __ldcg(rec_src + (size_t)(b0 + bt) * H + col)
-                                                    : __ldcg(in_src + (size_t)(b0 + bt) * in_ld + col);
+                auto gather = [&](uint32_t xbase, uint32_t c4, uint32_t flags, int left, float* dst) {
+                    const bool rec = (flags & kItemRecurrent) != 0;
+                    if (BT == 1) {
+                        // padding indices are zero; xbase (+ I for the recurrent part) is the block's
+                        // first column, which exists, so they may be read
+                        // (32-bit sum: for a block that straddles the x | h boundary xbase is "negative")
+                        const uint32_t base = xbase + (rec ? (uint32_t)I : 0u);
+                        float4 v;
+                        v.x = vs[base + (c4 & 0xffu)]; v.y = vs[base + ((c4 >> 8) & 0xffu)];
+                        v.z = vs[base + ((c4 >> 16) & 0xffu)]; v.w = vs[base + (c4 >> 24)];
+                        *reinterpret_cast<float4*>(dst) = v;
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t col = xbase + ((c4 >> (8 * j)) & 0xffu);
+#pragma unroll
+                            for (int bt = 0; bt < BT; ++bt)
+                                dst[j * BT + bt] = (j < left && bt < nb)
+                                    ? (rec ? __ldcg(rec_src + (size_t)(b0 + bt) * H + col) : __ldcg(in_src + (size_t)(b0 + bt) * in_ld + col))
+                                    : 0.f;
+                        }
+                    }
                 };
                 if (a.resident) {
                     if (alive)
