@@ -10,6 +10,9 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (sm_100a)")
+    # the shared library is a build product (not in the history): compile it when it is missing or stale
+    from paper_2005_05758_b200 import build
+    build.build()
 
 
 def pytest_collection_modifyitems(config, items):
