@@ -139,6 +139,35 @@ int csb_spmm(const csb_matrix_t* A, const float* X, int64_t ldx, int batch, floa
              void* stream);
 
 /*
+ * csb_spmv_static_scratch -- y = A . x like csb_spmv, for callers that must not allocate device
+ * memory.  (The paper has no counterpart; this is a packaging variant of the same kernel.)
+ *
+ * Who needs it: code that runs after an application has frozen its device-memory budget, or from
+ * a thread or callback in which cudaMalloc / cudaFree are off limits because they synchronise the
+ * whole device and may fail late -- an inference server's request loop, a real-time control loop,
+ * a plug-in that is handed a fixed arena.  The product kernel needs scratch in global memory
+ * (partial sums of block-rows shared by several warps, and their arrival counters).  csb_spmv
+ * takes it from buffers allocated together with the handle; this variant takes it from one fixed
+ * 4 MiB array that is part of the library image, so it calls no allocator at all (neither CUDA's
+ * nor any library's).  Every GPU that loads the library holds those 4 MiB until the process ends.
+ *
+ *   A, x, y, stream   as for csb_spmv (device pointers, fp32, y overwritten, asynchronous).
+ * Limits: at most 16384 block-rows (64 KiB of counters) and 4 MiB - 64 KiB of partial sums,
+ * i.e. (number of shared warp/block-row pairs) * block_r * 4 bytes; a matrix beyond either limit
+ * is refused with CSB_ERR_UNSUPPORTED and a message that names both sizes (csb_spmv still works).
+ * Set-up: the first call on each device looks up the array's device address (once, cached); make
+ * that first call outside of any stream capture.  Every call clears the counters it is going to
+ * use on `stream` before the kernel; the partial sums are not cleared because each slot is
+ * written before it is read.  The array is shared by ALL handles and keeps the last call's
+ * contents: two calls of this function that overlap on the GPU (different streams, or different
+ * host threads without ordering between their streams) race on it and give wrong results.  Calls
+ * queued on one stream are safe.  Results equal csb_spmv's bit for bit.
+ * Errors: INVALID_ARG (null), UNSUPPORTED (host-only handle, limits, device ordinal > 63),
+ * TIMEOUT (an earlier product on the handle gave up a bounded wait), CUDA.
+ */
+int csb_spmv_static_scratch(const csb_matrix_t* A, const float* x, float* y, void* stream);
+
+/*
  * csb_lstm_forward -- a stack of LSTM layers over a whole sequence in one persistent kernel
  * (Section 2.1; one CSB product per layer and step, gate arithmetic fused behind it).
  *   W[l]     CSB matrix [4*H, I_l + H], I_0 = I, I_l = H above; stacked gate rows i, f, g, o;

@@ -51,6 +51,8 @@ lib.csb_info.argtypes = [_P, C.POINTER(csb_info_t)]
 lib.csb_free.argtypes = [_P]
 lib.csb_free.restype = None
 lib.csb_spmv.argtypes = [_P, _P, _P, _P]
+lib.csb_spmv_static_scratch.argtypes = [_P, _P, _P, _P]
+lib.csb_spmv_static_scratch.restype = C.c_int
 lib.csb_spmm.argtypes = [_P, _P, C.c_int64, C.c_int, _P, C.c_int64, _P]
 lib.csb_lstm_forward.argtypes = [C.c_int, C.POINTER(_P), C.POINTER(_P), _P, C.c_int64, C.c_int, _P, _P, _P, _P, _P,
                                  C.c_uint, _P]
@@ -155,6 +157,12 @@ def csb_encode(dense: np.ndarray, block_r: int, block_c: int, row_keep: np.ndarr
 
 def csb_spmv(A: CsbMatrix, x, y, stream=None) -> None:
     _check(lib.csb_spmv(A.handle, _ptr(x), _ptr(y), _stream(stream)))
+
+
+def csb_spmv_static_scratch(A: CsbMatrix, x, y, stream=None) -> None:
+    """csb_spmv for callers that may not allocate device memory: the kernel's scratch is a fixed
+    array inside the library (4 MiB per GPU), shared by all handles -- do not overlap calls."""
+    _check(lib.csb_spmv_static_scratch(A.handle, _ptr(x), _ptr(y), _stream(stream)))
 
 
 def csb_spmm(A: CsbMatrix, X, Y, stream=None) -> None:

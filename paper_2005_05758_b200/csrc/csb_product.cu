@@ -8,6 +8,7 @@
 // read once, in large aligned pieces, while the irregular indexing happens on chip.
 #include <algorithm>
 #include <cstdio>
+#include <mutex>
 
 #include "csb_internal.hpp"
 #include "csb_device.cuh"
@@ -420,4 +421,76 @@ int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, 
     return rc;
 }
 
+
+// ---------------------------------------------------------------------------------------
+// SpMV whose scratch is built into the library image (see csb_spmv_static_scratch in csb.h).
+//
+// The block-row reduction of the product kernel needs scratch in global memory: one slot of
+// partial sums per (warp, block-row) pair that shares a block-row, and one arrival counter per
+// block-row.  csb_spmv keeps that scratch in buffers cudaMalloc'ed with the handle.  Here it
+// sits in one fixed array that every GPU loading the library carries until the process exits.
+// ---------------------------------------------------------------------------------------
+constexpr size_t kStaticArrivalBytes = 64u << 10;                 // 16384 block-rows
+constexpr size_t kStaticPartialBytes = (4u << 20) - kStaticArrivalBytes;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticArrivalBytes + kStaticPartialBytes];
+
+// In host code the array's name stands for the symbol, not for an address on the device; the
+// address is asked for once per device, with that device current.
+static unsigned char* g_static_scratch_addr[64] = {};
+static std::mutex g_static_scratch_mu;
+
+static int static_scratch_address(int device, unsigned char** out) {
+    if (device < 0 || device >= 64) { set_error("device ordinal %d is outside 0..63", device); return CSB_ERR_UNSUPPORTED; }
+    std::lock_guard<std::mutex> lk(g_static_scratch_mu);
+    if (!g_static_scratch_addr[device]) {
+        void* p = nullptr;
+        CSB_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));      // the caller made `device` current
+        g_static_scratch_addr[device] = (unsigned char*)p;
+    }
+    *out = g_static_scratch_addr[device];
+    return CSB_OK;
+}
+
+int launch_spmv_static_scratch(const csb_matrix* A, const float* x, float* y, void* stream) {
+    const ProductPlan& P = A->product;
+    if (P.h_status && *P.h_status != 0) { set_error("an earlier product on this handle gave up waiting on the device (code %u)", *P.h_status); return CSB_ERR_TIMEOUT; }
+    const size_t need_arrivals = (size_t)A->nbr * 4, need_partials = (size_t)P.n_slots * A->block_r * 4;
+    if (need_arrivals > kStaticArrivalBytes || need_partials > kStaticPartialBytes) {
+        set_error("matrix needs %zu bytes of arrival counters and %zu bytes of partial sums; the built-in scratch holds %zu and %zu "
+                  "(use csb_spmv, whose scratch is sized per handle)", need_arrivals, need_partials, kStaticArrivalBytes, kStaticPartialBytes);
+        return CSB_ERR_UNSUPPORTED;
+    }
+    int prev = 0;
+    CSB_CUDA(cudaGetDevice(&prev));
+    if (prev != A->device) CSB_CUDA(cudaSetDevice(A->device));
+    struct Restore { int prev, cur; ~Restore() { if (prev != cur) cudaSetDevice(prev); } } restore{prev, A->device};
+    unsigned char* scratch = nullptr;
+    int rc = static_scratch_address(A->device, &scratch);
+    if (rc != CSB_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    // The array keeps whatever the last call left.  The counters must start at zero; the partial
+    // sums need no clearing, every slot that is read is written first in the same launch.
+    CSB_CUDA(cudaMemsetAsync(scratch, 0, need_arrivals, st));
+    ProductArgs a{};
+    a.stream = P.d_stream; a.chunks = P.d_chunks; a.warp_desc = (const uint4*)P.d_warp_desc;
+    a.part_base = P.d_part_base; a.part_count = P.d_part_count;
+    a.arrivals = reinterpret_cast<uint32_t*>(scratch);
+    a.partials = reinterpret_cast<float*>(scratch + kStaticArrivalBytes);
+    a.ldx = A->cols; a.ldy = A->rows; a.status = P.d_status; a.n_warps = P.n_warps;
+    a.rows = (int)A->rows; a.cols = (int)A->cols; a.block_r = A->block_r; a.stage_bytes = P.stage_bytes; a.stages = P.stages;
+    a.X = x; a.Y = y; a.nb = 1;
+#ifdef CSB_PHASE_CLOCKS
+    a.clocks = g_phase_clocks;
+    if (!a.clocks) { set_error("instrumented build: call csb_spmv once first"); return CSB_ERR_UNSUPPORTED; }
+#endif
+    return dispatch_tile(A, a, st, 1);
+}
+
 }  // namespace csb
+
+extern "C" int csb_spmv_static_scratch(const csb_matrix_t* A, const float* x, float* y, void* stream) {
+    csb::clear_error();
+    if (!A || !x || !y) { csb::set_error("A, x or y is NULL"); return CSB_ERR_INVALID_ARG; }
+    if (A->device < 0) { csb::set_error("matrix was encoded host-only (device = -1)"); return CSB_ERR_UNSUPPORTED; }
+    return csb::launch_spmv_static_scratch(A, x, y, stream);
+}
