@@ -54,6 +54,10 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
+// Orders this thread's earlier generic-proxy view of memory before the asynchronous (bulk copy)
+// accesses it issues next.
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
 template <typename T> struct WordTraits;
 template <> struct WordTraits<__half> {
     static constexpr int kRows = 2;
@@ -72,7 +76,7 @@ template <> struct WordTraits<float> {
 __host__ __device__ constexpr int group_pad(int gw) { return gw == 32 ? 0 : gw; }
 __host__ __device__ constexpr int xg_stride(int gw, int bt) { return kMaxNk * bt + group_pad(gw); }
 
-#ifdef CSB_PHASE_CLOCKS
+#ifdef CSB_WALK_CLOCKS
 // instrumented build only: per-thread lap counters of walk_chunk (header, gather, multiply, fold, scatter, rounds)
 static __device__ long long csb_walk_prof_dummy;
 #define csb_walk_prof csb_walk_prof_local
@@ -104,7 +108,7 @@ __device__ __forceinline__ uint32_t chunk_bytes(const uint4& ch) {
 template <typename T, int BT, int GW, typename Gather>
 __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch, int lane, float* __restrict__ xg_w,
                                            float* __restrict__ zs_w, int zs_stride, Gather gather4
-#ifdef CSB_PHASE_CLOCKS
+#ifdef CSB_WALK_CLOCKS
                                            , long long* csb_walk_prof_local = &csb_walk_prof_dummy
 #endif
                                            ) {
@@ -121,7 +125,7 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
     const uint8_t* end = p + 16 * mine;
     float* xg = xg_w + g * xg_stride(GW, BT);
     float* zs = zs_w + g * zs_stride;
-#ifdef CSB_PHASE_CLOCKS
+#ifdef CSB_WALK_CLOCKS
     long long tq = clock64();
 #define CSB_WALK_LAP(i) do { const long long n_ = clock64(); csb_walk_prof[i] += n_ - tq; tq = n_; } while (0)
 #else
@@ -227,7 +231,7 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
         }
         __syncwarp();
         CSB_WALK_LAP(4);
-#ifdef CSB_PHASE_CLOCKS
+#ifdef CSB_WALK_CLOCKS
         csb_walk_prof[5] += 1;
 #endif
     }

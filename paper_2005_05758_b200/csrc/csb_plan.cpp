@@ -27,12 +27,14 @@ size_t item_bytes(const csb_matrix* A, const ItemSpec& it) {
     return pad_to(sizeof(ItemHeader) + pad_to((size_t)nk, 4) + pad_to((size_t)mr, 4) + (size_t)nk * row_words(A, mr) * 4, kItemAlign);
 }
 
-// Lock-step cost of an item for a lane group of width gw: column steps plus a fixed part
-// for header decode, gather, fold and scatter.
+// Lock-step cost of an item for a lane group of width gw, in units of one column step of the
+// multiply loop (about 7 instructions): the column steps plus a fixed part for header decode,
+// gather, fold and scatter (about 190 instructions, from instruction counts of the kernel).
+enum { kItemFixedSteps = 27 };
 int item_steps(const csb_matrix* A, const ItemSpec& it, int gw) {
     const int nk = it.k1 - it.k0, RL = std::max(1, row_words(A, it.r1 - it.r0));
     const int S = std::max(1, gw / RL);
-    return (nk + S - 1) / S + 8;
+    return (nk + S - 1) / S + kItemFixedSteps;
 }
 
 void emit_item(const csb_matrix* A, const ItemSpec& it, int gw, std::vector<uint8_t>& out) {

@@ -41,19 +41,18 @@ struct ProductArgs {
 #define CSB_ADD(i, v) do { } while (0)
 #endif
 
-constexpr int kXRegs = 4;      // float4 registers per thread used to stage x (covers 8192 columns at 512 threads)
-
 __host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t)15; }
 
 // Shared-memory carve-up, identical on host and device.
 struct ProductSmem {
-    size_t ring, bars, zs, xg, xs, total;
+    size_t ring, bars, xbar, zs, xg, xs, total;
     int zs_stride;                                     // floats per lane group
     __host__ __device__ ProductSmem(int W, int G, int stages, int stage_bytes, int block_r, int BT, int cols_in_smem) {
         zs_stride = block_r * BT + group_pad(32 / G);
         ring = 0;
         bars = ring + (size_t)W * stages * stage_bytes;
-        zs = align16(bars + (size_t)W * stages * 8);
+        xbar = bars + (size_t)W * stages * 8;
+        zs = align16(xbar + 8);
         xg = align16(zs + (size_t)W * G * zs_stride * 4);
         xs = align16(xg + (size_t)W * G * xg_stride(32 / G, BT) * 4);
         total = align16(xs + (size_t)cols_in_smem * 4);
@@ -133,15 +132,16 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
     uint4 wd = make_uint4(0u, 0u, 0u, 0u);
     if (gw < a.n_warps) wd = __ldg(a.warp_desc + gw);
     const uint32_t c0 = wd.x, c1 = wd.y;
-    float4 xr[kXRegs];
-    const bool x_vec = a.x_in_smem && (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && a.cols <= (int)blockDim.x * 4 * kXRegs;
-    if (x_vec) {
-        const float4* x4 = reinterpret_cast<const float4*>(a.X);
-#pragma unroll
-        for (int j = 0; j < kXRegs; ++j) {
-            const int i = threadIdx.x + j * blockDim.x;
-            xr[j] = i < a.cols / 4 ? __ldg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+    // x comes in with one bulk copy per CTA when its address and size allow (16-byte multiples)
+    bool x_dead = false;
+    uint64_t* xbar = reinterpret_cast<uint64_t*>(smem + L.xbar);
+    const bool x_bulk = a.x_in_smem && (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && (a.cols & 3) == 0;
+    if (x_bulk && threadIdx.x == 0) {
+        mbar_init(xbar, 1);
+        mbar_fence_init();
+        mbar_expect_tx(xbar, (uint32_t)a.cols * 4u);
+        for (uint32_t off = 0; off < (uint32_t)a.cols * 4u; off += 16384u)
+            bulk_g2s(smem + L.xs + off, reinterpret_cast<const uint8_t*>(a.X) + off, min(16384u, (uint32_t)a.cols * 4u - off), xbar);
     }
     if (lane == 0) {
         for (int s = 0; s < a.stages; ++s) mbar_init(&bars[s], 1);
@@ -158,24 +158,18 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
     }
     for (int i = lane; i < G * L.zs_stride; i += 32) zs[i] = 0.f;
     if (a.x_in_smem) {
-        float* xw = reinterpret_cast<float*>(smem + L.xs);
-        if (x_vec) {
-#pragma unroll
-            for (int j = 0; j < kXRegs; ++j) {
-                const int i = threadIdx.x + j * blockDim.x;
-                if (i < a.cols / 4) reinterpret_cast<float4*>(xw)[i] = xr[j];
-            }
-            for (int i = (a.cols & ~3) + threadIdx.x; i < a.cols; i += blockDim.x) xw[i] = __ldg(a.X + i);
-        } else {
+        if (!x_bulk) {
+            float* xw = reinterpret_cast<float*>(smem + L.xs);
             for (int i = threadIdx.x; i < a.cols; i += blockDim.x) xw[i] = __ldg(a.X + i);
         }
-        __syncthreads();
+        __syncthreads();                              // x staged by loads, or xbar initialised
+        if (x_bulk && !mbar_wait_bounded(xbar, 0)) x_dead = true;     // reported and drained below
     } else {
         __syncwarp();
     }
 
     CSB_STAMP(1);
-#ifdef CSB_PHASE_CLOCKS
+#if defined(CSB_PHASE_CLOCKS) || defined(CSB_WALK_CLOCKS)
     long long wprof[6] = {0, 0, 0, 0, 0, 0};
 #endif
     for (uint32_t c = c0; c < c1; ++c) {
@@ -185,13 +179,13 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
         const int s = (int)((c - c0) % (uint32_t)a.stages);
         const uint32_t parity = ((c - c0) / (uint32_t)a.stages) & 1u;
         const Chunk refill = (c + a.stages < c1) ? a.chunks[c + a.stages] : Chunk{0, 0};
-        bool dead = !mbar_wait_bounded(&bars[s], parity);
+        bool dead = x_dead || !mbar_wait_bounded(&bars[s], parity);
         dead = __any_sync(0xffffffffu, dead);
         if (dead) {
             // report, then give the copies still in flight a bounded chance to land before leaving
             if (lane == 0) {
                 *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout;
-                for (uint32_t j = c + 1; j < c1 && j < c + (uint32_t)a.stages; ++j)
+                for (uint32_t j = c; j < c1 && j < c + (uint32_t)a.stages; ++j)
                     mbar_wait_bounded(&bars[(j - c0) % (uint32_t)a.stages], ((j - c0) / (uint32_t)a.stages) & 1u);
             }
             break;
@@ -224,7 +218,7 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
                 }
             }
         }
-#ifdef CSB_PHASE_CLOCKS
+#ifdef CSB_WALK_CLOCKS
         , wprof
 #endif
         );

@@ -33,10 +33,20 @@ struct RnnArgs {
     unsigned long long barrier_ns;
     unsigned int barrier_extra;   // test hook: arrivals that never come
     int T, B, H, L, gates, stage_bytes, stages, resident, max_warp_bytes, max_U, max_C;
+    int v_bulk;                // batch 1: [u_t ; h_{t-1}] may come in by bulk copy (16-byte aligned pieces)
+#ifdef CSB_PHASE_CLOCKS
+    long long* clocks;         // [n_ctas][4] cycles summed over ticks: stage, walk, gates, barrier
+#endif
 };
 
+#ifdef CSB_PHASE_CLOCKS
+#define RNN_LAP(i) do { if (threadIdx.x == 0) { const long long n_ = clock64(); rprof[i] += n_ - rt; rt = n_; } } while (0)
+#else
+#define RNN_LAP(i) do { } while (0)
+#endif
+
 struct RnnSmem {
-    size_t weights, bars, zs, xg, v, cs, flag, total;
+    size_t weights, bars, zs, xg, v, cs, zsum, vbar, flag, total;
     int zs_stride;
     __host__ __device__ RnnSmem(int W, int G, int stages, int stage_bytes, int resident, int max_warp_bytes, int max_U, int BT,
                                 int B, int max_C) {
@@ -48,7 +58,9 @@ struct RnnSmem {
         xg = (zs + (size_t)W * G * zs_stride * 4 + 15) & ~(size_t)15;
         v = (xg + (size_t)W * G * xg_stride(32 / G, BT) * 4 + 15) & ~(size_t)15;
         cs = (v + (BT == 1 ? (size_t)max_C * 4 : 0) + 15) & ~(size_t)15;
-        flag = (cs + (size_t)max_U * B * 4 + 15) & ~(size_t)15;
+        zsum = (cs + (size_t)max_U * B * 4 + 15) & ~(size_t)15;
+        vbar = (zsum + (size_t)4 * max_U * BT * 4 + 15) & ~(size_t)15;
+        flag = vbar + 16;
         total = flag + 16;
     }
 };
@@ -103,6 +115,9 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     float* vs = reinterpret_cast<float*>(smem + S.v);
     float* cs = reinterpret_cast<float*>(smem + S.cs);
     volatile int* s_flag = reinterpret_cast<volatile int*>(smem + S.flag);
+    float* zsum = reinterpret_cast<float*>(smem + S.zsum);
+    uint64_t* vbar = reinterpret_cast<uint64_t*>(smem + S.vbar);
+    uint32_t v_uses = 0;
 
     const uint32_t c0 = a.warp_chunk_begin[me.warp0 + warp], c1 = a.warp_chunk_begin[me.warp0 + warp + 1];
     const uint32_t nchunks = c1 - c0;
@@ -145,11 +160,19 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
         const int b = i / U, u = i % U;
         cs[b * a.max_U + u] = a.gates == 4 ? a.cstate[((size_t)layer * B + b) * H + u0 + u] : 0.f;
     }
-    if (threadIdx.x == 0) *s_flag = 1;
+    if (threadIdx.x == 0) {
+        *s_flag = 1;
+        mbar_init(vbar, 1);
+        mbar_fence_init();
+    }
     __syncthreads();
 
     const float* bias = a.bias[layer];
     const int n_ticks = a.T + a.L - 1;
+#ifdef CSB_PHASE_CLOCKS
+    long long rprof[4] = {0, 0, 0, 0};
+    long long rt = clock64();
+#endif
     for (int tick = 0; tick < n_ticks; ++tick) {
         const int t = tick - layer;
         const bool active = t >= 0 && t < a.T;
@@ -160,10 +183,25 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
             float* h_dst = a.hbuf + ((size_t)layer * 2 + (t & 1)) * B * H;
             const int in_ld = layer == 0 ? I : H;
             if (BT == 1) {
+                if (a.v_bulk) {
+                    // two bulk copies bring [u_t ; h_{t-1}] in; h was written by other CTAs with
+                    // ordinary stores before the grid barrier, so the copy is ordered behind this
+                    // thread's (acquired) view with a proxy fence
+                    if (threadIdx.x == 0) {
+                        fence_proxy_async_all();
+                        mbar_expect_tx(vbar, (uint32_t)C * 4u);
+                        bulk_g2s(vs, in_src, (uint32_t)I * 4u, vbar);
+                        bulk_g2s(vs + I, rec_src, (uint32_t)H * 4u, vbar);
+                    }
+                    if (!mbar_wait_bounded(vbar, v_uses & 1u)) alive = false;
+                    ++v_uses;
+                } else {
 #pragma unroll 8
-                for (int i = threadIdx.x; i < C; i += blockDim.x) vs[i] = __ldcg(i < I ? in_src + i : rec_src + (i - I));
-                __syncthreads();
+                    for (int i = threadIdx.x; i < C; i += blockDim.x) vs[i] = __ldcg(i < I ? in_src + i : rec_src + (i - I));
+                    __syncthreads();
+                }
             }
+            RNN_LAP(0);
             for (int b0 = 0; b0 < B; b0 += BT) {
                 const int nb = min(BT, B - b0);
                 for (int i = lane; i < G * S.zs_stride; i += 32) zs[i] = 0.f;
@@ -224,15 +262,30 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                     }
                 }
                 __syncthreads();
+                RNN_LAP(1);
                 // ---- gate arithmetic for this batch tile ----
+                // add the W*G private accumulator copies: `parts` adjacent lanes share one entry,
+                // each adds every parts-th copy in order, then a fixed xor-tree joins them
+                {
+                    const int NZ = 4 * U * BT, NC = W * G;
+                    int parts = 1;
+                    while (parts < 32 && parts * 2 * NZ <= (int)blockDim.x) parts *= 2;
+                    const int span = (NZ * parts + 31) & ~31;
+                    for (int idx = threadIdx.x; idx < span; idx += blockDim.x) {
+                        const int e = idx / parts, pt = idx % parts;
+                        float sum = 0.f;
+                        if (e < NZ)
+                            for (int c = pt; c < NC; c += parts) sum += zs_all[c * S.zs_stride + e];
+                        for (int off = parts >> 1; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+                        if (e < NZ && pt == 0) zsum[e] = sum;
+                    }
+                }
+                __syncthreads();
                 for (int i = threadIdx.x; i < U * nb; i += blockDim.x) {
                     const int bt = i / U, u = i % U, b = b0 + bt;
-                    float z[4] = {0.f, 0.f, 0.f, 0.f};
-                    for (int w = 0; w < W * G; ++w) {           // warps, then lane groups: a fixed order
-                        const float* zw = zs_all + w * S.zs_stride;
+                    float z[4];
 #pragma unroll
-                        for (int g = 0; g < 4; ++g) z[g] += zw[(g * U + u) * BT + bt];
-                    }
+                    for (int g = 0; g < 4; ++g) z[g] = zsum[(g * U + u) * BT + bt];
                     float h;
                     if (a.gates == 4) {
                         if (bias) {
@@ -258,13 +311,18 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                     if (layer == a.L - 1 && a.y) a.y[((size_t)t * B + b) * H + u0 + u] = h;
                 }
                 __syncthreads();
+                RNN_LAP(2);
             }
         }
         if (tick + 1 < n_ticks) {
             if (!grid_barrier(a, (unsigned)(tick + 1) * (gridDim.x + a.barrier_extra), s_flag)) break;
         }
+        RNN_LAP(3);
     }
     if (!alive && lane == 0) *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout;
+#ifdef CSB_PHASE_CLOCKS
+    if (threadIdx.x == 0) for (int i = 0; i < 4; ++i) a.clocks[(size_t)blockIdx.x * 4 + i] = rprof[i];
+#endif
 }
 
 
@@ -405,6 +463,15 @@ static int dispatch_rnn_gw(const RnnPlan* P, RnnArgs& a, cudaStream_t st) {
     }
 }
 
+#ifdef CSB_PHASE_CLOCKS
+static long long* g_rnn_clocks = nullptr;
+static int g_rnn_clock_ctas = 0;
+extern "C" int csb_debug_rnn_clocks(long long* host_out, int max_ctas) {
+    cudaMemcpy(host_out, g_rnn_clocks, (size_t)std::min(max_ctas, g_rnn_clock_ctas) * 4 * 8, cudaMemcpyDeviceToHost);
+    return g_rnn_clock_ctas;
+}
+#endif
+
 static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const float* const* bias, const float* x, int64_t T,
                        int B, const float* h0, const float* c0, float* y, float* hT, float* cT, unsigned flags, void* stream) {
     clear_error();
@@ -491,7 +558,20 @@ static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const flo
     for (int l = 0; l < L; ++l) { a.bias[l] = bias ? bias[l] : nullptr; a.in_size[l] = in_size[l]; }
     a.barrier = P->d_barrier; a.status = P->d_status; a.barrier_ns = g_barrier_ns; a.barrier_extra = g_barrier_extra;
     a.T = (int)T; a.B = B; a.H = H; a.L = L; a.gates = gates; a.stage_bytes = P->stage_bytes; a.stages = P->stages;
+    a.v_bulk = 0;
+    if (P->BT == 1 && H % 4 == 0 && (reinterpret_cast<uintptr_t>(dx) & 15) == 0) {
+        a.v_bulk = 1;
+        for (int l = 0; l < L; ++l) if (in_size[l] % 4) a.v_bulk = 0;
+    }
+    if (env_int("CSB_RNN_NO_VBULK", 0)) a.v_bulk = 0;
     a.resident = P->resident; a.max_warp_bytes = P->max_warp_bytes; a.max_U = P->max_U; a.max_C = P->max_C;
+#ifdef CSB_PHASE_CLOCKS
+    static long long* d_rclocks = nullptr;
+    if (!d_rclocks) cudaMalloc((void**)&d_rclocks, 1 << 16);
+    a.clocks = d_rclocks;
+    g_rnn_clocks = d_rclocks;
+    g_rnn_clock_ctas = P->n_ctas;
+#endif
     int rc;
     const bool half = P->val_dtype == CSB_F16;
     if (P->BT == 1) rc = half ? dispatch_rnn_gw<__half, 1>(P, a, st) : dispatch_rnn_gw<float, 1>(P, a, st);

@@ -120,15 +120,39 @@ int plan_rnn_host(int gates, int n_layers, const csb_matrix* const* Wm, const in
         double tot = 0;
         for (double c : ucost) tot += c;
         std::vector<int>& cut = cuts[l];
-        cut.assign(ncta[l] + 1, H);
-        cut[0] = 0;
-        double cum = 0;
-        int t = 1;
-        for (int u = 0; u < H && t < ncta[l]; ++u) {
-            cum += ucost[u];
-            const int left_units = H - (u + 1), left_tiles = ncta[l] - t;
-            const bool full = u + 1 - cut[t - 1] >= kMaxTileUnits;
-            if (cum >= tot * t / ncta[l] || left_units <= left_tiles || full) cut[t++] = u + 1;
+        // A tile that straddles two block-rows gets twice the items of one that does not, and the
+        // fixed cost per item is what dominates small items.  So when the gates' block-rows line
+        // up with the units (H a multiple of the block height) and there are at least as many
+        // CTAs as block-rows, every block-row is cut into the same number of tiles, by cost, and
+        // no tile straddles.  Otherwise: contiguous tiles of about equal cost.
+        const int BR = A->block_r, nbr_g = (H + BR - 1) / BR;
+        const int per_row = ncta[l] / nbr_g;
+        if (H % BR == 0 && per_row >= 1 && BR / per_row <= kMaxTileUnits && per_row <= BR) {
+            cut.assign(1, 0);
+            for (int bi = 0; bi < nbr_g; ++bi) {
+                double rtot = 0, cum = 0;
+                for (int u = bi * BR; u < (bi + 1) * BR; ++u) rtot += ucost[u];
+                int t = 1;
+                for (int u = bi * BR; u < (bi + 1) * BR && t < per_row; ++u) {
+                    cum += ucost[u];
+                    const int left_units = (bi + 1) * BR - (u + 1), left_tiles = per_row - t;
+                    const bool full = u + 1 - cut.back() >= kMaxTileUnits;
+                    if (cum >= rtot * t / per_row || left_units <= left_tiles || full) { cut.push_back(u + 1); ++t; }
+                }
+                cut.push_back((bi + 1) * BR);
+            }
+            ncta[l] = (int)cut.size() - 1;
+        } else {
+            cut.assign(ncta[l] + 1, H);
+            cut[0] = 0;
+            double cum = 0;
+            int t = 1;
+            for (int u = 0; u < H && t < ncta[l]; ++u) {
+                cum += ucost[u];
+                const int left_units = H - (u + 1), left_tiles = ncta[l] - t;
+                const bool full = u + 1 - cut[t - 1] >= kMaxTileUnits;
+                if (cum >= tot * t / ncta[l] || left_units <= left_tiles || full) cut[t++] = u + 1;
+            }
         }
         for (int c = 0; c < ncta[l]; ++c) {
             const int U = cut[c + 1] - cut[c];
