@@ -35,7 +35,7 @@ struct RnnArgs {
     int T, B, H, L, gates, stage_bytes, stages, resident, max_warp_bytes, max_U, max_C;
     int v_bulk;                // batch 1: [u_t ; h_{t-1}] may come in by bulk copy (16-byte aligned pieces)
 #ifdef CSB_PHASE_CLOCKS
-    long long* clocks;         // [n_ctas][4] cycles summed over ticks: stage, walk, gates, barrier
+    long long* clocks;         // [n_ctas][5] cycles summed over ticks: stage, walk, reduce, gates, barrier
 #endif
 };
 
@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     const float* bias = a.bias[layer];
     const int n_ticks = a.T + a.L - 1;
 #ifdef CSB_PHASE_CLOCKS
-    long long rprof[4] = {0, 0, 0, 0};
+    long long rprof[5] = {0, 0, 0, 0, 0};
     long long rt = clock64();
 #endif
     for (int tick = 0; tick < n_ticks; ++tick) {
@@ -274,13 +274,22 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                     for (int idx = threadIdx.x; idx < span; idx += blockDim.x) {
                         const int e = idx / parts, pt = idx % parts;
                         float sum = 0.f;
-                        if (e < NZ)
-                            for (int c = pt; c < NC; c += parts) sum += zs_all[c * S.zs_stride + e];
+                        if (e < NZ) {
+                            const float* src = zs_all + e;
+                            for (int c = pt; c < NC; c += 8 * parts) {       // eight loads in flight, added in order
+                                float v[8];
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) v[j] = (c + j * parts < NC) ? src[(c + j * parts) * S.zs_stride] : 0.f;
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) sum += v[j];
+                            }
+                        }
                         for (int off = parts >> 1; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
                         if (e < NZ && pt == 0) zsum[e] = sum;
                     }
                 }
                 __syncthreads();
+                RNN_LAP(2);
                 for (int i = threadIdx.x; i < U * nb; i += blockDim.x) {
                     const int bt = i / U, u = i % U, b = b0 + bt;
                     float z[4];
@@ -311,17 +320,17 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                     if (layer == a.L - 1 && a.y) a.y[((size_t)t * B + b) * H + u0 + u] = h;
                 }
                 __syncthreads();
-                RNN_LAP(2);
+                RNN_LAP(3);
             }
         }
         if (tick + 1 < n_ticks) {
             if (!grid_barrier(a, (unsigned)(tick + 1) * (gridDim.x + a.barrier_extra), s_flag)) break;
         }
-        RNN_LAP(3);
+        RNN_LAP(4);
     }
     if (!alive && lane == 0) *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout;
 #ifdef CSB_PHASE_CLOCKS
-    if (threadIdx.x == 0) for (int i = 0; i < 4; ++i) a.clocks[(size_t)blockIdx.x * 4 + i] = rprof[i];
+    if (threadIdx.x == 0) for (int i = 0; i < 5; ++i) a.clocks[(size_t)blockIdx.x * 5 + i] = rprof[i];
 #endif
 }
 
@@ -407,16 +416,21 @@ static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, i
     bool fits = false;
     for (int wtry : {first, 12, 8, 6, 4, 2, 1}) {
         if (wtry > first) continue;
-        Hp = RnnHostPlan();
-        rc = plan_rnn_host(gates, L, W, in_size, H, want, wtry, P->stage_bytes, &Hp);
-        if (rc != CSB_OK) return rc;
-        P->warps = wtry;
-        P->max_U = Hp.max_U; P->max_warp_bytes = (int)Hp.max_warp_bytes; P->GW = Hp.stream.group_width;
-        const int G = 32 / P->GW;
-        const RnnSmem res(wtry, G, P->stages, P->stage_bytes, 1, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
-        const RnnSmem str(wtry, G, P->stages, P->stage_bytes, 0, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
-        if (res.total <= A0->smem_optin && !env_int("CSB_RNN_STREAM", 0)) { P->resident = 1; P->smem = res.total; fits = true; break; }
-        if (str.total <= A0->smem_optin) { P->resident = 0; P->smem = str.total; fits = true; break; }
+        // first with one chunk per warp (weights resident, no ring to fit the chunks into), then
+        // with ring-sized chunks for streaming
+        for (int pass = 0; pass < 2 && !fits; ++pass) {
+            if (pass == 0 && env_int("CSB_RNN_STREAM", 0)) continue;
+            const int chunk_bytes = pass == 0 ? (256 << 10) : P->stage_bytes;
+            Hp = RnnHostPlan();
+            rc = plan_rnn_host(gates, L, W, in_size, H, want, wtry, chunk_bytes, &Hp);
+            if (rc != CSB_OK) return rc;
+            P->warps = wtry;
+            P->max_U = Hp.max_U; P->max_warp_bytes = (int)Hp.max_warp_bytes; P->GW = Hp.stream.group_width;
+            const int G = 32 / P->GW;
+            const RnnSmem sm(wtry, G, P->stages, P->stage_bytes, pass == 0, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
+            if (sm.total <= A0->smem_optin) { P->resident = pass == 0; P->smem = sm.total; fits = true; }
+        }
+        if (fits) break;
     }
     if (!fits) { set_error("time-loop kernel does not fit the %zu bytes of shared memory per CTA", A0->smem_optin); return CSB_ERR_LAUNCH; }
     P->n_ctas = (int)Hp.ctas.size();
@@ -467,7 +481,7 @@ static int dispatch_rnn_gw(const RnnPlan* P, RnnArgs& a, cudaStream_t st) {
 static long long* g_rnn_clocks = nullptr;
 static int g_rnn_clock_ctas = 0;
 extern "C" int csb_debug_rnn_clocks(long long* host_out, int max_ctas) {
-    cudaMemcpy(host_out, g_rnn_clocks, (size_t)std::min(max_ctas, g_rnn_clock_ctas) * 4 * 8, cudaMemcpyDeviceToHost);
+    cudaMemcpy(host_out, g_rnn_clocks, (size_t)std::min(max_ctas, g_rnn_clock_ctas) * 5 * 8, cudaMemcpyDeviceToHost);
     return g_rnn_clock_ctas;
 }
 #endif

@@ -210,16 +210,20 @@ int plan_rnn_host(int gates, int n_layers, const csb_matrix* const* Wm, const in
             const int u0 = cuts[l][c], u1 = cuts[l][c + 1];
             std::vector<ItemSpec> items;
             tile_items(l, u0, u1, gw, &items, nullptr);
-            // warps of this CTA: contiguous runs of about equal cost
+            // warps of this CTA: items dealt longest first to the least loaded warp (any warp may
+            // take any item: accumulators are private and added in a fixed order afterwards)
             std::vector<std::vector<Segment>> per_warp(warps, std::vector<Segment>(1));
             double total = 0;
             std::vector<double> cost(items.size());
             for (size_t i = 0; i < items.size(); ++i) { cost[i] = (double)item_steps(A, items[i], gw); total += cost[i]; }
-            double cum = 0;
-            for (size_t i = 0; i < items.size(); ++i) {
-                const int w = total > 0 ? (int)((cum + 0.5 * cost[i]) / (total / warps)) : 0;
-                per_warp[std::min(std::max(w, 0), warps - 1)][0].items.push_back(items[i]);
-                cum += cost[i];
+            std::vector<size_t> order(items.size());
+            for (size_t i = 0; i < order.size(); ++i) order[i] = i;
+            std::stable_sort(order.begin(), order.end(), [&](size_t x, size_t y) { return cost[x] > cost[y]; });
+            std::vector<double> load(warps, 0.0);
+            for (size_t i : order) {
+                const int w = (int)(std::min_element(load.begin(), load.end()) - load.begin());
+                per_warp[w][0].items.push_back(items[i]);
+                load[w] += cost[i];
             }
             RnnCtaDesc d{l, u0, u1 - u0, (uint32_t)out->stream.n_warps};
             build_stream(A, per_warp, stage_bytes, &out->stream);
