@@ -285,7 +285,15 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                             }
                         }
                         for (int off = parts >> 1; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-                        if (e < NZ && pt == 0) zsum[e] = sum;
+                        // the lane that holds the total applies bias and the gate's own activation
+                        // right away, so the activations of one unit run in parallel
+                        if (e < NZ && pt == 0) {
+                            const int g = e / (U * BT), u = (e / BT) % U;
+                            float z = sum + (bias ? __ldg(bias + g * H + u0 + u) : 0.f);
+                            if (a.gates == 4) z = g == 2 ? tanhf(z) : sigmoidf_acc(z);      // i, f, o: logistic; g: tanh
+                            else if (g < 2) z = sigmoidf_acc(z);                            // r, z; the candidate's two parts stay raw
+                            zsum[e] = z;
+                        }
                     }
                 }
                 __syncthreads();
@@ -297,24 +305,15 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                     for (int g = 0; g < 4; ++g) z[g] = zsum[(g * U + u) * BT + bt];
                     float h;
                     if (a.gates == 4) {
-                        if (bias) {
-#pragma unroll
-                            for (int g = 0; g < 4; ++g) z[g] += __ldg(bias + g * H + u0 + u);
-                        }
-                        const float c = sigmoidf_acc(z[1]) * cs[b * a.max_U + u] + sigmoidf_acc(z[0]) * tanhf(z[2]);
+                        const float c = z[1] * cs[b * a.max_U + u] + z[0] * z[2];
                         cs[b * a.max_U + u] = c;
-                        h = sigmoidf_acc(z[3]) * tanhf(c);
+                        h = z[3] * tanhf(c);
                         if (t == a.T - 1) a.cstate[((size_t)layer * B + b) * H + u0 + u] = c;
                     } else {
-                        float br = 0.f, bz = 0.f, bin = 0.f, bhn = 0.f;
-                        if (bias) {
-                            br = __ldg(bias + u0 + u); bz = __ldg(bias + H + u0 + u);
-                            bin = __ldg(bias + 2 * H + u0 + u); bhn = __ldg(bias + 3 * H + u0 + u);
-                        }
-                        const float r = sigmoidf_acc(z[0] + br), zg = sigmoidf_acc(z[1] + bz);
-                        const float n = tanhf(z[2] + bin + r * (z[3] + bhn));
+                        // slots: r, z, candidate input part (+ b_in), candidate hidden part (+ b_hn)
+                        const float n = tanhf(z[2] + z[0] * z[3]);
                         const float hp = __ldcg(rec_src + (size_t)b * H + u0 + u);
-                        h = (1.f - zg) * n + zg * hp;
+                        h = (1.f - z[1]) * n + z[1] * hp;
                     }
                     h_dst[(size_t)b * H + u0 + u] = h;
                     if (layer == a.L - 1 && a.y) a.y[((size_t)t * B + b) * H + u0 + u] = h;
