@@ -173,6 +173,7 @@ enum { kMaxTileUnits = 64, kMaxLayers = 8 };
 struct RnnHostPlan {
     StreamPlan stream;                 // stream.group_width is chosen by the planner
     std::vector<RnnCtaDesc> ctas;
+    std::vector<uint32_t> warp_in_chunks;   // per warp: chunks of input-column items (laid out first)
     int warps = 0, max_U = 0;
     size_t max_warp_bytes = 0;
     double balance = 1.0;

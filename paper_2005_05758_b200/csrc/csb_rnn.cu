@@ -21,6 +21,7 @@ struct RnnArgs {
     const uint8_t* stream;
     const Chunk* chunks;
     const uint32_t* warp_chunk_begin;
+    const uint32_t* warp_in_chunks;   // per warp: how many of its chunks hold input-column items (they come first)
     const RnnCtaDesc* ctas;
     const float* x;            // [T, B, I0]
     float* y;                  // [T, B, H] or null
@@ -60,7 +61,7 @@ struct RnnSmem {
         cs = (v + (BT == 1 ? (size_t)max_C * 4 : 0) + 15) & ~(size_t)15;
         zsum = (cs + (size_t)max_U * B * 4 + 15) & ~(size_t)15;
         vbar = (zsum + (size_t)4 * max_U * BT * 4 + 15) & ~(size_t)15;
-        flag = vbar + 16;
+        flag = vbar + 16;                              // two mbarriers: input half, recurrent half
         total = flag + 16;
     }
 };
@@ -71,13 +72,19 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
     return v;
 }
 
-// All CTAs arrive, then wait until `target` arrivals are visible.  The wait is bounded in
-// wall-clock time; on expiry the status word is raised and every thread gets `false`.
-__device__ __forceinline__ bool grid_barrier(const RnnArgs& a, unsigned int target, volatile int* s_flag) {
+// Grid barrier in two halves, so that work that does not need the other CTAs' results can sit
+// between them.  arrive: every thread's stores are ordered before one release-increment.
+// wait: one thread polls until `target` arrivals are visible; the wait is bounded in wall-clock
+// time, on expiry the status word is raised and every thread gets `false`.
+__device__ __forceinline__ void grid_arrive(const RnnArgs& a) {
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
         atomicAdd(a.barrier, 1u);
+    }
+}
+__device__ __forceinline__ bool grid_wait(const RnnArgs& a, unsigned int target, volatile int* s_flag) {
+    if (threadIdx.x == 0) {
         bool ok = true;
         unsigned long long t0 = 0;
         unsigned int spins = 0;
@@ -97,6 +104,16 @@ __device__ __forceinline__ bool grid_barrier(const RnnArgs& a, unsigned int targ
 
 __device__ __forceinline__ float sigmoidf_acc(float a) { return 1.f / (1.f + expf(-a)); }
 
+// Time loop.  Tick k: layer l works on step t = k - lag*l (lag = 2 above the first layer).  Inside
+// a tick a CTA
+//   1. waits for the previous tick's barrier (h_{t-1} of its own layer is then visible),
+//   2. stages h_{t-1}, walks the items that multiply it (the input half of the product was done
+//      before the wait), adds up the accumulators, does the gate arithmetic, writes h_t,
+//   3. arrives at this tick's barrier,
+//   4. and, while the others arrive, stages u_{t+1} and walks the input-half items of the NEXT
+//      step (batch 1 only).  With lag 2 the layer below produced u_{t+1} a full tick ago, so that
+//      needs nothing from the barrier it has just arrived at.
+// h of step s of a layer lives in slot s & 3 of a four-slot ring in global memory.
 template <typename T, int BT, int GW>
 __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -105,7 +122,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     const RnnSmem S(W, G, a.stages, a.stage_bytes, a.resident, a.max_warp_bytes, a.max_U, BT, a.B, a.max_C);
     const RnnCtaDesc me = a.ctas[blockIdx.x];
     const int layer = me.layer, U = me.U, u0 = me.u0, H = a.H, B = a.B;
-    const int I = a.in_size[layer], C = I + H;
+    const int I = a.in_size[layer];
     const size_t per_warp = a.resident ? (size_t)a.max_warp_bytes : (size_t)a.stages * a.stage_bytes;
     uint8_t* wbuf = smem + S.weights + warp * per_warp;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S.bars) + warp * (a.resident ? 1 : a.stages);
@@ -116,13 +133,14 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     float* cs = reinterpret_cast<float*>(smem + S.cs);
     volatile int* s_flag = reinterpret_cast<volatile int*>(smem + S.flag);
     float* zsum = reinterpret_cast<float*>(smem + S.zsum);
-    uint64_t* vbar = reinterpret_cast<uint64_t*>(smem + S.vbar);
-    uint32_t v_uses = 0;
+    uint64_t* vbar = reinterpret_cast<uint64_t*>(smem + S.vbar);       // [0] input half, [1] recurrent half
+    uint32_t v_uses[2] = {0, 0};
 
     const uint32_t c0 = a.warp_chunk_begin[me.warp0 + warp], c1 = a.warp_chunk_begin[me.warp0 + warp + 1];
     const uint32_t nchunks = c1 - c0;
+    const uint32_t n_in = a.warp_in_chunks[me.warp0 + warp];        // chunks of the input half come first
     const uint8_t* wsrc = a.stream + (size_t)(nchunks ? a.chunks[c0].off16 : 0) * 16;
-    uint32_t wbytes = 0;
+    uint32_t wbytes = 0, rec_off = 0;
     bool alive = true;
 
     // ---- weights: load once (resident) or prime the ring (streaming) ----
@@ -130,7 +148,11 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     unsigned long long n_done = 0;
     const unsigned long long n_total = (unsigned long long)a.T * ((B + BT - 1) / BT) * nchunks;
     if (a.resident) {
-        for (uint32_t c = c0; c < c1; ++c) wbytes += a.chunks[c].bytes;   // chunks of a warp are contiguous
+        for (uint32_t c = c0; c < c1; ++c) {                               // chunks of a warp are contiguous
+            if (c - c0 == n_in) rec_off = wbytes;
+            wbytes += a.chunks[c].bytes;
+        }
+        if (n_in == nchunks) rec_off = wbytes;
         if (lane == 0) {
             mbar_init(&bars[0], 1);
             mbar_fence_init();
@@ -162,105 +184,136 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     }
     if (threadIdx.x == 0) {
         *s_flag = 1;
-        mbar_init(vbar, 1);
+        mbar_init(&vbar[0], 1);
+        mbar_init(&vbar[1], 1);
         mbar_fence_init();
     }
     __syncthreads();
 
     const float* bias = a.bias[layer];
-    const int n_ticks = a.T + a.L - 1;
+    const int lag = a.L > 1 ? 2 : 1;
+    const int n_ticks = a.T + lag * (a.L - 1);
+    const size_t slot_sz = (size_t)B * H;
+    auto h_slot = [&](int l, int step) { return a.hbuf + ((size_t)l * 4 + (step & 3)) * slot_sz; };
+    auto input_of = [&](int step) -> const float* { return layer == 0 ? a.x + (size_t)step * B * I : h_slot(layer - 1, step); };
+    const int in_ld = layer == 0 ? I : H;
 #ifdef CSB_PHASE_CLOCKS
     long long rprof[5] = {0, 0, 0, 0, 0};
     long long rt = clock64();
 #endif
-    for (int tick = 0; tick < n_ticks; ++tick) {
-        const int t = tick - layer;
-        const bool active = t >= 0 && t < a.T;
-        if (active) {
-            const float* in_src = layer == 0 ? a.x + (size_t)t * B * I
-                                             : a.hbuf + ((size_t)(layer - 1) * 2 + (t & 1)) * B * H;
-            const float* rec_src = a.hbuf + ((size_t)layer * 2 + ((t + 1) & 1)) * B * H;   // slot of step t-1
-            float* h_dst = a.hbuf + ((size_t)layer * 2 + (t & 1)) * B * H;
-            const int in_ld = layer == 0 ? I : H;
+
+    // One half of [u ; h] into shared memory (batch 1; half 0 = input, 1 = recurrent).  With bulk
+    // copies the issue and the wait are separate, so a copy can be in flight while other work
+    // runs; without them stage_wait does the loads.
+    auto stage_issue = [&](int half, float* dst, const float* src, int n) {
+        if (a.v_bulk && threadIdx.x == 0) {
+            fence_proxy_async_all();          // src may have been written with ordinary stores by other CTAs
+            mbar_expect_tx(&vbar[half], (uint32_t)n * 4u);
+            bulk_g2s(dst, src, (uint32_t)n * 4u, &vbar[half]);
+        }
+    };
+    auto stage_wait = [&](int half, float* dst, const float* src, int n) {
+        if (a.v_bulk) {
+            if (!mbar_wait_bounded(&vbar[half], v_uses[half] & 1u)) alive = false;
+            ++v_uses[half];
+        } else {
+#pragma unroll 4
+            for (int i = threadIdx.x; i < n; i += blockDim.x) dst[i] = __ldcg(src + i);
+            __syncthreads();
+        }
+    };
+    // walk this warp's chunks of one half (part 0: input columns, part 1: recurrent columns)
+    auto walk_part = [&](int part, const float* in_src, const float* rec_src, int b0, int nb) {
+        auto gather = [&](uint32_t xbase, uint32_t c4, uint32_t flags, int left, float* dst) {
+            const bool rec = (flags & kItemRecurrent) != 0;
             if (BT == 1) {
-                if (a.v_bulk) {
-                    // two bulk copies bring [u_t ; h_{t-1}] in; h was written by other CTAs with
-                    // ordinary stores before the grid barrier, so the copy is ordered behind this
-                    // thread's (acquired) view with a proxy fence
-                    if (threadIdx.x == 0) {
-                        fence_proxy_async_all();
-                        mbar_expect_tx(vbar, (uint32_t)C * 4u);
-                        bulk_g2s(vs, in_src, (uint32_t)I * 4u, vbar);
-                        bulk_g2s(vs + I, rec_src, (uint32_t)H * 4u, vbar);
-                    }
-                    if (!mbar_wait_bounded(vbar, v_uses & 1u)) alive = false;
-                    ++v_uses;
-                } else {
-#pragma unroll 8
-                    for (int i = threadIdx.x; i < C; i += blockDim.x) vs[i] = __ldcg(i < I ? in_src + i : rec_src + (i - I));
-                    __syncthreads();
+                // padding indices are zero; xbase (+ I for the recurrent part) is the block's first
+                // column, which exists, so they may be read.  (32-bit sum: for a block that
+                // straddles the x | h boundary xbase is "negative".)
+                const uint32_t base = xbase + (rec ? (uint32_t)I : 0u);
+                float4 v;
+                v.x = vs[base + (c4 & 0xffu)]; v.y = vs[base + ((c4 >> 8) & 0xffu)];
+                v.z = vs[base + ((c4 >> 16) & 0xffu)]; v.w = vs[base + (c4 >> 24)];
+                *reinterpret_cast<float4*>(dst) = v;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t col = xbase + ((c4 >> (8 * j)) & 0xffu);
+#pragma unroll
+                    for (int bt = 0; bt < BT; ++bt)
+                        dst[j * BT + bt] = (j < left && bt < nb)
+                            ? (rec ? __ldcg(rec_src + (size_t)(b0 + bt) * H + col) : __ldcg(in_src + (size_t)(b0 + bt) * in_ld + col))
+                            : 0.f;
                 }
             }
-            RNN_LAP(0);
+        };
+        if (!alive) return;
+        if (a.resident) {
+            const uint8_t* p = wbuf + (part ? rec_off : 0u);
+            const uint8_t* end = wbuf + (part ? wbytes : rec_off);
+            while (p < end) {
+                const uint4 ch = *reinterpret_cast<const uint4*>(p);
+                walk_chunk<T, BT, GW>(p, ch, lane, xg, zs, S.zs_stride, gather);
+                p += chunk_bytes(ch);
+            }
+        } else {
+            const uint32_t cnt = part ? nchunks - n_in : n_in;
+            for (uint32_t c = 0; c < cnt; ++c) {
+                const int s = (int)(n_done % (unsigned)a.stages);
+                const uint32_t parity = (uint32_t)((n_done / (unsigned)a.stages) & 1u);
+                if (!mbar_wait_bounded(&bars[s], parity)) alive = false;
+                alive = !__any_sync(0xffffffffu, !alive);
+                if (!alive) {
+                    if (lane == 0)        // bounded drain of the copies still in flight
+                        for (unsigned long long n = n_done + 1; n < n_done + a.stages && n < n_total; ++n)
+                            mbar_wait_bounded(&bars[n % (unsigned)a.stages], (uint32_t)((n / (unsigned)a.stages) & 1u));
+                    return;
+                }
+                const uint8_t* p = wbuf + (size_t)s * a.stage_bytes;
+                const uint4 ch = *reinterpret_cast<const uint4*>(p);
+                walk_chunk<T, BT, GW>(p, ch, lane, xg, zs, S.zs_stride, gather);
+                __syncwarp();
+                ++n_done;
+                if (lane == 0 && n_done + a.stages - 1 < n_total) {
+                    const unsigned long long n = n_done + a.stages - 1;
+                    const Chunk nx = a.chunks[c0 + (uint32_t)(n % nchunks)];
+                    mbar_expect_tx(&bars[s], nx.bytes);
+                    bulk_g2s(wbuf + (size_t)s * a.stage_bytes, a.stream + (size_t)nx.off16 * 16, nx.bytes, &bars[s]);
+                }
+            }
+        }
+    };
+    auto zero_zs = [&]() {
+        for (int i = lane; i < G * S.zs_stride; i += 32) zs[i] = 0.f;
+        __syncwarp();
+    };
+
+    bool pre_done = false;        // the input half of the coming step is already in the accumulators
+    bool in_flight = false;       // the copy of the coming step's input half has been issued
+    for (int tick = 0; tick < n_ticks; ++tick) {
+        const int t = tick - lag * layer;
+        const bool active = t >= 0 && t < a.T;
+        const bool pre_next = BT == 1 && t + 1 >= 0 && t + 1 < a.T && tick + 1 < n_ticks;
+        if (tick > 0 && !grid_wait(a, (unsigned)tick * (gridDim.x + a.barrier_extra), s_flag)) break;
+        RNN_LAP(4);
+        if (active) {
+            const float* in_src = input_of(t);
+            const float* rec_src = h_slot(layer, t - 1);
+            float* h_dst = h_slot(layer, t);
             for (int b0 = 0; b0 < B; b0 += BT) {
                 const int nb = min(BT, B - b0);
-                for (int i = lane; i < G * S.zs_stride; i += 32) zs[i] = 0.f;
-                __syncwarp();
-                auto gather = [&](uint32_t xbase, uint32_t c4, uint32_t flags, int left, float* dst) {
-                    const bool rec = (flags & kItemRecurrent) != 0;
-                    if (BT == 1) {
-                        // padding indices are zero; xbase (+ I for the recurrent part) is the block's
-                        // first column, which exists, so they may be read
-                        // (32-bit sum: for a block that straddles the x | h boundary xbase is "negative")
-                        const uint32_t base = xbase + (rec ? (uint32_t)I : 0u);
-                        float4 v;
-                        v.x = vs[base + (c4 & 0xffu)]; v.y = vs[base + ((c4 >> 8) & 0xffu)];
-                        v.z = vs[base + ((c4 >> 16) & 0xffu)]; v.w = vs[base + (c4 >> 24)];
-                        *reinterpret_cast<float4*>(dst) = v;
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t col = xbase + ((c4 >> (8 * j)) & 0xffu);
-#pragma unroll
-                            for (int bt = 0; bt < BT; ++bt)
-                                dst[j * BT + bt] = (j < left && bt < nb)
-                                    ? (rec ? __ldcg(rec_src + (size_t)(b0 + bt) * H + col) : __ldcg(in_src + (size_t)(b0 + bt) * in_ld + col))
-                                    : 0.f;
-                        }
-                    }
-                };
-                if (a.resident) {
-                    if (alive)
-                        for (const uint8_t* p = wbuf; p < wbuf + wbytes;) {
-                            const uint4 ch = *reinterpret_cast<const uint4*>(p);
-                            walk_chunk<T, BT, GW>(p, ch, lane, xg, zs, S.zs_stride, gather);
-                            p += chunk_bytes(ch);
-                        }
-                } else {
-                    for (uint32_t c = 0; c < nchunks && alive; ++c) {
-                        const int s = (int)(n_done % (unsigned)a.stages);
-                        const uint32_t parity = (uint32_t)((n_done / (unsigned)a.stages) & 1u);
-                        if (!mbar_wait_bounded(&bars[s], parity)) alive = false;
-                        alive = !__any_sync(0xffffffffu, !alive);
-                        if (!alive) {
-                            if (lane == 0)        // bounded drain of the copies still in flight
-                                for (unsigned long long n = n_done + 1; n < n_done + a.stages && n < n_total; ++n)
-                                    mbar_wait_bounded(&bars[n % (unsigned)a.stages], (uint32_t)((n / (unsigned)a.stages) & 1u));
-                            break;
-                        }
-                        const uint8_t* p = wbuf + (size_t)s * a.stage_bytes;
-                        const uint4 ch = *reinterpret_cast<const uint4*>(p);
-                        walk_chunk<T, BT, GW>(p, ch, lane, xg, zs, S.zs_stride, gather);
-                        __syncwarp();
-                        ++n_done;
-                        if (lane == 0 && n_done + a.stages - 1 < n_total) {
-                            const unsigned long long n = n_done + a.stages - 1;
-                            const Chunk nx = a.chunks[c0 + (uint32_t)(n % nchunks)];
-                            mbar_expect_tx(&bars[s], nx.bytes);
-                            bulk_g2s(wbuf + (size_t)s * a.stage_bytes, a.stream + (size_t)nx.off16 * 16, nx.bytes, &bars[s]);
-                        }
-                    }
+                if (BT == 1) stage_issue(1, vs + I, rec_src, H);
+                if (!pre_done) {
+                    if (BT == 1) { stage_issue(0, vs, in_src, I); stage_wait(0, vs, in_src, I); }
+                    zero_zs();
+                    walk_part(0, in_src, rec_src, b0, nb);
+                    if (BT == 1) __syncthreads();          // every warp is done with the input half of vs
                 }
+                // the next step's input half is on its way while this step's recurrent half is walked
+                if (pre_next) { stage_issue(0, vs, input_of(t + 1), I); in_flight = true; }
+                if (BT == 1) stage_wait(1, vs + I, rec_src, H);
+                RNN_LAP(0);
+                walk_part(1, in_src, rec_src, b0, nb);
                 __syncthreads();
                 RNN_LAP(1);
                 // ---- gate arithmetic for this batch tile ----
@@ -319,13 +372,21 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                     if (layer == a.L - 1 && a.y) a.y[((size_t)t * B + b) * H + u0 + u] = h;
                 }
                 __syncthreads();
+                pre_done = false;
                 RNN_LAP(3);
             }
         }
-        if (tick + 1 < n_ticks) {
-            if (!grid_barrier(a, (unsigned)(tick + 1) * (gridDim.x + a.barrier_extra), s_flag)) break;
+        if (tick + 1 < n_ticks) grid_arrive(a);
+        // the input half of the next step, while the other CTAs arrive
+        if (pre_next) {
+            if (!in_flight) stage_issue(0, vs, input_of(t + 1), I);
+            stage_wait(0, vs, input_of(t + 1), I);
+            in_flight = false;
+            zero_zs();
+            walk_part(0, nullptr, nullptr, 0, 1);
+            pre_done = true;
         }
-        RNN_LAP(4);
+        RNN_LAP(1);
     }
     if (!alive && lane == 0) *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout;
 #ifdef CSB_PHASE_CLOCKS
@@ -353,12 +414,12 @@ struct RnnPlan {
     size_t smem = 0;
     double balance = 1.0;
     int64_t stream_bytes = 0;
-    uint8_t* d_stream = nullptr; Chunk* d_chunks = nullptr; uint32_t* d_wcb = nullptr; RnnCtaDesc* d_ctas = nullptr;
+    uint8_t* d_stream = nullptr; Chunk* d_chunks = nullptr; uint32_t* d_wcb = nullptr; uint32_t* d_win = nullptr; RnnCtaDesc* d_ctas = nullptr;
     float* d_hbuf = nullptr; float* d_cstate = nullptr; unsigned int* d_barrier = nullptr;
     uint32_t* h_status = nullptr; uint32_t* d_status = nullptr;
     float* d_stage = nullptr; size_t stage_cap = 0;      // host-I/O staging: x, y, states
     ~RnnPlan() {
-        cudaFree(d_stream); cudaFree(d_chunks); cudaFree(d_wcb); cudaFree(d_ctas); cudaFree(d_hbuf);
+        cudaFree(d_stream); cudaFree(d_chunks); cudaFree(d_wcb); cudaFree(d_win); cudaFree(d_ctas); cudaFree(d_hbuf);
         cudaFree(d_cstate); cudaFree(d_barrier); cudaFree(d_stage);
         if (h_status) cudaFreeHost(h_status);
     }
@@ -438,8 +499,9 @@ static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, i
     if ((rc = upload_vec(Hp.stream.bytes, &P->d_stream)) != CSB_OK) return rc;
     if ((rc = upload_vec(Hp.stream.chunks, &P->d_chunks)) != CSB_OK) return rc;
     if ((rc = upload_vec(Hp.stream.warp_chunk_begin, &P->d_wcb)) != CSB_OK) return rc;
+    if ((rc = upload_vec(Hp.warp_in_chunks, &P->d_win)) != CSB_OK) return rc;
     if ((rc = upload_vec(Hp.ctas, &P->d_ctas)) != CSB_OK) return rc;
-    CSB_CUDA(cudaMalloc((void**)&P->d_hbuf, (size_t)L * 2 * B * H * 4));
+    CSB_CUDA(cudaMalloc((void**)&P->d_hbuf, (size_t)L * 4 * B * H * 4));
     CSB_CUDA(cudaMalloc((void**)&P->d_cstate, (size_t)L * B * H * 4));
     CSB_CUDA(cudaMalloc((void**)&P->d_barrier, 4));
     CSB_CUDA(cudaHostAlloc((void**)&P->h_status, 4, cudaHostAllocMapped));
@@ -555,9 +617,9 @@ static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const flo
     const cudaMemcpyKind in_kind = host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
     const cudaMemcpyKind out_kind = host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice;
     const size_t row = (size_t)B * H * 4;
-    // h0 goes to slot 1 of every layer (the slot of "step -1"), c0 to the cell-state buffer
-    if (h0) CSB_CUDA(cudaMemcpy2DAsync(P->d_hbuf + (size_t)B * H, 2 * row, h0, row, row, L, in_kind, st));
-    else CSB_CUDA(cudaMemsetAsync(P->d_hbuf, 0, 2 * row * L, st));
+    // h0 goes to slot 3 of every layer's four-slot ring (the slot of "step -1"), c0 to the cell-state buffer
+    if (h0) CSB_CUDA(cudaMemcpy2DAsync(P->d_hbuf + 3 * (size_t)B * H, 4 * row, h0, row, row, L, in_kind, st));
+    else CSB_CUDA(cudaMemsetAsync(P->d_hbuf, 0, 4 * row * L, st));
     if (gates == 4) {
         if (c0) CSB_CUDA(cudaMemcpyAsync(P->d_cstate, c0, ns * 4, in_kind, st));
         else CSB_CUDA(cudaMemsetAsync(P->d_cstate, 0, ns * 4, st));
@@ -566,7 +628,7 @@ static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const flo
     *P->h_status = 0;
 
     RnnArgs a{};
-    a.stream = P->d_stream; a.chunks = P->d_chunks; a.warp_chunk_begin = P->d_wcb; a.ctas = P->d_ctas;
+    a.stream = P->d_stream; a.chunks = P->d_chunks; a.warp_chunk_begin = P->d_wcb; a.warp_in_chunks = P->d_win; a.ctas = P->d_ctas;
     a.x = dx; a.y = dy; a.hbuf = P->d_hbuf; a.cstate = P->d_cstate;
     for (int l = 0; l < L; ++l) { a.bias[l] = bias ? bias[l] : nullptr; a.in_size[l] = in_size[l]; }
     a.barrier = P->d_barrier; a.status = P->d_status; a.barrier_ns = g_barrier_ns; a.barrier_extra = g_barrier_extra;
@@ -591,8 +653,8 @@ static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const flo
     else if (P->BT == 4) rc = half ? dispatch_rnn_gw<__half, 4>(P, a, st) : dispatch_rnn_gw<float, 4>(P, a, st);
     else rc = half ? dispatch_rnn_gw<__half, 8>(P, a, st) : dispatch_rnn_gw<float, 8>(P, a, st);
     if (rc != CSB_OK) return rc;
-    const int last_slot = (int)((T - 1) & 1);
-    if (hT) CSB_CUDA(cudaMemcpy2DAsync(hT, row, P->d_hbuf + (size_t)last_slot * B * H, 2 * row, row, L, out_kind, st));
+    const int last_slot = (int)((T - 1) & 3);
+    if (hT) CSB_CUDA(cudaMemcpy2DAsync(hT, row, P->d_hbuf + (size_t)last_slot * B * H, 4 * row, row, L, out_kind, st));
     if (cT && gates == 4) CSB_CUDA(cudaMemcpyAsync(cT, P->d_cstate, ns * 4, out_kind, st));
     if (host_io && y) CSB_CUDA(cudaMemcpyAsync(y, dy, ny * 4, cudaMemcpyDeviceToHost, st));
     if (host_io || !(flags & CSB_FLAG_ASYNC)) {

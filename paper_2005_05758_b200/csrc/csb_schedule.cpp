@@ -211,23 +211,45 @@ int plan_rnn_host(int gates, int n_layers, const csb_matrix* const* Wm, const in
             std::vector<ItemSpec> items;
             tile_items(l, u0, u1, gw, &items, nullptr);
             // warps of this CTA: items dealt longest first to the least loaded warp (any warp may
-            // take any item: accumulators are private and added in a fixed order afterwards)
-            std::vector<std::vector<Segment>> per_warp(warps, std::vector<Segment>(1));
+            // take any item: accumulators are private and added in a fixed order afterwards).
+            // Input-column items and recurrent-column items are dealt separately and laid out as
+            // two segments per warp, input first: the kernel walks them at different times.
+            std::vector<std::vector<Segment>> per_warp(warps, std::vector<Segment>(2));
+            for (int w = 0; w < warps; ++w) per_warp[w][1].zbase = 1;       // chunk tag: 0 input, 1 recurrent
             double total = 0;
             std::vector<double> cost(items.size());
             for (size_t i = 0; i < items.size(); ++i) { cost[i] = (double)item_steps(A, items[i], gw); total += cost[i]; }
-            std::vector<size_t> order(items.size());
-            for (size_t i = 0; i < order.size(); ++i) order[i] = i;
-            std::stable_sort(order.begin(), order.end(), [&](size_t x, size_t y) { return cost[x] > cost[y]; });
-            std::vector<double> load(warps, 0.0);
-            for (size_t i : order) {
-                const int w = (int)(std::min_element(load.begin(), load.end()) - load.begin());
-                per_warp[w][0].items.push_back(items[i]);
-                load[w] += cost[i];
+            for (int part = 0; part < 2; ++part) {
+                std::vector<size_t> order;
+                for (size_t i = 0; i < items.size(); ++i)
+                    if (((items[i].flags & kItemRecurrent) != 0) == (part == 1)) order.push_back(i);
+                std::stable_sort(order.begin(), order.end(), [&](size_t x, size_t y) { return cost[x] > cost[y]; });
+                // bins are lane groups (G per warp): equal item counts per group matter as much as
+                // equal cost, because the groups of a warp advance in lock-step rounds
+                const int G = 32 / gw;
+                std::vector<double> load((size_t)warps * G, 0.0);
+                for (size_t i : order) {
+                    const int bin = (int)(std::min_element(load.begin(), load.end()) - load.begin());
+                    per_warp[bin / G][part].items.push_back(items[i]);
+                    load[bin] += cost[i];
+                }
             }
+            const size_t first_chunk = out->stream.chunks.size();
             RnnCtaDesc d{l, u0, u1 - u0, (uint32_t)out->stream.n_warps};
             build_stream(A, per_warp, stage_bytes, &out->stream);
             out->ctas.push_back(d);
+            // how many chunks of each warp carry the input tag
+            for (int w = 0; w < warps; ++w) {
+                uint32_t n_in = 0;
+                const uint32_t cb = out->stream.warp_chunk_begin[d.warp0 + w], ce = out->stream.warp_chunk_begin[d.warp0 + w + 1];
+                for (uint32_t c = cb; c < ce; ++c) {
+                    ChunkHeader h;
+                    std::memcpy(&h, out->stream.bytes.data() + (size_t)out->stream.chunks[c].off16 * 16, sizeof h);
+                    if (h.zbase == 0) ++n_in;
+                }
+                out->warp_in_chunks.push_back(n_in);
+            }
+            (void)first_chunk;
             cost_sum += total;
             cost_max = std::max(cost_max, total);
         }
