@@ -114,18 +114,18 @@ __device__ __forceinline__ float sigmoidf_acc(float a) { return 1.f / (1.f + exp
 //      step (batch 1 only).  With lag 2 the layer below produced u_{t+1} a full tick ago, so that
 //      needs nothing from the barrier it has just arrived at.
 // h of step s of a layer lives in slot s & 3 of a four-slot ring in global memory.
-template <typename T, int BT, int GW>
+template <typename T, int BT, int GW, bool RES>
 __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int G = 32 / GW;
     const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const RnnSmem S(W, G, a.stages, a.stage_bytes, a.resident, a.max_warp_bytes, a.max_U, BT, a.B, a.max_C);
+    const RnnSmem S(W, G, a.stages, a.stage_bytes, RES, a.max_warp_bytes, a.max_U, BT, a.B, a.max_C);
     const RnnCtaDesc me = a.ctas[blockIdx.x];
     const int layer = me.layer, U = me.U, u0 = me.u0, H = a.H, B = a.B;
     const int I = a.in_size[layer];
-    const size_t per_warp = a.resident ? (size_t)a.max_warp_bytes : (size_t)a.stages * a.stage_bytes;
+    const size_t per_warp = RES ? (size_t)a.max_warp_bytes : (size_t)a.stages * a.stage_bytes;
     uint8_t* wbuf = smem + S.weights + warp * per_warp;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S.bars) + warp * (a.resident ? 1 : a.stages);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S.bars) + warp * (RES ? 1 : a.stages);
     float* zs_all = reinterpret_cast<float*>(smem + S.zs);
     float* zs = zs_all + warp * G * S.zs_stride;
     float* xg = reinterpret_cast<float*>(smem + S.xg) + warp * G * xg_stride(GW, BT);
@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     // streaming: every step walks the ring once per batch tile; chunk sequence numbers keep counting
     unsigned long long n_done = 0;
     const unsigned long long n_total = (unsigned long long)a.T * ((B + BT - 1) / BT) * nchunks;
-    if (a.resident) {
+    if (RES) {
         for (uint32_t c = c0; c < c1; ++c) {                               // chunks of a warp are contiguous
             if (c - c0 == n_in) rec_off = wbytes;
             wbytes += a.chunks[c].bytes;
@@ -248,7 +248,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
             }
         };
         if (!alive) return;
-        if (a.resident) {
+        if (RES) {
             const uint8_t* p = wbuf + (part ? rec_off : 0u);
             const uint8_t* end = wbuf + (part ? wbytes : rec_off);
             while (p < end) {
@@ -510,11 +510,11 @@ static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, i
     return CSB_OK;
 }
 
-template <typename T, int BT, int GW>
+template <typename T, int BT, int GW, bool RES>
 static int launch_rnn(const RnnPlan* P, RnnArgs& a, cudaStream_t st) {
-    CSB_CUDA(cudaFuncSetAttribute(csb_rnn_kernel<T, BT, GW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem));
+    CSB_CUDA(cudaFuncSetAttribute(csb_rnn_kernel<T, BT, GW, RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem));
     int occ = 0;
-    CSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, csb_rnn_kernel<T, BT, GW>, P->warps * 32, P->smem));
+    CSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, csb_rnn_kernel<T, BT, GW, RES>, P->warps * 32, P->smem));
     int sms = 0;
     CSB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, P->device));
     if (occ < 1 || P->n_ctas > occ * sms) {
@@ -522,7 +522,7 @@ static int launch_rnn(const RnnPlan* P, RnnArgs& a, cudaStream_t st) {
         return CSB_ERR_LAUNCH;
     }
     void* params[] = {(void*)&a};
-    const cudaError_t e = cudaLaunchCooperativeKernel((const void*)csb_rnn_kernel<T, BT, GW>, dim3(P->n_ctas), dim3(P->warps * 32),
+    const cudaError_t e = cudaLaunchCooperativeKernel((const void*)csb_rnn_kernel<T, BT, GW, RES>, dim3(P->n_ctas), dim3(P->warps * 32),
                                                       params, P->smem, st);
     if (e == cudaErrorCooperativeLaunchTooLarge) { set_error("cooperative launch too large"); return CSB_ERR_LAUNCH; }
     CSB_CUDA(e);
@@ -532,9 +532,9 @@ static int launch_rnn(const RnnPlan* P, RnnArgs& a, cudaStream_t st) {
 template <typename T, int BT>
 static int dispatch_rnn_gw(const RnnPlan* P, RnnArgs& a, cudaStream_t st) {
     switch (P->GW) {
-        case 8: return launch_rnn<T, BT, 8>(P, a, st);
-        case 16: return launch_rnn<T, BT, 16>(P, a, st);
-        default: return launch_rnn<T, BT, 32>(P, a, st);
+        case 8: return P->resident ? launch_rnn<T, BT, 8, true>(P, a, st) : launch_rnn<T, BT, 8, false>(P, a, st);
+        case 16: return P->resident ? launch_rnn<T, BT, 16, true>(P, a, st) : launch_rnn<T, BT, 16, false>(P, a, st);
+        default: return P->resident ? launch_rnn<T, BT, 32, true>(P, a, st) : launch_rnn<T, BT, 32, false>(P, a, st);
     }
 }
 
