@@ -96,10 +96,13 @@ __device__ __forceinline__ uint32_t chunk_bytes(const uint4& ch) {
 // group g walks sub-stream g, so G items are in flight and share every instruction.
 //
 // Lane mapping inside a group, per item: a word is kRows consecutive kept rows of one kept
-// column; the kernel matrix is stored column-major in words, RL words per column.  The group is
-// cut into S = GW / RL sub-groups; sub-group kg takes columns kg, kg + S, ...; lane rl of a
-// sub-group owns word rl of each column, i.e. the same output rows for the whole item.  The
-// A = S * RL active lanes read words s*A .. s*A + A-1 in step s: consecutive, conflict-free.
+// column, RL words per column.  Columns are taken four at a time: a quad-word holds the words
+// of one row pair for columns 4q .. 4q+3 (16 bytes), quad-column q has RL quad-words, and the
+// nk % 4 columns left over follow as plain words, column-major.  The group is cut into
+// S = GW / RL sub-groups; sub-group kg takes quad-columns kg, kg + S, ... (and tail columns
+// kg, kg + S, ...); lane rl of a sub-group owns row word rl, i.e. the same output rows for the
+// whole item.  The A = S * RL active lanes read quad-words s*A .. s*A + A-1 in step s:
+// consecutive 16-byte pieces, conflict-free.
 //
 // Per item: gather the kept inputs through the column indices (gather4(xbase, c4, flags, left,
 // dst) resolves four packed indices, `left` of them real, and writes dst[j * BT + bt]) into xg, multiply, fold the sub-groups, and add into
@@ -137,12 +140,15 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
         if (p < end) h = *reinterpret_cast<const uint4*>(p);
         const int nk = (int)(h.x & 0xffu), mr = (int)((h.x >> 8) & 0xffu), RL = (int)((h.x >> 16) & 0xffu), S = (int)(h.x >> 24);
         const uint32_t xbase = h.y, zbase = h.z, magic = h.w & 0xffffu, flags = h.w >> 16;
-        const uint8_t* cidx = p + 16;
+        // item = header | quads | tail words | col_idx | row_idx: the values come first so that
+        // the 16-byte quads are aligned
+        const int nwords = nk * RL, nq = (nk >> 2) * RL;                  // all words; quad-words (4 words each)
+        const uint4* quads = reinterpret_cast<const uint4*>(p + 16);
+        const uint32_t* tailw = reinterpret_cast<const uint32_t*>(p + 16) + 4 * nq;
+        const uint8_t* cidx = p + 16 + nwords * 4;
         const int cidx_bytes = (nk + 3) & ~3, ridx_bytes = (mr + 3) & ~3;
         const uint8_t* ridx = cidx + cidx_bytes;
-        const uint32_t* vals = reinterpret_cast<const uint32_t*>(ridx + ridx_bytes);
-        const int nwords = nk * RL;
-        if (p < end) p += (16 + cidx_bytes + ridx_bytes + nwords * 4 + 15) & ~15;     // items are 16-byte aligned
+        if (p < end) p += (16 + nwords * 4 + cidx_bytes + ridx_bytes + 15) & ~15;     // items are 16-byte aligned
         CSB_WALK_LAP(0);
 
         // ---- gather: each lane resolves four column indices at a time; indices past nk are
@@ -161,34 +167,48 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
 #pragma unroll
             for (int bt = 0; bt < BT; ++bt) acc[q][bt] = 0.f;
         if (gl < A) {
-            const uint32_t* vp = vals + gl;
-            const uint32_t* vend = vals + nwords;
-            const float* xp = xg + kg * BT;
-            const int xs = S * BT;
-            for (; vp + 3 * A < vend; vp += 4 * A, xp += 4 * xs) {
-                uint32_t w[4];
+            // four columns at a time: lane gl reads quad-words gl, gl + A, ... (16 bytes each,
+            // consecutive lanes consecutive quad-words) and the four inputs of those columns
+            const uint4* qp = quads + gl;
+            const uint4* qend = quads + nq;
+            const float* xp = xg + 4 * kg * BT;
+            const int xs = 4 * S * BT;
+#pragma unroll 2
+            for (; qp < qend; qp += A, xp += xs) {
+                const uint4 w = *qp;
+                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+                float xv[4][BT];
+                if (BT == 1) {
+                    const float4 x4 = *reinterpret_cast<const float4*>(xp);
+                    xv[0][0] = x4.x; xv[1][0] = x4.y; xv[2][0] = x4.z; xv[3][0] = x4.w;
+                } else {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) w[j] = vp[j * A];
+                    for (int j = 0; j < 4; ++j)
+#pragma unroll
+                        for (int bt = 0; bt < BT; ++bt) xv[j][bt] = xp[j * BT + bt];
+                }
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     float v[R];
-                    WordTraits<T>::unpack(w[j], v);
+                    WordTraits<T>::unpack(ww[j], v);
 #pragma unroll
-                    for (int bt = 0; bt < BT; ++bt) {
-                        const float xv = xp[j * xs + bt];
+                    for (int bt = 0; bt < BT; ++bt)
 #pragma unroll
-                        for (int q = 0; q < R; ++q) acc[q][bt] = fmaf(v[q], xv, acc[q][bt]);
-                    }
+                        for (int q = 0; q < R; ++q) acc[q][bt] = fmaf(v[q], xv[j][bt], acc[q][bt]);
                 }
             }
-            for (; vp < vend; vp += A, xp += xs) {
+            // the last nk % 4 columns, one word per column and lane
+            const uint32_t* vp = tailw + gl;
+            const uint32_t* vend = tailw + (nk & 3) * RL;
+            const float* xt = xg + ((nk & ~3) + kg) * BT;
+            for (; vp < vend; vp += A, xt += S * BT) {
                 float v[R];
                 WordTraits<T>::unpack(*vp, v);
 #pragma unroll
                 for (int bt = 0; bt < BT; ++bt) {
-                    const float xv = xp[bt];
+                    const float x1 = xt[bt];
 #pragma unroll
-                    for (int q = 0; q < R; ++q) acc[q][bt] = fmaf(v[q], xv, acc[q][bt]);
+                    for (int q = 0; q < R; ++q) acc[q][bt] = fmaf(v[q], x1, acc[q][bt]);
                 }
             }
         }

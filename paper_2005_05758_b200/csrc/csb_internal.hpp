@@ -25,12 +25,14 @@ void clear_error();
 //   chunk  = ChunkHeader (16 B), then the G sub-streams back to back
 //   sub-stream g = the items of lane group g, each aligned to 16 B
 //   item   = ItemHeader (16 B)
+//            values: a word is the kept rows of one kept column that one lane owns
+//                      f16: two consecutive kept rows (half2), RL = ceil(mr/2) words per column
+//                      f32: one kept row, RL = mr
+//                    (padding rows inside the last word are zero); columns 4q..4q+3 are
+//                    interleaved into 16-byte quad-words [q][w][4], the nk % 4 columns left
+//                    over follow as plain words [k][w]
 //            col_idx[nk]  uint8   gather indices, relative to xbase     (padded to 4 B)
-//            row_idx[mr]  uint8   scatter indices, relative to zbase    (padded to 4 B)
-//            values       nk columns of RL "row words" each, column-major:
-//                           f16: a word is two consecutive kept rows (half2), RL = ceil(mr/2)
-//                           f32: a word is one kept row, RL = mr
-//                         padding rows inside the last word are zero  (item padded to 16 B)
+//            row_idx[mr]  uint8   scatter indices, relative to zbase    (item padded to 16 B)
 //
 // An item is one block of the CSB matrix or a slice of it (a range of its kept
 // rows and of its kept columns).  Column-major kernel matrices let one lane own

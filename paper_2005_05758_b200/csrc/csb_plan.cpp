@@ -51,18 +51,25 @@ void emit_item(const csb_matrix* A, const ItemSpec& it, int gw, std::vector<uint
     p += sizeof h;
     const uint8_t* ci = A->col_idx.data() + A->cidx_off[it.block];
     const uint8_t* ri = A->row_idx.data() + A->ridx_off[it.block];
-    for (int k = 0; k < nk; ++k) p[k] = ci[it.k0 + k];
-    p += pad_to((size_t)nk, 4);
-    for (int r = 0; r < mr; ++r) p[r] = (uint8_t)(ri[it.r0 + r] - it.ridx_bias);
-    p += pad_to((size_t)mr, 4);
     const int n = A->n[it.block];
     const uint8_t* v = A->val.data() + A->val_off[it.block] * vs;
+    // word (k, w) = kept rows w*rpw .. of kept column k.  Columns 4q..4q+3 are interleaved into
+    // quad-words [q][w][4]; the nk % 4 columns left over follow as [k][w].
+    const int nquad = nk / 4;
+    auto word_at = [&](int k, int w) -> uint8_t* {
+        if (k < nquad * 4) return p + ((((size_t)(k / 4) * RL + w) * 4) + (k % 4)) * 4;
+        return p + ((size_t)nquad * RL * 4 + (size_t)(k - nquad * 4) * RL + w) * 4;
+    };
     for (int k = 0; k < nk; ++k)
         for (int w = 0; w < RL; ++w)
             for (int q = 0; q < rpw; ++q) {
                 const int r = it.r0 + w * rpw + q;
-                if (r < it.r1) std::memcpy(p + (((size_t)k * RL + w) * rpw + q) * vs, v + ((size_t)r * n + it.k0 + k) * vs, vs);
+                if (r < it.r1) std::memcpy(word_at(k, w) + q * vs, v + ((size_t)r * n + it.k0 + k) * vs, vs);
             }
+    p += (size_t)nk * RL * 4;
+    for (int k = 0; k < nk; ++k) p[k] = ci[it.k0 + k];
+    p += pad_to((size_t)nk, 4);
+    for (int r = 0; r < mr; ++r) p[r] = (uint8_t)(ri[it.r0 + r] - it.ridx_bias);
 }
 
 // Largest value payload of one item so that a chunk can hold one item per lane group.
