@@ -57,12 +57,12 @@ struct ChunkHeader {
 };
 static_assert(sizeof(ChunkHeader) == 16, "header is one 16-byte word");
 
-enum : uint32_t { kFlushNone = 0, kFlushDirect = 1, kFlushPartial = 2, kSlotShift = 3 };
+enum : uint32_t { kFlushNone = 0, kFlushDirect = 1, kFlushPartial = 2, kFlushCta = 3, kSlotShift = 3 };
 enum : uint16_t { kItemRecurrent = 1 };
 enum { kMaxNk = 64, kItemAlign = 16 };
 
 struct Chunk {
-    uint32_t off16;    // offset of the chunk in the stream, in 16-byte units
+    uint32_t off16;    // offset of the chunk in the stream, in 16-byte units; top two bits: flush kind
     uint32_t bytes;    // multiple of 16, <= stage_bytes
 };
 
@@ -79,6 +79,7 @@ struct StreamPlan {
 // Planned product (SpMV / SpMM) on the device.
 struct ProductPlan {
     int ctas = 0, warps = 0, stage_bytes = 0, stages = 0, group_width = 32;
+    int row_owned = 0;                     // every block-row belongs to one CTA: launch shape is fixed
     int x_in_smem = 0;
     size_t smem_bytes = 0;
     uint8_t* d_stream = nullptr;
@@ -163,8 +164,10 @@ struct ProductHostPlan {
     std::vector<uint32_t> part_base, part_count;   // per block-row
     uint32_t n_slots = 0;
     double balance = 1.0;
+    int row_owned = 0, ctas = 0, warps_per_cta = 0;   // row-owned mode fixes the launch shape
 };
-int plan_product_host(const csb_matrix* A, int n_warps, int stage_bytes, ProductHostPlan* out);
+int plan_product_host(const csb_matrix* A, int ctas, int warps_per_cta, int64_t useful_warps, int stage_bytes,
+                      ProductHostPlan* out);
 
 // Recurrent time loop: one descriptor per CTA.
 struct RnnCtaDesc {

@@ -114,7 +114,8 @@ static void emit_chunk(const csb_matrix* A, const std::vector<ItemSpec>& items, 
         h.sub16[g] = (uint16_t)((out->bytes.size() - s0) / 16);
     }
     std::memcpy(out->bytes.data() + start, &h, sizeof h);
-    out->chunks.push_back({(uint32_t)(start / 16), (uint32_t)(out->bytes.size() - start)});
+    // the flush kind rides in the top two bits of the offset, so the kernel knows it without the chunk
+    out->chunks.push_back({(uint32_t)(start / 16) | ((tail & 3u) << 30), (uint32_t)(out->bytes.size() - start)});
     *cost += (double)*std::max_element(load.begin(), load.end()) + 4.0;
 }
 

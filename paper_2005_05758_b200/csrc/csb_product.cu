@@ -41,6 +41,8 @@ struct ProductArgs {
 #define CSB_ADD(i, v) do { } while (0)
 #endif
 
+constexpr uint32_t kOffMask = 0x3fffffffu;   // Chunk::off16 without the flush kind in its top two bits
+
 __host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t)15; }
 
 // Shared-memory carve-up, identical on host and device.
@@ -109,6 +111,38 @@ __device__ __forceinline__ void flush_block_row(const ProductArgs& a, float* zs,
     if (lane == 0) a.arrivals[bi] = 0u;                // ready for the next launch
 }
 
+// End of a block-row that one CTA owns (all its warps are past the barrier): add the private
+// sums of every warp and lane group in a fixed order and store y.  `parts` adjacent lanes share
+// one output, each adds every parts-th copy, a fixed xor-tree joins them.
+template <int BT>
+__device__ __forceinline__ void cta_flush_block_row(const ProductArgs& a, const float* zs_all, int zs_stride, int copies,
+                                                    uint32_t zbase) {
+    const int nrows = min(a.block_r, a.rows - (int)zbase);
+    const int NZ = nrows * BT;
+    int parts = 1;
+    while (parts < 32 && parts * 2 * NZ <= (int)blockDim.x && parts * 2 <= copies) parts *= 2;
+    const int span = (NZ * parts + 31) & ~31;
+    for (int idx = threadIdx.x; idx < span; idx += blockDim.x) {
+        const int e = idx / parts, pt = idx % parts;
+        float sum = 0.f;
+        if (e < NZ) {
+            const float* src = zs_all + e;
+            for (int c = pt; c < copies; c += 8 * parts) {
+                float v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = (c + j * parts < copies) ? src[(c + j * parts) * zs_stride] : 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) sum += v[j];
+            }
+        }
+        for (int off = parts >> 1; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        if (e < NZ && pt == 0) {
+            const int r = e / BT, bt = e % BT;
+            if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = sum;
+        }
+    }
+}
+
 template <typename T, int BT, int GW>
 __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -148,12 +182,12 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
         mbar_fence_init();
         if (c0 < c1) {
             mbar_expect_tx(&bars[0], wd.w);
-            bulk_g2s(ring, a.stream + (size_t)wd.z * 16, wd.w, &bars[0]);
+            bulk_g2s(ring, a.stream + (size_t)(wd.z & kOffMask) * 16, wd.w, &bars[0]);
         }
         for (int s = 1; s < a.stages && c0 + s < c1; ++s) {
             const Chunk ch = a.chunks[c0 + s];
             mbar_expect_tx(&bars[s], ch.bytes);
-            bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)ch.off16 * 16, ch.bytes, &bars[s]);
+            bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)(ch.off16 & kOffMask) * 16, ch.bytes, &bars[s]);
         }
     }
     for (int i = lane; i < G * L.zs_stride; i += 32) zs[i] = 0.f;
@@ -172,23 +206,34 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
 #if defined(CSB_PHASE_CLOCKS) || defined(CSB_WALK_CLOCKS)
     long long wprof[6] = {0, 0, 0, 0, 0, 0};
 #endif
+    bool dead = x_dead;
+    bool reported = false;
+    Chunk cur = Chunk{wd.z, wd.w};
     for (uint32_t c = c0; c < c1; ++c) {
 #ifdef CSB_PHASE_CLOCKS
         const long long tc0 = clock64();
 #endif
         const int s = (int)((c - c0) % (uint32_t)a.stages);
         const uint32_t parity = ((c - c0) / (uint32_t)a.stages) & 1u;
+        const uint32_t flush = cur.off16 >> 30;                       // known without the chunk itself
+        const Chunk nxt = (c + 1 < c1) ? a.chunks[c + 1] : Chunk{0, 0};
         const Chunk refill = (c + a.stages < c1) ? a.chunks[c + a.stages] : Chunk{0, 0};
-        bool dead = x_dead || !mbar_wait_bounded(&bars[s], parity);
-        dead = __any_sync(0xffffffffu, dead);
-        if (dead) {
-            // report, then give the copies still in flight a bounded chance to land before leaving
+        if (!dead) dead = __any_sync(0xffffffffu, !mbar_wait_bounded(&bars[s], parity));
+        if (dead && !reported) {
+            // report, then give the copies still in flight a bounded chance to land.  A warp of
+            // a row-owned CTA keeps going through its chunk list without touching any data: the
+            // other warps of the CTA expect it at every block-row's barrier.
+            reported = true;
             if (lane == 0) {
                 *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout;
                 for (uint32_t j = c; j < c1 && j < c + (uint32_t)a.stages; ++j)
                     mbar_wait_bounded(&bars[(j - c0) % (uint32_t)a.stages], ((j - c0) / (uint32_t)a.stages) & 1u);
             }
-            break;
+        }
+        if (dead) {
+            if (flush == kFlushCta) { __syncthreads(); __syncthreads(); }
+            cur = nxt;
+            continue;
         }
 #ifdef CSB_PHASE_CLOCKS
         const long long tc1 = clock64();
@@ -226,7 +271,14 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
         const long long tc2 = clock64();
         CSB_ADD(3, tc2 - tc1);
 #endif
-        if ((ch.w & 3u) != kFlushNone) {
+        if (flush == kFlushCta) {
+            // the CTA owns this block-row: every warp is here with its last chunk of it
+            __syncthreads();
+            cta_flush_block_row<BT>(a, reinterpret_cast<const float*>(smem + L.zs), L.zs_stride, W * G, ch.z);
+            __syncthreads();
+            for (int i = lane; i < G * L.zs_stride; i += 32) zs[i] = 0.f;
+            __syncwarp();
+        } else if (flush != kFlushNone) {
             flush_block_row<BT, G>(a, zs, L.zs_stride, ch.z, ch.w, lane);
             __syncwarp();
         }
@@ -235,8 +287,9 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
 #endif
         if (lane == 0 && refill.bytes) {
             mbar_expect_tx(&bars[s], refill.bytes);
-            bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)refill.off16 * 16, refill.bytes, &bars[s]);
+            bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)(refill.off16 & kOffMask) * 16, refill.bytes, &bars[s]);
         }
+        cur = nxt;
     }
     CSB_STAMP(5);
 #ifdef CSB_PHASE_CLOCKS
@@ -263,7 +316,8 @@ static int upload(const std::vector<V>& h, V** d) {
 }
 
 static const int kBatchTiles[] = {8, 4, 1};
-enum { kMaxBatchTile = 8 };
+enum { kMaxBatchTile = 8, kTileDoesNotFit = 1 };
+
 
 // Largest warp count per CTA whose carve-up fits the opt-in shared memory.
 static int fit_warps(const csb_matrix* A, int want, int BT, int cols_in_smem, size_t* smem) {
@@ -293,12 +347,13 @@ int plan_product(csb_matrix* A) {
     // small matrices: no more warps than there is work for (about 2 KB of stream each)
     const int64_t approx = A->nnz * val_size(A->val_dtype) + (int64_t)A->ridx_off[A->nblk] + A->cidx_off[A->nblk] + 16 * A->nblk;
     const int64_t useful = std::max<int64_t>(1, approx / 2048);
-    const int n_warps = (int)std::min<int64_t>((int64_t)ctas * wpc, useful);
     ProductHostPlan H;
-    int rc = plan_product_host(A, n_warps, P.stage_bytes, &H);
+    int rc = plan_product_host(A, ctas, wpc, useful, P.stage_bytes, &H);
     if (rc != CSB_OK) return rc;
-    P.warps = std::max(1, (n_warps + ctas - 1) / ctas);
-    P.ctas = (n_warps + P.warps - 1) / P.warps;
+    const int n_warps = H.stream.n_warps;
+    P.row_owned = H.row_owned;
+    if (H.row_owned) { P.warps = H.warps_per_cta; P.ctas = H.ctas; }
+    else { P.warps = std::max(1, (n_warps + ctas - 1) / ctas); P.ctas = (n_warps + P.warps - 1) / P.warps; }
     P.n_slots = H.n_slots;
     P.group_width = H.stream.group_width;
     P.balance = H.balance;
@@ -309,7 +364,7 @@ int plan_product(csb_matrix* A) {
     std::vector<uint4> wdesc(n_warps);
     for (int w = 0; w < n_warps; ++w) {
         const uint32_t c0 = H.stream.warp_chunk_begin[w], c1 = H.stream.warp_chunk_begin[w + 1];
-        wdesc[w] = make_uint4(c0, c1, c0 < c1 ? H.stream.chunks[c0].off16 : 0u, c0 < c1 ? H.stream.chunks[c0].bytes : 0u);
+        wdesc[w] = make_uint4(c0, c1, c0 < c1 ? H.stream.chunks[c0].off16 : 0u, c0 < c1 ? H.stream.chunks[c0].bytes : 0u);   // off16 keeps its flush bits
     }
     if ((rc = upload(wdesc, (uint4**)&P.d_warp_desc)) != CSB_OK) return rc;
     if ((rc = upload(H.part_base, &P.d_part_base)) != CSB_OK) return rc;
@@ -349,6 +404,7 @@ static int launch_tile(const csb_matrix* A, ProductArgs a, cudaStream_t st) {
     }
     const int W = fit_warps(A, P.warps, BT, cols_in_smem, &smem);
     if (W == 0) { set_error("a single warp's shared-memory ring does not fit (%d stages of %d bytes)", P.stages, P.stage_bytes); return CSB_ERR_LAUNCH; }
+    if (P.row_owned && W != P.warps) return kTileDoesNotFit;      // the CTA shape is part of the plan: caller narrows the batch tile
     a.x_in_smem = cols_in_smem > 0;
     const int ctas = (P.n_warps + W - 1) / W;
     static bool configured[64] = {};                   // per device; setting it twice is harmless
@@ -403,12 +459,14 @@ int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, 
 #endif
     cudaStream_t st = (cudaStream_t)stream;
     int rc = CSB_OK;
+    int widest = kMaxBatchTile;                        // narrowed when a tile's shared memory does not fit the planned CTA
     for (int b0 = 0; b0 < batch && rc == CSB_OK;) {
         int bt = 1;
-        for (int cand : kBatchTiles) if (batch - b0 >= cand || cand == 1) { bt = cand; break; }
-        if (batch - b0 > 1 && bt == 1) bt = 4;          // 2 or 3 left: one padded tile of 4
+        for (int cand : kBatchTiles) if (cand <= widest && (batch - b0 >= cand || cand == 1)) { bt = cand; break; }
+        if (batch - b0 > 1 && bt == 1 && widest >= 4) bt = 4;          // 2 or 3 left: one padded tile of 4
         a.X = X + (int64_t)b0 * ldx; a.Y = Y + (int64_t)b0 * ldy; a.nb = std::min(bt, batch - b0);
         rc = dispatch_tile(A, a, st, bt);
+        if (rc == kTileDoesNotFit) { widest = bt == 8 ? 4 : 1; rc = CSB_OK; continue; }
         b0 += a.nb;
     }
     if (prev != A->device) cudaSetDevice(prev);

@@ -16,7 +16,9 @@ static int env_gw() {
 // the persistent grid one contiguous, equal-cost run of items, and mark the end of each
 // block-row inside a warp with how its accumulators leave the warp: straight to y when the
 // warp owns the whole block-row, else as a partial sum in its own slot.
-int plan_product_host(const csb_matrix* A, int n_warps, int stage_bytes, ProductHostPlan* out) {
+int plan_product_host(const csb_matrix* A, int ctas, int warps_per_cta, int64_t useful_warps, int stage_bytes,
+                      ProductHostPlan* out) {
+    int n_warps = (int)std::min<int64_t>((int64_t)ctas * warps_per_cta, std::max<int64_t>(1, useful_warps));
     const int rpw = rows_per_word(A->val_dtype);
     std::vector<int> rl;
     rl.reserve(A->nblk);
@@ -44,6 +46,65 @@ int plan_product_host(const csb_matrix* A, int n_warps, int stage_bytes, Product
     std::vector<double> cost(items.size());
     double total = 0;
     for (size_t i = 0; i < items.size(); ++i) { cost[i] = placeholder[i] ? 4.0 : (double)item_steps(A, items[i], gw); total += cost[i]; }
+
+    // Row-owned mode: with about as many block-rows as CTAs (or more), every block-row belongs to
+    // ONE CTA, whose warps share its items and add their sums up in shared memory behind a CTA
+    // barrier: no partial sums in global memory, no fences, no arrival counters.
+    const char* ro_env = getenv("CSB_ROW_OWNED");
+    const bool row_owned = ro_env && *ro_env ? atoi(ro_env) != 0 : (A->nbr * 5 >= (int64_t)ctas * 4 && n_warps >= ctas);
+    if (row_owned) {
+        const int G = 32 / gw;
+        const int n_ctas = (int)std::min<int64_t>(ctas, A->nbr);
+        // warps per CTA: enough lane groups for the items of a typical block-row, no more
+        const double items_per_row = (double)items.size() / (double)A->nbr;
+        const int wpc = std::max(1, std::min(warps_per_cta, (int)(items_per_row / G / 2.0 + 0.999)));
+        // block-rows to CTAs: heaviest first onto the least loaded CTA
+        std::vector<double> row_cost(A->nbr, 0.0);
+        std::vector<size_t> row_begin(A->nbr + 1, items.size());
+        for (size_t i = items.size(); i-- > 0;) { row_cost[item_row[i]] += cost[i] + 1.0; row_begin[item_row[i]] = i; }
+        std::vector<int64_t> order(A->nbr);
+        for (int64_t i = 0; i < A->nbr; ++i) order[i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](int64_t x, int64_t y) { return row_cost[x] > row_cost[y]; });
+        std::vector<double> cta_load(n_ctas, 0.0);
+        std::vector<std::vector<int64_t>> cta_rows(n_ctas);
+        for (int64_t bi : order) {
+            const int c = (int)(std::min_element(cta_load.begin(), cta_load.end()) - cta_load.begin());
+            cta_rows[c].push_back(bi);
+            cta_load[c] += row_cost[bi] / (wpc * G) + 60.0;      // a block-row also costs a CTA barrier and a reduction
+        }
+        std::vector<std::vector<Segment>> per_warp((size_t)n_ctas * wpc);
+        for (int c = 0; c < n_ctas; ++c) {
+            for (int64_t bi : cta_rows[c]) {
+                // this block-row's items, dealt longest first to the CTA's lane groups
+                std::vector<size_t> idx;
+                for (size_t i = row_begin[bi]; i < row_begin[bi + 1] && i < items.size() && item_row[i] == bi; ++i)
+                    if (!placeholder[i]) idx.push_back(i);
+                std::stable_sort(idx.begin(), idx.end(), [&](size_t x, size_t y) { return cost[x] > cost[y]; });
+                std::vector<double> load((size_t)wpc * G, 0.0);
+                for (int w = 0; w < wpc; ++w) {
+                    per_warp[(size_t)c * wpc + w].emplace_back();
+                    Segment& sg = per_warp[(size_t)c * wpc + w].back();
+                    sg.zbase = (uint32_t)(bi * A->block_r);
+                    sg.tail = kFlushCta;
+                }
+                for (size_t i : idx) {
+                    const int bin = (int)(std::min_element(load.begin(), load.end()) - load.begin());
+                    per_warp[(size_t)c * wpc + bin / G].back().items.push_back(items[i]);
+                    load[bin] += cost[i];
+                }
+            }
+        }
+        out->part_base.assign(A->nbr, 0);
+        out->part_count.assign(A->nbr, 0);
+        out->n_slots = 0;
+        out->row_owned = 1; out->ctas = n_ctas; out->warps_per_cta = wpc;
+        build_stream(A, per_warp, stage_bytes, &out->stream);
+        double mx = 0, sum = 0;
+        for (double l : cta_load) { mx = std::max(mx, l); sum += l; }
+        out->balance = mx > 0 ? sum / ctas / mx : 1.0;           // idle CTAs count against the balance
+        return CSB_OK;
+    }
+
     std::vector<std::vector<Segment>> per_warp(n_warps);
     const double target = total / n_warps;
     double cum = 0;
