@@ -208,7 +208,43 @@ def time_calls(torch, fn, steps, warmup, flush):
     return [a.elapsed_time(b) for a, b in ev]
 
 
-def spmv_sweep(binding, torch, dev, rates, batch, reps=10):
+def l2_read_roofline(torch, mbytes=48, reps=20):
+    """Read bandwidth of a buffer that stays in L2 (48 MiB, summed repeatedly inside one CUDA graph):
+    the denominator for products whose matrix is re-read from L2.  Measured here, nothing assumed."""
+    x = torch.ones(mbytes << 18, dtype=torch.float32, device="cuda")
+    out = torch.empty((), dtype=torch.float32, device="cuda")
+    for _ in range(3):
+        torch.sum(x, out=out)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        with torch.cuda.graph(g, stream=st):
+            for _ in range(reps):
+                torch.sum(x, out=out)
+    g.replay()
+    torch.cuda.synchronize()
+    best = 1e9
+    for _ in range(5):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); g.replay(); b.record()
+        torch.cuda.synchronize()
+        best = min(best, a.elapsed_time(b) / reps)
+    return x.numel() * 4 / (best * 1e-3) / 1e9
+
+
+def cpu_csb_loops(m, x, reps=3):
+    """The plain C loop nest over the CSB arrays (the oracle's second form) on the host cores."""
+    from oracle import csb_oracle
+    from oracle.csb_loops import CsbLoops
+    stored = csb_oracle.round_to_storage(m.dense, m.val_dtype).astype(np.float32)
+    L = CsbLoops(stored, m.block_r, m.block_c, m.row_keep, m.col_keep)
+    cores = len(os.sched_getaffinity(0))
+    return {"us_1_thread": round(L.seconds_per_spmv(x, 1, reps) * 1e6, 1),
+            "us_all_cores": round(L.seconds_per_spmv(x, cores, reps) * 1e6, 1), "cores": cores, "kind": "oracle (C loop nest)"}
+
+
+def spmv_sweep(binding, torch, dev, rates, batch, reps=10, with_cpu=False):
     """Bare CSB-SpMV on the 8192x8192 / 64x64 matrix, cold: launches rotate through enough encoded
     copies of the matrix to exceed L2, captured in one CUDA graph, timed with events."""
     hbm, _ = peaks()
@@ -247,15 +283,53 @@ def spmv_sweep(binding, torch, dev, rates, batch, reps=10):
             torch.cuda.synchronize()
             ts.append(a.elapsed_time(b) / n * 1e3)
         us = float(np.median(ts))
+        # warm: the same matrix again and again (it fits L2), against the measured L2 read rate
+        gw_ = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(st):
+            with torch.cuda.graph(gw_, stream=st):
+                for _ in range(40):
+                    if batch == 1:
+                        binding.csb_spmv(A0, X[0], Y[0])
+                    else:
+                        binding.csb_spmm(A0, X, Y)
+        gw_.replay()
+        torch.cuda.synchronize()
+        tw = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); gw_.replay(); b.record()
+            torch.cuda.synchronize()
+            tw.append(a.elapsed_time(b) / 40 * 1e3)
+        us_warm = float(np.median(tw))
+        del gw_
         alg = info["algorithmic_bytes"] + (m.cols + m.rows) * 4 * batch
         out.append({"rate": rate, "batch": batch, "nnz": info["nnz"], "us": round(us, 3), "algorithmic_bytes": alg,
                     "GBps": round(alg / us / 1e3, 1), "frac_hbm_measured": round(alg / us / 1e3 / hbm, 4),
                     "frac_hbm_8TBps": round(alg / us / 1e3 / 8000.0, 4), "GFLOPs": round(2 * info["nnz"] * batch / us / 1e3, 1),
+                    "us_warm_l2": round(us_warm, 3), "GBps_warm_l2": round(alg / us_warm / 1e3, 1),
                     "balance": round(info["balance"], 3), "copies": ncopy})
+        if with_cpu and rate == rates[0]:
+            out[-1]["cpu_csb_loops"] = cpu_csb_loops(m, w.X[0])
         for a in As:
             a.free()
         del g
     return out
+
+
+def slowest_rank_ms(local_ms, dist=None, device="cpu"):
+    """Replicas only: every rank runs its own sequences with no data-path collective; the job's
+    time for a step is the slowest rank's (max over ranks of the device-timed mean)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(local_ms)
+    import torch
+    t = torch.tensor([float(local_ms)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_us_per_timestep(ms_slowest, seq_len, world):
+    """All replicas' timesteps over the slowest replica's time (aggregate, weak scaling)."""
+    return ms_slowest * 1e3 / (seq_len * world)
 
 
 def other_configs(binding, torch, dev, flush, quick):
@@ -335,12 +409,8 @@ def main():
     barrier()
     wall = time.perf_counter() - wall0
     clocks = sampler.stop() if sampler else None
-    mean_ms = float(np.mean(ms))
-    if dist is not None:
-        t = torch.tensor([mean_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        mean_ms = float(t.item())
-    us_step = mean_ms * 1e3 / (w.T * world)          # all replicas' timesteps over the slowest replica's time
+    mean_ms = slowest_rank_ms(float(np.mean(ms)), dist, "cuda")
+    us_step = job_us_per_timestep(mean_ms, w.T, world)
 
     line = {"metric": METRIC, "value": round(us_step, 4), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(mean_ms, 4), "higher_is_better": False, "scaling": "weak",
@@ -365,18 +435,18 @@ def main():
         for _ in range(args.steps):
             fn_h()                                     # synchronous: copies in, kernel, copies out
         barrier()
-        e2e_ms = (time.perf_counter() - t0) / args.steps * 1e3
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        line["e2e"] = {"value": round(e2e_ms * 1e3 / (w.T * world), 4), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e_ms = slowest_rank_ms((time.perf_counter() - t0) / args.steps * 1e3, dist, "cuda")
+        line["e2e"] = {"value": round(job_us_per_timestep(e2e_ms, w.T, world), 4), "unit": UNIT, "h2d_bytes_per_step": h2d,
                        "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4)}
     for m in mats:
         m.free()
     if rank == 0 and "spmv" in sections:
         line["spmv"] = spmv_sweep(binding, torch, local, [float(r) for r in args.spmv_rates.split(",")], 1,
-                                  reps=args.spmv_reps)
+                                  reps=args.spmv_reps, with_cpu="cpu" in sections)
+        l2 = l2_read_roofline(torch)
+        line["l2_read_GBps_measured"] = round(l2, 1)
+        for r in line["spmv"]:
+            r["frac_l2_warm"] = round(r["GBps_warm_l2"] / l2, 4)
         best = max(line["spmv"], key=lambda r: r["frac_hbm_measured"])
         line["roofline_spmv"] = {"kernel": "csb_product_kernel<half,1>", "bound": "hbm", "achieved": best["GBps"], "peak": hbm,
                                  "peak_kind": peak_kind, "unit": "GB/s", "frac": best["frac_hbm_measured"], "traffic": None,

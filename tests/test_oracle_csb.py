@@ -177,3 +177,16 @@ def test_round_to_storage_is_ieee_binary16():
     # below half the smallest subnormal (2^-25) the result is zero.
     assert got.tolist() == [1.0, 1.0, 1.0 + 2.0 ** -9, 65504.0, np.inf, 0.0, -2.0 ** -24]
     assert np.array_equal(O.round_to_storage(v, "f32"), v.astype(np.float64))
+
+
+def test_c_loop_nest_matches_masked_dense():
+    # the second oracle form (plain C loops over the five CSB arrays) against the definition
+    from oracle.csb_loops import CsbLoops
+    w = workloads.make_spmv_workload(9, 200, 333, 32, 64, "lognormal", rate=5.0, batch=1, w_std=0.05)
+    m = w.matrix
+    stored = O.round_to_storage(m.dense, "f16").astype(np.float32)
+    L = CsbLoops(stored, 32, 64, m.row_keep, m.col_keep)
+    want = O.spmm(m.dense, 32, 64, m.row_keep, m.col_keep, "f16", w.X)[0]
+    for threads in (1, 3):
+        np.testing.assert_allclose(L.spmv(w.X[0], threads), want, rtol=1e-12, atol=1e-13)
+    assert L.nnz == int(O.block_mask(200, 333, 32, 64, m.row_keep, m.col_keep).sum())
