@@ -100,6 +100,7 @@ int csb_info(const csb_matrix_t* A, csb_info_t* o) {
 void csb_free(csb_matrix_t* A) {
     if (!A) return;
     drop_rnn_plans(A);
+    free_mma(A);
     free_product(A);
     delete A;
 }
@@ -112,6 +113,10 @@ int csb_spmm(const csb_matrix_t* A, const float* X, int64_t ldx, int batch, floa
     if (!X || !Y) { set_error("X or Y is NULL"); return CSB_ERR_INVALID_ARG; }
     if (ldx < A->cols || ldy < A->rows) { set_error("ldx=%lld < cols or ldy=%lld < rows", (long long)ldx, (long long)ldy); return CSB_ERR_SHAPE; }
     if (A->device < 0) { set_error("matrix was encoded host-only (device = -1)"); return CSB_ERR_UNSUPPORTED; }
+    if (spmm_mma_applicable(A, batch)) {
+        const int rc = launch_spmm_mma(A, X, ldx, batch, Y, ldy, stream);
+        if (rc != 1) return rc;                       // 1: the tensor-core plan does not fit this matrix
+    }
     return launch_product(A, X, ldx, batch, Y, ldy, stream);
 }
 

@@ -59,7 +59,7 @@ static_assert(sizeof(ChunkHeader) == 16, "header is one 16-byte word");
 
 enum : uint32_t { kFlushNone = 0, kFlushDirect = 1, kFlushPartial = 2, kFlushCta = 3, kSlotShift = 3 };
 enum : uint16_t { kItemRecurrent = 1 };
-enum { kMaxNk = 64, kItemAlign = 16 };
+enum { kMaxNk = 64, kItemAlign = 16, kMmaMaxNk = 32 };
 
 struct Chunk {
     uint32_t off16;    // offset of the chunk in the stream, in 16-byte units; top two bits: flush kind
@@ -100,6 +100,7 @@ struct ProductPlan {
 
 struct Planner;                            // csb_plan.cpp
 struct RnnPlan;                            // csb_rnn.cu
+struct MmaPlan;                            // tensor-core SpMM plan (below)
 
 }  // namespace csb
 
@@ -119,6 +120,8 @@ struct csb_matrix {
     std::vector<uint8_t> val;              // nnz * (2 | 4) bytes
     // device side
     csb::ProductPlan product;
+    mutable csb::MmaPlan* mma = nullptr;   // tensor-core SpMM plan, built lazily
+    mutable std::mutex mma_mu;
     int sm_count = 0;
     size_t smem_optin = 0;
     uint64_t uid = 0;                      // identity for the recurrent-plan cache
@@ -185,6 +188,34 @@ struct RnnHostPlan {
 };
 int plan_rnn_host(int gates, int n_layers, const csb_matrix* const* Wm, const int* in_size, int H, int n_ctas,
                   int warps, int stage_bytes, RnnHostPlan* out);
+
+// ---- tensor-core SpMM path (csb_mma_plan.cpp, csb_spmm_mma.cu) ----
+struct MmaItemHeader {
+    uint8_t nk, mr, RT, KT;   // kept columns / rows of the item, its 16-row and 8-column tile counts
+    uint32_t xbase;           // first column of the block
+    uint32_t pad[2];
+};
+static_assert(sizeof(MmaItemHeader) == 16, "header is one 16-byte word");
+struct MmaHostPlan {
+    std::vector<uint8_t> bytes;
+    std::vector<Chunk> chunks;
+    std::vector<uint32_t> warp_chunk_begin;
+    int ctas = 0, warps_per_cta = 0;
+    size_t max_chunk_bytes = 0;
+    double balance = 1.0;
+};
+int plan_mma_host(const csb_matrix* A, int ctas, int warps_per_cta, int stage_bytes, MmaHostPlan* out);
+struct MmaPlan {                           // device side, built on the first batched product
+    int ctas = 0, warps = 0, stage_bytes = 0, stages = 0, n_warps = 0;
+    uint8_t* d_stream = nullptr; Chunk* d_chunks = nullptr; void* d_warp_desc = nullptr;
+    void* d_xp = nullptr; size_t xp_bytes = 0;   // packed fp16 hi/lo copy of a 32-column batch slab
+    int64_t stream_bytes = 0;
+    double balance = 1.0;
+    bool built = false, unusable = false;
+};
+int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream);
+bool spmm_mma_applicable(const csb_matrix* A, int batch);
+void free_mma(csb_matrix* A);
 
 // csb_product.cu
 int plan_product(csb_matrix* A);           // plans, uploads, fills A->product
