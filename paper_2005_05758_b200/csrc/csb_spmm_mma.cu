@@ -68,6 +68,7 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(row_ptr)));
 }
 
+template <int NT>
 __global__ void __launch_bounds__(256, 1) csb_spmm_mma_kernel(const MmaArgs a) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -172,9 +173,9 @@ __global__ void __launch_bounds__(256, 1) csb_spmm_mma_kernel(const MmaArgs a) {
             buf ^= 1;
             // ---- multiply: D[16 kept rows x 8 batch] += A[16 x 8 kept columns] . B[8 x 8], four batch tiles
             for (int rt = 0; rt < RT; ++rt) {
-                float acc[4][4];
+                float acc[NT][4];
 #pragma unroll
-                for (int nt = 0; nt < 4; ++nt)
+                for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
                 const uint2* at = reinterpret_cast<const uint2*>(tiles + (size_t)rt * KT * 256) + lane;
@@ -186,7 +187,7 @@ __global__ void __launch_bounds__(256, 1) csb_spmm_mma_kernel(const MmaArgs a) {
                     ldmatrix_x4_trans(bh, xs_hi + off);
                     ldmatrix_x4_trans(bl, xs_lo + off);
 #pragma unroll
-                    for (int nt = 0; nt < 4; ++nt) {
+                    for (int nt = 0; nt < NT; ++nt) {          // batch tiles past NT hold zero columns: skipped
                         mma_m16n8k8(acc[nt], af.x, af.y, bh[nt]);
                         mma_m16n8k8(acc[nt], af.x, af.y, bl[nt]);
                     }
@@ -199,7 +200,7 @@ __global__ void __launch_bounds__(256, 1) csb_spmm_mma_kernel(const MmaArgs a) {
                     if (r < mr) {
                         float* z = zs + (int)ridx[r] * kZStride + 2 * t;
 #pragma unroll
-                        for (int nt = 0; nt < 4; ++nt) {
+                        for (int nt = 0; nt < NT; ++nt) {
                             float2 cur2 = *reinterpret_cast<float2*>(z + nt * 8);
                             cur2.x += acc[nt][2 * half]; cur2.y += acc[nt][2 * half + 1];
                             *reinterpret_cast<float2*>(z + nt * 8) = cur2;
@@ -276,7 +277,9 @@ static int build_mma_plan(const csb_matrix* A, MmaPlan* P) {
     if ((rc = upload_v(wdesc, (uint4**)&P->d_warp_desc)) != CSB_OK) return rc;
     P->xp_bytes = (size_t)A->cols * 64 * sizeof(__half);
     CSB_CUDA(cudaMalloc(&P->d_xp, P->xp_bytes));
-    CSB_CUDA(cudaFuncSetAttribute(csb_spmm_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
+    CSB_CUDA(cudaFuncSetAttribute(csb_spmm_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
+    CSB_CUDA(cudaFuncSetAttribute(csb_spmm_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
+    CSB_CUDA(cudaFuncSetAttribute(csb_spmm_mma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
     CSB_CUDA(cudaDeviceSynchronize());
     P->built = true;
     return CSB_OK;
@@ -324,7 +327,9 @@ int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch,
         a.nb = std::min(kSlab, batch - b0);
         a.Y = Y + (int64_t)b0 * ldy;
         csb_pack_x_kernel<<<(unsigned)((A->cols + 7) / 8), 256, 0, st>>>(X + (int64_t)b0 * ldx, ldx, a.nb, (int)A->cols, (__half*)P.d_xp);
-        csb_spmm_mma_kernel<<<P.ctas, P.warps * 32, L.total, st>>>(a);
+        if (a.nb <= 8) csb_spmm_mma_kernel<1><<<P.ctas, P.warps * 32, L.total, st>>>(a);
+        else if (a.nb <= 16) csb_spmm_mma_kernel<2><<<P.ctas, P.warps * 32, L.total, st>>>(a);
+        else csb_spmm_mma_kernel<4><<<P.ctas, P.warps * 32, L.total, st>>>(a);
         CSB_CUDA(cudaGetLastError());
     }
     return CSB_OK;
