@@ -357,11 +357,12 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="rnn,e2e,spmv,configs,cpu",
-                    help="comma list of: rnn (always), e2e, spmv, configs, cpu")
+    ap.add_argument("--sections", default="rnn,e2e,spmv,spmm,configs,cpu",
+                    help="comma list of: rnn (always), e2e, spmv, spmm, configs, cpu")
     ap.add_argument("--seq-len", type=int, default=512)
     ap.add_argument("--spmv-rates", default="4,8,16,25", help="pruning rates of the bare SpMV sweep")
     ap.add_argument("--spmv-reps", type=int, default=10)
+    ap.add_argument("--spmm-batches", default="8,64", help="batch sizes of the SpMM sweep (section spmm)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -451,6 +452,11 @@ def main():
         line["roofline_spmv"] = {"kernel": "csb_product_kernel<half,1>", "bound": "hbm", "achieved": best["GBps"], "peak": hbm,
                                  "peak_kind": peak_kind, "unit": "GB/s", "frac": best["frac_hbm_measured"], "traffic": None,
                                  "workload": "cfg4 8192x8192, 64x64 blocks, rate %gx, batch 1, cold (rotating copies > L2)" % best["rate"]}
+    if rank == 0 and "spmm" in sections:
+        line["spmm"] = []
+        for bsz in [int(b) for b in args.spmm_batches.split(",")]:
+            line["spmm"] += spmv_sweep(binding, torch, local, [float(r) for r in args.spmv_rates.split(",")], bsz,
+                                       reps=args.spmv_reps)
     if rank == 0 and "configs" in sections:
         line["configs"] = other_configs(binding, torch, local, flush, quick=False)
     if rank == 0 and "cpu" in sections:

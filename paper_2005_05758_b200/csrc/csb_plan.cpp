@@ -27,14 +27,19 @@ size_t item_bytes(const csb_matrix* A, const ItemSpec& it) {
     return pad_to(sizeof(ItemHeader) + pad_to((size_t)nk, 4) + pad_to((size_t)mr, 4) + (size_t)nk * row_words(A, mr) * 4, kItemAlign);
 }
 
-// Lock-step cost of an item for a lane group of width gw, in units of one column step of the
-// multiply loop (about 7 instructions): the column steps plus a fixed part for header decode,
-// gather, fold and scatter (about 190 instructions, from instruction counts of the kernel).
+// Lock-step cost of an item for a lane group of width gw (unit: about nine instructions), from
+// instruction counts of the kernel: a fixed part for header decode, gather, fold and scatter, and
+// the multiply loop's iterations over quad-columns and tail columns.
 enum { kItemFixedSteps = 27 };
 int item_steps(const csb_matrix* A, const ItemSpec& it, int gw) {
+    // about 9 instructions per unit: ~150 fixed, ~22 per quad-column iteration, ~9 per tail-column
+    // iteration, ~10 per fold round
     const int nk = it.k1 - it.k0, RL = std::max(1, row_words(A, it.r1 - it.r0));
     const int S = std::max(1, gw / RL);
-    return (nk + S - 1) / S + kItemFixedSteps;
+    int fold = 0;
+    while ((1 << fold) < S) ++fold;
+    const int quad_iters = ((nk >> 2) + S - 1) / S, tail_iters = ((nk & 3) + S - 1) / S;
+    return (150 + 22 * quad_iters + 9 * tail_iters + 10 * fold + 4) / 9;
 }
 
 void emit_item(const csb_matrix* A, const ItemSpec& it, int gw, std::vector<uint8_t>& out) {
