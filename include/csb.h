@@ -133,7 +133,14 @@ int csb_spmv(const csb_matrix_t* A, const float* x, float* y, void* stream);
  * csb_spmm -- Y[b, :] = A . X[b, :] for b < batch (the same product with a batch of vectors).
  *   X  device, float32, batch rows of `cols` values, row stride ldx >= cols;
  *   Y  device, float32, batch rows of `rows` values, row stride ldy >= rows, overwritten.
- * batch = 0 is a no-op.  Same ordering / overlap rules as csb_spmv.
+ * batch = 0 is a no-op.  Same ordering / overlap rules as csb_spmv; results are bit-reproducible.
+ * With batch >= 8, fp16 values and block_r <= 64 the product runs on tensor cores (the kernel
+ * matrix times the gathered inputs is then a dense contraction): the inputs of a slab of 32 batch
+ * columns are split into two binary16 halves (x = hi + lo, so no input precision is lost as long
+ * as |x| < 65504) and multiplied with mma.sync, fp32 accumulation.  The first such call on a
+ * handle builds a second device layout and a staging buffer for it (allocates and synchronises
+ * the device once; make it outside of any stream capture).  Other cases use the CUDA-core kernel
+ * in batch tiles of 8 / 4 / 1.
  */
 int csb_spmm(const csb_matrix_t* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy,
              void* stream);

@@ -34,6 +34,7 @@ struct RnnArgs {
     unsigned long long barrier_ns;
     unsigned int barrier_extra;   // test hook: arrivals that never come
     int T, B, H, L, gates, stage_bytes, stages, resident, max_warp_bytes, max_U, max_C;
+    int v_tile;                // batched: [u_t ; h_{t-1}] of the current batch tile is staged in shared memory, [bt][column]
     int v_bulk;                // batch 1: [u_t ; h_{t-1}] may come in by bulk copy (16-byte aligned pieces)
 #ifdef CSB_PHASE_CLOCKS
     long long* clocks;         // [n_ctas][5] cycles summed over ticks: stage, walk, reduce, gates, barrier
@@ -50,7 +51,7 @@ struct RnnSmem {
     size_t weights, bars, zs, xg, v, cs, zsum, vbar, flag, total;
     int zs_stride;
     __host__ __device__ RnnSmem(int W, int G, int stages, int stage_bytes, int resident, int max_warp_bytes, int max_U, int BT,
-                                int B, int max_C) {
+                                int B, int max_C, int v_tile) {
         zs_stride = 4 * max_U * BT + group_pad(32 / G);   // floats per lane group
         weights = 0;
         const size_t per_warp = resident ? (size_t)max_warp_bytes : (size_t)stages * stage_bytes;
@@ -58,7 +59,7 @@ struct RnnSmem {
         zs = (bars + (size_t)W * (resident ? 1 : stages) * 8 + 15) & ~(size_t)15;
         xg = (zs + (size_t)W * G * zs_stride * 4 + 15) & ~(size_t)15;
         v = (xg + (size_t)W * G * xg_stride(32 / G, BT) * 4 + 15) & ~(size_t)15;
-        cs = (v + (BT == 1 ? (size_t)max_C * 4 : 0) + 15) & ~(size_t)15;
+        cs = (v + (BT == 1 ? (size_t)max_C * 4 : (v_tile ? (size_t)max_C * BT * 4 : 0)) + 15) & ~(size_t)15;
         zsum = (cs + (size_t)max_U * B * 4 + 15) & ~(size_t)15;
         vbar = (zsum + (size_t)4 * max_U * BT * 4 + 15) & ~(size_t)15;
         flag = vbar + 16;                              // two mbarriers: input half, recurrent half
@@ -119,7 +120,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int G = 32 / GW;
     const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const RnnSmem S(W, G, a.stages, a.stage_bytes, RES, a.max_warp_bytes, a.max_U, BT, a.B, a.max_C);
+    const RnnSmem S(W, G, a.stages, a.stage_bytes, RES, a.max_warp_bytes, a.max_U, BT, a.B, a.max_C, a.v_tile);
     const RnnCtaDesc me = a.ctas[blockIdx.x];
     const int layer = me.layer, U = me.U, u0 = me.u0, H = a.H, B = a.B;
     const int I = a.in_size[layer];
@@ -236,14 +237,26 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                 v.z = vs[base + ((c4 >> 16) & 0xffu)]; v.w = vs[base + (c4 >> 24)];
                 *reinterpret_cast<float4*>(dst) = v;
             } else {
+                if (a.v_tile) {
+                    // staged tile: row bt holds [u ; h] of batch column b0 + bt (zeros past nb); padding
+                    // indices are zero and land on the block's first column, which exists
+                    const uint32_t base = xbase + (rec ? (uint32_t)I : 0u);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t col = xbase + ((c4 >> (8 * j)) & 0xffu);
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t c = base + ((c4 >> (8 * j)) & 0xffu);
 #pragma unroll
-                    for (int bt = 0; bt < BT; ++bt)
-                        dst[j * BT + bt] = (j < left && bt < nb)
-                            ? (rec ? __ldcg(rec_src + (size_t)(b0 + bt) * H + col) : __ldcg(in_src + (size_t)(b0 + bt) * in_ld + col))
-                            : 0.f;
+                        for (int bt = 0; bt < BT; ++bt) dst[j * BT + bt] = vs[(uint32_t)bt * (uint32_t)a.max_C + c];
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t col = xbase + ((c4 >> (8 * j)) & 0xffu);
+#pragma unroll
+                        for (int bt = 0; bt < BT; ++bt)
+                            dst[j * BT + bt] = (j < left && bt < nb)
+                                ? (rec ? __ldcg(rec_src + (size_t)(b0 + bt) * H + col) : __ldcg(in_src + (size_t)(b0 + bt) * in_ld + col))
+                                : 0.f;
+                    }
                 }
             }
         };
@@ -303,6 +316,19 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
             for (int b0 = 0; b0 < B; b0 += BT) {
                 const int nb = min(BT, B - b0);
                 if (BT == 1) stage_issue(1, vs + I, rec_src, H);
+                if (BT > 1 && a.v_tile) {
+                    // this batch tile's [u ; h], one row per batch column (the previous tile's readers
+                    // left at the barrier that ends the gate arithmetic)
+                    const int C = I + H;
+                    for (int bt = 0; bt < BT; ++bt) {
+                        const float* ui = in_src + (size_t)(b0 + bt) * in_ld;
+                        const float* hi = rec_src + (size_t)(b0 + bt) * H;
+                        float* row = vs + (size_t)bt * a.max_C;
+                        for (int i = threadIdx.x; i < C; i += blockDim.x)
+                            row[i] = bt < nb ? __ldcg(i < I ? ui + i : hi + (i - I)) : 0.f;
+                    }
+                    __syncthreads();
+                }
                 if (!pre_done) {
                     if (BT == 1) { stage_issue(0, vs, in_src, I); stage_wait(0, vs, in_src, I); }
                     zero_zs();
@@ -410,7 +436,7 @@ struct RnnPlan {
     int gates = 0, L = 0, B = 0, H = 0, device = 0, val_dtype = 0;
     std::vector<uint64_t> uids;
     int in_size[kMaxLayers] = {};
-    int n_ctas = 0, warps = 0, BT = 1, GW = 32, resident = 0, stages = 0, stage_bytes = 0, max_warp_bytes = 0, max_U = 0, max_C = 0;
+    int n_ctas = 0, warps = 0, BT = 1, GW = 32, v_tile = 0, resident = 0, stages = 0, stage_bytes = 0, max_warp_bytes = 0, max_U = 0, max_C = 0;
     size_t smem = 0;
     double balance = 1.0;
     int64_t stream_bytes = 0;
@@ -467,6 +493,7 @@ static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, i
     for (int l = 0; l < L; ++l) approx += W[l]->nnz * val_size(W[l]->val_dtype) + 32 * W[l]->nblk;
     int want = (int)std::min<int64_t>(A0->sm_count, std::max<int64_t>(L, approx / (24 * 1024)));
     want = std::max(want, L * ((H + 47) / 48));        // tiles are cut by cost; leave room under the 64-unit limit
+    if (P->BT > 1) want = A0->sm_count;               // batched: small unit tiles keep the per-group accumulators small
     want = env_int("CSB_RNN_CTAS", want);
     want = std::min(std::max(want, L), A0->sm_count);
     // fewer warps per CTA shrink the per-warp accumulators and rings until the carve-up fits
@@ -474,10 +501,15 @@ static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, i
     int rc = CSB_OK;
     const int first = P->warps;
     bool fits = false;
-    for (int wtry : {first, 12, 8, 6, 4, 2, 1}) {
-        if (wtry > first) continue;
-        // first with one chunk per warp (weights resident, no ring to fit the chunks into), then
-        // with ring-sized chunks for streaming
+    // candidates, best first: with the batched input tile staged in shared memory when it fits beside
+    // at least 8 warps; each with one chunk per warp (weights resident) before ring-sized chunks
+    struct Cand { int warps, v_tile; };
+    std::vector<Cand> cands;
+    for (int vt : {1, 0})
+        for (int wt : {first, 12, 8}) if (wt <= first && (vt == 0 || P->BT > 1)) cands.push_back({wt, vt});
+    for (int wt : {6, 4, 2, 1}) if (wt <= first) { if (P->BT > 1) cands.push_back({wt, 1}); cands.push_back({wt, 0}); }
+    for (const Cand& cd : cands) {
+        const int wtry = cd.warps;
         for (int pass = 0; pass < 2 && !fits; ++pass) {
             if (pass == 0 && env_int("CSB_RNN_STREAM", 0)) continue;
             const int chunk_bytes = pass == 0 ? (256 << 10) : P->stage_bytes;
@@ -485,9 +517,10 @@ static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, i
             rc = plan_rnn_host(gates, L, W, in_size, H, want, wtry, chunk_bytes, &Hp);
             if (rc != CSB_OK) return rc;
             P->warps = wtry;
+            P->v_tile = cd.v_tile;
             P->max_U = Hp.max_U; P->max_warp_bytes = (int)Hp.max_warp_bytes; P->GW = Hp.stream.group_width;
             const int G = 32 / P->GW;
-            const RnnSmem sm(wtry, G, P->stages, P->stage_bytes, pass == 0, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C);
+            const RnnSmem sm(wtry, G, P->stages, P->stage_bytes, pass == 0, P->max_warp_bytes, P->max_U, P->BT, B, P->max_C, cd.v_tile);
             if (sm.total <= A0->smem_optin) { P->resident = pass == 0; P->smem = sm.total; fits = true; }
         }
         if (fits) break;
@@ -633,6 +666,7 @@ static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const flo
     for (int l = 0; l < L; ++l) { a.bias[l] = bias ? bias[l] : nullptr; a.in_size[l] = in_size[l]; }
     a.barrier = P->d_barrier; a.status = P->d_status; a.barrier_ns = g_barrier_ns; a.barrier_extra = g_barrier_extra;
     a.T = (int)T; a.B = B; a.H = H; a.L = L; a.gates = gates; a.stage_bytes = P->stage_bytes; a.stages = P->stages;
+    a.v_tile = env_int("CSB_RNN_NO_VTILE", 0) ? 0 : P->v_tile;
     a.v_bulk = 0;
     if (P->BT == 1 && H % 4 == 0 && (reinterpret_cast<uintptr_t>(dx) & 15) == 0) {
         a.v_bulk = 1;
