@@ -173,7 +173,7 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
             const uint4* qend = quads + nq;
             const float* xp = xg + 4 * kg * BT;
             const int xs = 4 * S * BT;
-#pragma unroll 2
+#pragma unroll 1
             for (; qp < qend; qp += A, xp += xs) {
                 const uint4 w = *qp;
                 const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
