@@ -217,6 +217,24 @@ int csb_gru_forward(int n_layers, const csb_matrix_t* const* W, const float* con
  */
 void csb_test_barrier_hook(unsigned int extra_arrivals, unsigned long long limit_ns);
 
+/*
+ * csb_plan_dump -- inspection / testing aid (the paper has no counterpart): plan the bare product
+ * for a persistent grid of `ctas` x `warps_per_cta` warps and ring stages of `stage_bytes` bytes,
+ * on the host only (works for handles encoded with device = -1), and copy the planned device
+ * stream out so that its layout and schedule can be checked without a GPU.
+ *   info_out        host, int64[8]: warps, chunks, stream bytes, lane-group width, row-owned flag,
+ *                   CTAs, warps per CTA, partial-sum slots.  Always written.
+ *   stream_out      host, `stream_cap` bytes, or NULL;  chunks_out  host, uint32 pairs
+ *                   (offset in 16-byte units with the flush kind in the top two bits, bytes),
+ *                   `chunks_cap` pairs, or NULL;  warp_begin_out  host, uint32[`warp_cap`], first
+ *                   chunk of every warp plus one end entry, or NULL.
+ * A buffer that is too small is an error (CSB_ERR_INVALID_ARG); call once with NULL buffers to
+ * learn the sizes.
+ */
+int csb_plan_dump(const csb_matrix_t* A, int ctas, int warps_per_cta, int stage_bytes, int64_t* info_out,
+                  uint8_t* stream_out, int64_t stream_cap, uint32_t* chunks_out, int64_t chunks_cap,
+                  uint32_t* warp_begin_out, int64_t warp_cap);
+
 /* Short text for a status code; never NULL. */
 const char* csb_strerror(int status);
 

@@ -155,6 +155,23 @@ def csb_encode(dense: np.ndarray, block_r: int, block_c: int, row_keep: np.ndarr
     return CsbMatrix(out.value)
 
 
+def csb_plan_dump(A: CsbMatrix, ctas: int, warps_per_cta: int, stage_bytes: int) -> dict:
+    """Host-only plan of the bare product, copied out for inspection (see csb.h)."""
+    lib.csb_plan_dump.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, C.c_int64, _P, C.c_int64, _P, C.c_int64]
+    lib.csb_plan_dump.restype = C.c_int
+    info = np.zeros(8, np.int64)
+    _check(lib.csb_plan_dump(A.handle, ctas, warps_per_cta, stage_bytes, info.ctypes.data, None, 0, None, 0, None, 0))
+    stream = np.zeros(max(int(info[2]), 1), np.uint8)
+    chunks = np.zeros((max(int(info[1]), 1), 2), np.uint32)
+    wbeg = np.zeros(int(info[0]) + 1, np.uint32)
+    _check(lib.csb_plan_dump(A.handle, ctas, warps_per_cta, stage_bytes, info.ctypes.data, stream.ctypes.data, stream.size,
+                             chunks.ctypes.data, chunks.shape[0], wbeg.ctypes.data, wbeg.size))
+    keys = ("warps", "chunks", "stream_bytes", "group_width", "row_owned", "ctas", "warps_per_cta", "slots")
+    out = {k: int(v) for k, v in zip(keys, info)}
+    out.update(stream=stream[: out["stream_bytes"]], chunk_table=chunks[: out["chunks"]], warp_begin=wbeg)
+    return out
+
+
 def csb_spmv(A: CsbMatrix, x, y, stream=None) -> None:
     _check(lib.csb_spmv(A.handle, _ptr(x), _ptr(y), _stream(stream)))
 

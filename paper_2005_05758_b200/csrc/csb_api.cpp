@@ -97,6 +97,38 @@ int csb_info(const csb_matrix_t* A, csb_info_t* o) {
     return CSB_OK;
 }
 
+int csb_plan_dump(const csb_matrix_t* A, int ctas, int warps_per_cta, int stage_bytes, int64_t* info_out,
+                  uint8_t* stream_out, int64_t stream_cap, uint32_t* chunks_out, int64_t chunks_cap,
+                  uint32_t* warp_begin_out, int64_t warp_cap) {
+    clear_error();
+    if (!A || !info_out || ctas < 1 || warps_per_cta < 1 || warps_per_cta > 16 || stage_bytes < 1024 || (stage_bytes & 15)) {
+        set_error("csb_plan_dump: bad argument");
+        return CSB_ERR_INVALID_ARG;
+    }
+    ProductHostPlan H;
+    int rc;
+    try { rc = plan_product_host(A, ctas, warps_per_cta, (int64_t)ctas * warps_per_cta, stage_bytes, &H); }
+    catch (const std::bad_alloc&) { set_error("out of host memory while planning"); return CSB_ERR_ALLOC; }
+    if (rc != CSB_OK) return rc;
+    const StreamPlan& S = H.stream;
+    info_out[0] = S.n_warps; info_out[1] = (int64_t)S.chunks.size(); info_out[2] = (int64_t)S.bytes.size();
+    info_out[3] = S.group_width; info_out[4] = H.row_owned; info_out[5] = H.row_owned ? H.ctas : ctas;
+    info_out[6] = H.row_owned ? H.warps_per_cta : warps_per_cta; info_out[7] = H.n_slots;
+    if (stream_out) {
+        if (stream_cap < (int64_t)S.bytes.size()) { set_error("stream buffer too small"); return CSB_ERR_INVALID_ARG; }
+        std::memcpy(stream_out, S.bytes.data(), S.bytes.size());
+    }
+    if (chunks_out) {
+        if (chunks_cap < (int64_t)S.chunks.size()) { set_error("chunk buffer too small"); return CSB_ERR_INVALID_ARG; }
+        for (size_t i = 0; i < S.chunks.size(); ++i) { chunks_out[2 * i] = S.chunks[i].off16; chunks_out[2 * i + 1] = S.chunks[i].bytes; }
+    }
+    if (warp_begin_out) {
+        if (warp_cap < (int64_t)S.warp_chunk_begin.size()) { set_error("warp table too small"); return CSB_ERR_INVALID_ARG; }
+        for (size_t i = 0; i < S.warp_chunk_begin.size(); ++i) warp_begin_out[i] = S.warp_chunk_begin[i];
+    }
+    return CSB_OK;
+}
+
 void csb_free(csb_matrix_t* A) {
     if (!A) return;
     drop_rnn_plans(A);
