@@ -214,14 +214,14 @@ def l2_read_roofline(torch, mbytes=48, reps=20):
     x = torch.ones(mbytes << 18, dtype=torch.float32, device="cuda")
     out = torch.empty((), dtype=torch.float32, device="cuda")
     for _ in range(3):
-        torch.sum(x, out=out)
+        torch.sum(x, dim=0, out=out)
     torch.cuda.synchronize()
     g = torch.cuda.CUDAGraph()
     st = torch.cuda.Stream()
     with torch.cuda.stream(st):
         with torch.cuda.graph(g, stream=st):
             for _ in range(reps):
-                torch.sum(x, out=out)
+                torch.sum(x, dim=0, out=out)
     g.replay()
     torch.cuda.synchronize()
     best = 1e9
