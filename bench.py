@@ -34,6 +34,13 @@ UNIT = "us/timestep"
 WORKLOAD = "cfg5: 2-layer LSTM, I=H=2048, 8192x4096 CSB weights, 64x64 blocks, ~10x pruning, T=512, B=1, fp16 values / fp32 accumulate"
 
 
+# dram__bytes_read + dram__bytes_write per launch from the ncu captures summarised under profiles/
+# (csb_rnn_kernel_cfg5.md: T = 512 launch; csb_product_kernel_cfg4_rate4_b1.md).  They describe the
+# kernels as committed with those summaries; set to None when a kernel or its layout changes.
+RNN_DRAM_BYTES_PER_LAUNCH = 20288768 + 11008
+SPMV4X_DRAM_BYTES_PER_LAUNCH = 35873280
+
+
 def peaks():
     """Measured HBM copy bandwidth of this machine's B200 (generated file), else the fallback."""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -423,7 +430,8 @@ def main():
     alg_step = rnn_alg_bytes_per_step(w, infos)
     achieved = alg_step * w.T / (mean_ms * 1e-3) / 1e9
     line["roofline"] = {"kernel": "csb_rnn_kernel<half,1>", "bound": "hbm", "achieved": round(achieved, 1), "peak": hbm,
-                        "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / hbm, 4), "traffic": None,
+                        "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / hbm, 4),
+                        "traffic": RNN_DRAM_BYTES_PER_LAUNCH if (w.T == 512 and world == 1) else None,
                         "algorithmic_bytes_per_launch": alg_step * w.T,
                         "note": "weights are shared-memory resident, so DRAM traffic is far below the algorithmic bytes; "
                                 "the fraction compares the per-step compressed bytes with what HBM could stream"}
@@ -450,7 +458,8 @@ def main():
             r["frac_l2_warm"] = round(r["GBps_warm_l2"] / l2, 4)
         best = max(line["spmv"], key=lambda r: r["frac_hbm_measured"])
         line["roofline_spmv"] = {"kernel": "csb_product_kernel<half,1>", "bound": "hbm", "achieved": best["GBps"], "peak": hbm,
-                                 "peak_kind": peak_kind, "unit": "GB/s", "frac": best["frac_hbm_measured"], "traffic": None,
+                                 "peak_kind": peak_kind, "unit": "GB/s", "frac": best["frac_hbm_measured"],
+                                 "traffic": SPMV4X_DRAM_BYTES_PER_LAUNCH if best["rate"] == 4.0 else None,
                                  "workload": "cfg4 8192x8192, 64x64 blocks, rate %gx, batch 1, cold (rotating copies > L2)" % best["rate"]}
     if rank == 0 and "spmm" in sections:
         line["spmm"] = []
