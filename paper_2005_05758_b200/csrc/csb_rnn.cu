@@ -6,7 +6,7 @@
 // rows of those units; its compressed weights stay in shared memory for the whole sequence
 // when they fit (otherwise they are re-streamed from L2 through the same bulk-copy ring as
 // the bare product).  Only h_t crosses CTAs, through global memory and one bounded grid
-// barrier per step.  Stacked layers run as a wavefront: in tick k layer l does step k - l.
+// barrier per step.  Stacked layers run as a wavefront: in tick k layer l does step k - 2 l.
 #include <algorithm>
 #include <list>
 #include <memory>
@@ -25,7 +25,7 @@ struct RnnArgs {
     const RnnCtaDesc* ctas;
     const float* x;            // [T, B, I0]
     float* y;                  // [T, B, H] or null
-    float* hbuf;               // [L][2][B][H]: h of step t lives in slot t & 1
+    float* hbuf;               // [L][4][B][H]: h of step t lives in slot t & 3 (h0 in slot 3)
     float* cstate;             // [L][B][H], in: c0, out: cT
     const float* bias[kMaxLayers];
     int in_size[kMaxLayers];
