@@ -134,27 +134,44 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
 #else
 #define CSB_WALK_LAP(i) do { } while (0)
 #endif
+    // The header and the column indices of an item are fetched one item ahead: both sit at fixed
+    // places, so the loads go out together with the rest of the previous item's loads.  A lane
+    // whose four indices lie past nk reads whatever follows (still inside the CTA's shared
+    // memory) and never uses it.
+    uint4 h = make_uint4(0u, 0u, 0u, 0u);
+    uint32_t c4 = 0u;
+    if (p < end) {
+        h = *reinterpret_cast<const uint4*>(p);
+        c4 = *reinterpret_cast<const uint32_t*>(p + 16 + 4 * gl);
+    }
     while (__any_sync(0xffffffffu, p < end)) {
-        // ---- header: a finished group reads zeros, which turns every step below into a no-op
-        uint4 h = make_uint4(0u, 0u, 0u, 0u);
-        if (p < end) h = *reinterpret_cast<const uint4*>(p);
+        // ---- header: a finished group holds zeros, which turns every step below into a no-op
         const int nk = (int)(h.x & 0xffu), mr = (int)((h.x >> 8) & 0xffu), RL = (int)((h.x >> 16) & 0xffu), S = (int)(h.x >> 24);
-        const uint32_t xbase = h.y, zbase = h.z, magic = h.w & 0xffffu, flags = h.w >> 16;
-        // item = header | quads | tail words | col_idx | row_idx: the values come first so that
-        // the 16-byte quads are aligned
-        const int nwords = nk * RL, nq = (nk >> 2) * RL;                  // all words; quad-words (4 words each)
-        const uint4* quads = reinterpret_cast<const uint4*>(p + 16);
-        const uint32_t* tailw = reinterpret_cast<const uint32_t*>(p + 16) + 4 * nq;
-        const uint8_t* cidx = p + 16 + nwords * 4;
-        const int cidx_bytes = (nk + 3) & ~3, ridx_bytes = (mr + 3) & ~3;
-        const uint8_t* ridx = cidx + cidx_bytes;
-        if (p < end) p += (16 + nwords * 4 + cidx_bytes + ridx_bytes + 15) & ~15;     // items are 16-byte aligned
+        const uint32_t xbase = h.y, zbase = h.z & 0xffffu, magic = h.z >> 16, flags = (h.w >> 16) & 0xffu;
+        const uint8_t* item = p;
+        p += 16u * (h.w & 0xffffu);
+        const uint4* quads = reinterpret_cast<const uint4*>(item + 16u * (h.w >> 24));
+        const int nq = (nk >> 2) * RL;                                    // quad-words (4 words each)
+        const uint32_t* tailw = reinterpret_cast<const uint32_t*>(quads + nq);
+        const uint8_t* ridx = item + 16 + ((nk + 3) & ~3);
+        // everything that does not depend on other loads goes out now: the next item's header and
+        // indices, this lane's row indices
+        uint4 hn = make_uint4(0u, 0u, 0u, 0u);
+        uint32_t c4n = 0u;
+        if (p < end) {
+            hn = *reinterpret_cast<const uint4*>(p);
+            c4n = *reinterpret_cast<const uint32_t*>(p + 16 + 4 * gl);
+        }
+        uint32_t rr = 0u;                                                 // this lane's R row indices, one byte each
+        if (gl < RL) rr = (R == 2) ? (uint32_t)*reinterpret_cast<const uint16_t*>(ridx + 2 * gl) : (uint32_t)ridx[gl];
         CSB_WALK_LAP(0);
 
         // ---- gather: each lane resolves four column indices at a time; indices past nk are
         // padding zeros, gather4 decides whether they may be dereferenced
-        for (int k4 = gl * 4; k4 < nk; k4 += 4 * GW)
-            gather4(xbase, *reinterpret_cast<const uint32_t*>(cidx + k4), flags, nk - k4, xg + k4 * BT);
+        if (gl * 4 < nk) gather4(xbase, c4, flags, nk - gl * 4, xg + gl * 4 * BT);
+        if (GW * 4 < kMaxNk)
+            for (int k4 = (gl + GW) * 4; k4 < nk; k4 += 4 * GW)
+                gather4(xbase, *reinterpret_cast<const uint32_t*>(item + 16 + k4), flags, nk - k4, xg + k4 * BT);
         __syncwarp();
         CSB_WALK_LAP(1);
 
@@ -237,7 +254,7 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
             float cur[R][BT];
 #pragma unroll
             for (int q = 0; q < R; ++q) {
-                const int ri = (r0 + q < mr) ? (int)ridx[r0 + q] : (int)ridx[r0];
+                const int ri = (r0 + q < mr) ? (int)((rr >> (8 * q)) & 0xffu) : (int)(rr & 0xffu);
                 zr[q] = zs + ((int)zbase + ri) * BT;
 #pragma unroll
                 for (int bt = 0; bt < BT; ++bt) cur[q][bt] = zr[q][bt];
@@ -249,6 +266,8 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
                     for (int bt = 0; bt < BT; ++bt) zr[q][bt] = cur[q][bt] + acc[q][bt];
                 }
         }
+        h = hn;
+        c4 = c4n;
         __syncwarp();
         CSB_WALK_LAP(4);
 #ifdef CSB_WALK_CLOCKS

@@ -25,14 +25,17 @@ void clear_error();
 //   chunk  = ChunkHeader (16 B), then the G sub-streams back to back
 //   sub-stream g = the items of lane group g, each aligned to 16 B
 //   item   = ItemHeader (16 B)
+//            col_idx[nk]  uint8   gather indices, relative to xbase     (padded to 4 B)
+//            row_idx[mr]  uint8   scatter indices, relative to zbase    (padded to 16 B from the item's start)
 //            values: a word is the kept rows of one kept column that one lane owns
 //                      f16: two consecutive kept rows (half2), RL = ceil(mr/2) words per column
 //                      f32: one kept row, RL = mr
 //                    (padding rows inside the last word are zero); columns 4q..4q+3 are
 //                    interleaved into 16-byte quad-words [q][w][4], the nk % 4 columns left
-//                    over follow as plain words [k][w]
-//            col_idx[nk]  uint8   gather indices, relative to xbase     (padded to 4 B)
-//            row_idx[mr]  uint8   scatter indices, relative to zbase    (item padded to 16 B)
+//                    over follow as plain words [k][w]                  (item padded to 16 B)
+//
+// The indices sit at fixed places behind the header, so a lane can ask for them (and for the
+// next item's header) before it has looked at anything else of the item.
 //
 // An item is one block of the CSB matrix or a slice of it (a range of its kept
 // rows and of its kept columns).  Column-major kernel matrices let one lane own
@@ -44,20 +47,22 @@ struct ItemHeader {
     uint8_t RL;        // row words per column
     uint8_t S;         // column sub-groups, GW / RL
     uint32_t xbase;    // first column of the block in the gathered vector
-    uint32_t zbase;    // first accumulator slot of the block's rows
+    uint16_t zbase;    // first accumulator slot of the block's rows
     uint16_t magic;    // ceil(1024 / RL): lane / RL == (lane * magic) >> 10 for lane < 32
-    uint16_t flags;    // bit 0: columns index the recurrent (h) vector
+    uint16_t size16;   // size of the item in 16-byte units
+    uint8_t flags;     // bit 0: columns index the recurrent (h) vector
+    uint8_t voff16;    // where the values start, in 16-byte units from the item's start
 };
 static_assert(sizeof(ItemHeader) == 16, "header is one 16-byte word");
 
 struct ChunkHeader {
     uint16_t sub16[4]; // size of each lane group's sub-stream in 16-byte units
     uint32_t zbase;    // product: first matrix row of the block-row this chunk belongs to
-    uint32_t tail;     // bits 0..1 flush kind, bits 3.. partial-sum slot
+    uint32_t tail;     // bits 0..1 flush kind, bit 2 with kFlushCta: the CTA holds a piece only, bits 3.. partial-sum slot
 };
 static_assert(sizeof(ChunkHeader) == 16, "header is one 16-byte word");
 
-enum : uint32_t { kFlushNone = 0, kFlushDirect = 1, kFlushPartial = 2, kFlushCta = 3, kSlotShift = 3 };
+enum : uint32_t { kFlushNone = 0, kFlushDirect = 1, kFlushPartial = 2, kFlushCta = 3, kFlushCtaPartial = 4, kSlotShift = 3 };
 enum : uint16_t { kItemRecurrent = 1 };
 enum { kMaxNk = 64, kItemAlign = 16, kMmaMaxNk = 32 };
 
@@ -79,7 +84,7 @@ struct StreamPlan {
 // Planned product (SpMV / SpMM) on the device.
 struct ProductPlan {
     int ctas = 0, warps = 0, stage_bytes = 0, stages = 0, group_width = 32;
-    int row_owned = 0;                     // every block-row belongs to one CTA: launch shape is fixed
+    int row_owned = 0;                     // CTA-run schedule (block-rows reduced per CTA): launch shape is fixed
     int x_in_smem = 0;
     size_t smem_bytes = 0;
     uint8_t* d_stream = nullptr;

@@ -22,9 +22,13 @@ static inline int row_words(const csb_matrix* A, int mr) {
     return (mr + rpw - 1) / rpw;
 }
 
+static inline size_t item_values_offset(int nk, int mr) {
+    return pad_to(sizeof(ItemHeader) + pad_to((size_t)nk, 4) + pad_to((size_t)mr, 4), kItemAlign);
+}
+
 size_t item_bytes(const csb_matrix* A, const ItemSpec& it) {
     const int nk = it.k1 - it.k0, mr = it.r1 - it.r0;
-    return pad_to(sizeof(ItemHeader) + pad_to((size_t)nk, 4) + pad_to((size_t)mr, 4) + (size_t)nk * row_words(A, mr) * 4, kItemAlign);
+    return pad_to(item_values_offset(nk, mr) + (size_t)nk * row_words(A, mr) * 4, kItemAlign);
 }
 
 // Lock-step cost of an item for a lane group of width gw (unit: about nine instructions), from
@@ -51,13 +55,18 @@ void emit_item(const csb_matrix* A, const ItemSpec& it, int gw, std::vector<uint
     uint8_t* p = out.data() + base;
     ItemHeader h{};
     h.nk = (uint8_t)nk; h.mr = (uint8_t)mr; h.RL = (uint8_t)RL; h.S = (uint8_t)(gw / std::max(RL, 1));
-    h.xbase = it.xbase; h.zbase = it.zbase; h.magic = (uint16_t)((1024 + RL - 1) / std::max(RL, 1)); h.flags = it.flags;
+    h.xbase = it.xbase; h.zbase = (uint16_t)it.zbase; h.magic = (uint16_t)((1024 + RL - 1) / std::max(RL, 1));
+    h.size16 = (uint16_t)(item_bytes(A, it) / 16); h.flags = (uint8_t)it.flags; h.voff16 = (uint8_t)(item_values_offset(nk, mr) / 16);
     std::memcpy(p, &h, sizeof h);
-    p += sizeof h;
     const uint8_t* ci = A->col_idx.data() + A->cidx_off[it.block];
     const uint8_t* ri = A->row_idx.data() + A->ridx_off[it.block];
     const int n = A->n[it.block];
     const uint8_t* v = A->val.data() + A->val_off[it.block] * vs;
+    uint8_t* idx = p + sizeof h;
+    for (int k = 0; k < nk; ++k) idx[k] = ci[it.k0 + k];
+    idx += pad_to((size_t)nk, 4);
+    for (int r = 0; r < mr; ++r) idx[r] = (uint8_t)(ri[it.r0 + r] - it.ridx_bias);
+    p += item_values_offset(nk, mr);
     // word (k, w) = kept rows w*rpw .. of kept column k.  Columns 4q..4q+3 are interleaved into
     // quad-words [q][w][4]; the nk % 4 columns left over follow as [k][w].
     const int nquad = nk / 4;
@@ -71,16 +80,12 @@ void emit_item(const csb_matrix* A, const ItemSpec& it, int gw, std::vector<uint
                 const int r = it.r0 + w * rpw + q;
                 if (r < it.r1) std::memcpy(word_at(k, w) + q * vs, v + ((size_t)r * n + it.k0 + k) * vs, vs);
             }
-    p += (size_t)nk * RL * 4;
-    for (int k = 0; k < nk; ++k) p[k] = ci[it.k0 + k];
-    p += pad_to((size_t)nk, 4);
-    for (int r = 0; r < mr; ++r) p[r] = (uint8_t)(ri[it.r0 + r] - it.ridx_bias);
 }
 
 // Largest value payload of one item so that a chunk can hold one item per lane group.
 int item_value_budget(int stage_bytes, int gw) {
     const int G = 32 / gw;
-    return std::max(128, (stage_bytes - 16) / G - 16 - 2 * kMaxNk - 16);
+    return std::max(128, (stage_bytes - 16) / G - 16 - 2 * kMaxNk - 32);
 }
 
 // The narrowest lane group that still fits four out of five items without row slicing.

@@ -47,14 +47,15 @@ __host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t
 
 // Shared-memory carve-up, identical on host and device.
 struct ProductSmem {
-    size_t ring, bars, xbar, zs, xg, xs, total;
+    size_t ring, bars, xbar, flag, zs, xg, xs, total;
     int zs_stride;                                     // floats per lane group
     __host__ __device__ ProductSmem(int W, int G, int stages, int stage_bytes, int block_r, int BT, int cols_in_smem) {
         zs_stride = block_r * BT + group_pad(32 / G);
         ring = 0;
         bars = ring + (size_t)W * stages * stage_bytes;
         xbar = bars + (size_t)W * stages * 8;
-        zs = align16(xbar + 8);
+        flag = xbar + 8;                               // one word: did this CTA arrive last at a divided block-row
+        zs = align16(flag + 8);
         xg = align16(zs + (size_t)W * G * zs_stride * 4);
         xs = align16(xg + (size_t)W * G * xg_stride(32 / G, BT) * 4);
         total = align16(xs + (size_t)cols_in_smem * 4);
@@ -114,9 +115,11 @@ __device__ __forceinline__ void flush_block_row(const ProductArgs& a, float* zs,
 // End of a block-row that one CTA owns (all its warps are past the barrier): add the private
 // sums of every warp and lane group in a fixed order and store y.  `parts` adjacent lanes share
 // one output, each adds every parts-th copy, a fixed xor-tree joins them.
+// When the CTA holds only a piece of the block-row (`partial` points at its slot), the sums go
+// there instead, each thread fencing what it wrote.
 template <int BT>
 __device__ __forceinline__ void cta_flush_block_row(const ProductArgs& a, const float* zs_all, int zs_stride, int copies,
-                                                    uint32_t zbase) {
+                                                    uint32_t zbase, float* partial) {
     const int nrows = min(a.block_r, a.rows - (int)zbase);
     const int NZ = nrows * BT;
     int parts = 1;
@@ -138,9 +141,33 @@ __device__ __forceinline__ void cta_flush_block_row(const ProductArgs& a, const 
         for (int off = parts >> 1; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
         if (e < NZ && pt == 0) {
             const int r = e / BT, bt = e % BT;
-            if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = sum;
+            if (partial) { __stcg(partial + e, sum); __threadfence(); }
+            else if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = sum;
         }
     }
+}
+
+// The CTA that arrived last at a divided block-row adds the pieces in slot order and stores y.
+template <int BT>
+__device__ __forceinline__ void cta_join_block_row(const ProductArgs& a, uint32_t zbase) {
+    const int nrows = min(a.block_r, a.rows - (int)zbase);
+    const uint32_t bi = zbase / (uint32_t)a.block_r;
+    const uint32_t pb = a.part_base[bi], pc = a.part_count[bi];
+    const size_t pstride = (size_t)a.block_r * BT;
+    for (int e = threadIdx.x; e < nrows * BT; e += blockDim.x) {
+        const float* src = a.partials + (size_t)pb * pstride + e;
+        float sum = 0.f;
+        for (uint32_t q = 0; q < pc; q += 4) {
+            float v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = (q + j < pc) ? __ldcg(src + (size_t)(q + j) * pstride) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) sum += v[j];
+        }
+        const int r = e / BT, bt = e % BT;
+        if (bt < a.nb) a.Y[(long long)bt * a.ldy + zbase + r] = sum;
+    }
+    if (threadIdx.x == 0) a.arrivals[bi] = 0u;         // ready for the next launch
 }
 
 template <typename T, int BT, int GW>
@@ -231,7 +258,7 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
             }
         }
         if (dead) {
-            if (flush == kFlushCta) { __syncthreads(); __syncthreads(); }
+            if (flush == kFlushCta) { __syncthreads(); __syncthreads(); __syncthreads(); }
             cur = nxt;
             continue;
         }
@@ -273,10 +300,25 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
 #endif
         if (flush == kFlushCta) {
             // the CTA owns this block-row: every warp is here with its last chunk of it
+            // (three barriers whether the block-row is whole or a piece, so that a warp that gave
+            // up on its copies can keep step without reading the chunk)
+            volatile uint32_t* s_last = reinterpret_cast<volatile uint32_t*>(smem + L.flag);
+            const bool piece = (ch.w & kFlushCtaPartial) != 0;
             __syncthreads();
-            cta_flush_block_row<BT>(a, reinterpret_cast<const float*>(smem + L.zs), L.zs_stride, W * G, ch.z);
+            cta_flush_block_row<BT>(a, reinterpret_cast<const float*>(smem + L.zs), L.zs_stride, W * G, ch.z,
+                                    piece ? a.partials + (size_t)(ch.w >> kSlotShift) * a.block_r * BT : nullptr);
             __syncthreads();
             for (int i = lane; i < G * L.zs_stride; i += 32) zs[i] = 0.f;
+            if (piece && threadIdx.x == 0) {
+                const uint32_t bi = ch.z / (uint32_t)a.block_r;
+                __threadfence();
+                *s_last = (atomicAdd(&a.arrivals[bi], 1u) == a.part_count[bi] - 1u) ? 1u : 0u;
+            }
+            __syncthreads();
+            if (piece && *s_last) {
+                __threadfence();
+                cta_join_block_row<BT>(a, ch.z);
+            }
             __syncwarp();
         } else if (flush != kFlushNone) {
             flush_block_row<BT, G>(a, zs, L.zs_stride, ch.z, ch.w, lane);

@@ -1,5 +1,7 @@
 // Block -> warp schedules for the two kernels (host side, run once per matrix / stack).
 #include <algorithm>
+#include <cmath>
+#include <cstdio>
 #include <cstdlib>
 
 #include "csb_internal.hpp"
@@ -47,45 +49,114 @@ int plan_product_host(const csb_matrix* A, int ctas, int warps_per_cta, int64_t 
     double total = 0;
     for (size_t i = 0; i < items.size(); ++i) { cost[i] = placeholder[i] ? 4.0 : (double)item_steps(A, items[i], gw); total += cost[i]; }
 
-    // Row-owned mode: with about as many block-rows as CTAs (or more), every block-row belongs to
-    // ONE CTA, whose warps share its items and add their sums up in shared memory behind a CTA
-    // barrier: no partial sums in global memory, no fences, no arrival counters.
+    // Row-owned mode: with about as many block-rows as CTAs (or more), a block-row belongs to ONE
+    // CTA, whose warps share its items and add their sums up in shared memory behind a CTA
+    // barrier: no partial sums in global memory, no fences, no arrival counters.  Only a
+    // block-row so heavy that it alone would set the run time is divided into pieces for several
+    // CTAs; each piece leaves its CTA as one partial sum, and the CTA that arrives last adds them.
     const char* ro_env = getenv("CSB_ROW_OWNED");
     const bool row_owned = ro_env && *ro_env ? atoi(ro_env) != 0 : (A->nbr * 5 >= (int64_t)ctas * 4 && n_warps >= ctas);
     if (row_owned) {
         const int G = 32 / gw;
-        const int n_ctas = (int)std::min<int64_t>(ctas, A->nbr);
+        const int n_ctas = ctas;
         // warps per CTA: enough lane groups for the items of a typical block-row, no more
         const double items_per_row = (double)items.size() / (double)A->nbr;
         const int wpc = std::max(1, std::min(warps_per_cta, (int)(items_per_row / G / 2.0 + 0.999)));
-        // block-rows to CTAs: heaviest first onto the least loaded CTA
-        std::vector<double> row_cost(A->nbr, 0.0);
+        // Costs in the time of one CTA (its items spread over wpc * G lane groups): a piece also
+        // costs a barrier and a reduction, a divided block-row the round trips of the exchange.
+        const double kFlush = 16.0, kExchange = 70.0;
+        const char* split_env = getenv("CSB_ROW_SPLIT");
+        const bool may_split = !(split_env && *split_env && atoi(split_env) == 0);
+        const double bins = (double)wpc * G;
         std::vector<size_t> row_begin(A->nbr + 1, items.size());
-        for (size_t i = items.size(); i-- > 0;) { row_cost[item_row[i]] += cost[i] + 1.0; row_begin[item_row[i]] = i; }
-        std::vector<int64_t> order(A->nbr);
-        for (int64_t i = 0; i < A->nbr; ++i) order[i] = i;
-        std::stable_sort(order.begin(), order.end(), [&](int64_t x, int64_t y) { return row_cost[x] > row_cost[y]; });
-        std::vector<double> cta_load(n_ctas, 0.0);
-        std::vector<std::vector<int64_t>> cta_rows(n_ctas);
-        for (int64_t bi : order) {
-            const int c = (int)(std::min_element(cta_load.begin(), cta_load.end()) - cta_load.begin());
-            cta_rows[c].push_back(bi);
-            cta_load[c] += row_cost[bi] / (wpc * G) + 60.0;      // a block-row also costs a CTA barrier and a reduction
+        std::vector<double> row_cost(A->nbr, 0.0);
+        for (size_t i = items.size(); i-- > 0;) { row_cost[item_row[i]] += cost[i] / bins; row_begin[item_row[i]] = i; }
+        struct Piece { int64_t row; int k, of; double cost; };
+        auto make_pieces = [&](double T, std::vector<Piece>* out_pieces) {
+            out_pieces->clear();
+            for (int64_t bi = 0; bi < A->nbr; ++bi) {
+                int p = 1;
+                const double room = T - kFlush - kExchange;
+                if (may_split && row_cost[bi] + kFlush > T && room > 0) p = (int)std::ceil(row_cost[bi] / room);
+                const int n_items = (int)(row_begin[bi + 1] - row_begin[bi]);
+                p = std::max(1, std::min(p, std::min(n_items, 64)));
+                for (int k = 0; k < p; ++k)
+                    out_pieces->push_back({bi, k, p, row_cost[bi] / p + kFlush + (p > 1 ? kExchange : 0.0)});
+            }
+        };
+        auto pack = [&](const std::vector<Piece>& pcs, std::vector<int>* where) {
+            // heaviest piece first onto the least loaded CTA; returns the largest load
+            std::vector<size_t> order(pcs.size());
+            for (size_t i = 0; i < order.size(); ++i) order[i] = i;
+            std::stable_sort(order.begin(), order.end(), [&](size_t x, size_t y) { return pcs[x].cost > pcs[y].cost; });
+            std::vector<double> load(n_ctas, 0.0);
+            where->assign(pcs.size(), 0);
+            for (size_t i : order) {
+                const int c = (int)(std::min_element(load.begin(), load.end()) - load.begin());
+                (*where)[i] = c;
+                load[c] += pcs[i].cost;
+            }
+            return *std::max_element(load.begin(), load.end());
+        };
+        // the target time T decides which block-rows are divided; try a ladder of targets between
+        // the even share and the heaviest block-row and keep the best packing
+        double sum_cost = 0, max_cost = 0;
+        for (double c : row_cost) { sum_cost += c + kFlush; max_cost = std::max(max_cost, c + kFlush); }
+        const double lo = std::max(sum_cost / n_ctas, 1.0);
+        std::vector<Piece> pieces, best_pieces;
+        std::vector<int> where, best_where;
+        double best = -1, undivided = 0;
+        for (int step = 0; step <= 24; ++step) {
+            // step 0 divides nothing; a division has to pay for itself with some margin
+            const double T = max_cost <= lo ? max_cost : lo * std::pow(max_cost / lo, (24 - step) / 24.0);
+            make_pieces(T, &pieces);
+            const double mk = pack(pieces, &where);
+            if (step == 0) undivided = mk;
+            if (getenv("CSB_PLAN_DEBUG")) fprintf(stderr, "T=%.1f pieces=%zu makespan=%.1f lo=%.1f max=%.1f\n", T, pieces.size(), mk, lo, max_cost);
+            if (best < 0 || (mk < best && mk < 0.95 * undivided)) { best = mk; best_pieces = pieces; best_where = where; }
+            if (max_cost <= lo) break;
         }
-        std::vector<std::vector<Segment>> per_warp((size_t)n_ctas * wpc);
-        for (int c = 0; c < n_ctas; ++c) {
-            for (int64_t bi : cta_rows[c]) {
-                // this block-row's items, dealt longest first to the CTA's lane groups
+        // slots of the divided block-rows
+        out->part_base.assign(A->nbr, 0);
+        out->part_count.assign(A->nbr, 0);
+        uint32_t slots = 0;
+        for (const Piece& pc : best_pieces)
+            if (pc.of > 1 && pc.k == 0) { out->part_base[pc.row] = slots; out->part_count[pc.row] = (uint32_t)pc.of; slots += (uint32_t)pc.of; }
+        out->n_slots = slots;
+        // per CTA: its pieces, divided ones first (their partner may be waiting), then by row
+        std::vector<std::vector<size_t>> cta_pieces(n_ctas);
+        int n_used = 1;                                          // the packing fills CTAs from the front
+        for (size_t i = 0; i < best_pieces.size(); ++i) { cta_pieces[best_where[i]].push_back(i); n_used = std::max(n_used, best_where[i] + 1); }
+        std::vector<std::vector<Segment>> per_warp((size_t)n_used * wpc);
+        std::vector<double> cta_load(n_ctas, 0.0);
+        for (int c = 0; c < n_used; ++c) {
+            std::stable_sort(cta_pieces[c].begin(), cta_pieces[c].end(), [&](size_t x, size_t y) {
+                return (best_pieces[x].of > 1) > (best_pieces[y].of > 1);
+            });
+            for (size_t pi : cta_pieces[c]) {
+                const Piece& pc = best_pieces[pi];
+                cta_load[c] += pc.cost;
+                const int64_t bi = pc.row;
+                // the piece's items: a contiguous range of the block-row, cut by cost
                 std::vector<size_t> idx;
-                for (size_t i = row_begin[bi]; i < row_begin[bi + 1] && i < items.size() && item_row[i] == bi; ++i)
-                    if (!placeholder[i]) idx.push_back(i);
+                {
+                    double cum = 0;
+                    const double tot = row_cost[bi] * bins;
+                    for (size_t i = row_begin[bi]; i < row_begin[bi + 1]; ++i) {
+                        const int k = tot > 0 ? std::min(pc.of - 1, (int)((cum + 0.5 * cost[i]) / tot * pc.of)) : 0;
+                        if (k == pc.k && !placeholder[i]) idx.push_back(i);
+                        cum += cost[i];
+                    }
+                }
+                const uint32_t tail = pc.of > 1 ? (kFlushCta | kFlushCtaPartial | ((out->part_base[bi] + (uint32_t)pc.k) << kSlotShift))
+                                                : (uint32_t)kFlushCta;
                 std::stable_sort(idx.begin(), idx.end(), [&](size_t x, size_t y) { return cost[x] > cost[y]; });
                 std::vector<double> load((size_t)wpc * G, 0.0);
                 for (int w = 0; w < wpc; ++w) {
                     per_warp[(size_t)c * wpc + w].emplace_back();
                     Segment& sg = per_warp[(size_t)c * wpc + w].back();
                     sg.zbase = (uint32_t)(bi * A->block_r);
-                    sg.tail = kFlushCta;
+                    sg.tail = tail;
                 }
                 for (size_t i : idx) {
                     const int bin = (int)(std::min_element(load.begin(), load.end()) - load.begin());
@@ -94,14 +165,11 @@ int plan_product_host(const csb_matrix* A, int ctas, int warps_per_cta, int64_t 
                 }
             }
         }
-        out->part_base.assign(A->nbr, 0);
-        out->part_count.assign(A->nbr, 0);
-        out->n_slots = 0;
-        out->row_owned = 1; out->ctas = n_ctas; out->warps_per_cta = wpc;
+        out->row_owned = 1; out->ctas = n_used; out->warps_per_cta = wpc;
         build_stream(A, per_warp, stage_bytes, &out->stream);
         double mx = 0, sum = 0;
         for (double l : cta_load) { mx = std::max(mx, l); sum += l; }
-        out->balance = mx > 0 ? sum / ctas / mx : 1.0;           // idle CTAs count against the balance
+        out->balance = mx > 0 ? sum / n_ctas / mx : 1.0;         // idle CTAs count against the balance
         return CSB_OK;
     }
 

@@ -78,6 +78,22 @@ def test_rows_kept_nowhere_and_empty_block_rows():
     run_case(mat, rng.standard_normal((4, C)).astype(np.float32))
 
 
+@pytest.mark.parametrize("B", [1, 3])
+def test_heavy_block_row_is_divided_between_ctas(B):
+    # one block-row keeps everything, the others about a tenth: the planner divides the heavy one
+    # into pieces for several CTAs, which meet through partial sums; result and bit-reproducibility
+    # as everywhere else
+    w = workloads.make_spmv_workload(11, 8192, 4096, 64, 64, "lognormal", rate=10.0, batch=B, w_std=0.05)
+    m = w.matrix
+    m.row_keep.reshape(128, 64, 64)[5] = 1
+    m.col_keep.reshape(128, 64, 64)[5] = 1
+    info = run_case(m, w.X)
+    A = binding.csb_encode(m.dense, 64, 64, m.row_keep, m.col_keep, "f16", device=-1)
+    plan = binding.csb_plan_dump(A, info["plan_ctas"], 16, 4096)
+    A.free()
+    assert info["plan_ctas"] > 128 and plan["row_owned"] and plan["slots"] >= 2, "the case must exercise divided block-rows"
+
+
 @pytest.mark.parametrize("opts", [dict(ctas=1, warps_per_cta=1), dict(ctas=3, warps_per_cta=5, stages=1),
                                   dict(ctas=148, warps_per_cta=16, stage_bytes=1024, stages=2), dict(ctas=500)])
 def test_schedules_agree(opts):
