@@ -235,6 +235,24 @@ int csb_plan_dump(const csb_matrix_t* A, int ctas, int warps_per_cta, int stage_
                   uint8_t* stream_out, int64_t stream_cap, uint32_t* chunks_out, int64_t chunks_cap,
                   uint32_t* warp_begin_out, int64_t warp_cap);
 
+/*
+ * csb_panel_dump -- inspection / testing aid (the paper has no counterpart): plan the panel layout
+ * that csb_spmv streams for fp16 matrices (one panel per CTA, which owns a contiguous range of
+ * output rows: bookkeeping, then the re-tiled kernel-matrix rows), on the host only, and copy it
+ * out so that layout and schedule can be checked without a GPU.
+ *   info_out    host, int64[8]: CTAs, bytes of all panels, 0, largest bookkeeping part, largest
+ *               gathered-input count, most output rows per CTA, and the CTA-level and warp-level
+ *               balance (mean / max of the modelled cost) times 1e6.
+ *   panels_out  host, `panels_cap` bytes, or NULL;  cta_out  host, four uint32 per CTA (offset of
+ *               the panel in 16-byte units, bytes of bookkeeping, bytes of values, output rows),
+ *               `cta_cap` entries, or NULL.
+ * Errors: UNSUPPORTED when the layout does not apply (fp32 values, block_c > 128, cols > 16384,
+ * stage_bytes not a power of two >= 8192, or a panel beyond the kernel's limits), INVALID_ARG for
+ * a buffer that is too small; call once with NULL buffers to learn the sizes.
+ */
+int csb_panel_dump(const csb_matrix_t* A, int ctas, int warps_per_cta, int stage_bytes, int64_t* info_out,
+                   uint8_t* panels_out, int64_t panels_cap, uint32_t* cta_out, int64_t cta_cap);
+
 /* Short text for a status code; never NULL. */
 const char* csb_strerror(int status);
 

@@ -172,6 +172,21 @@ def csb_plan_dump(A: CsbMatrix, ctas: int, warps_per_cta: int, stage_bytes: int)
     return out
 
 
+def csb_panel_dump(A: CsbMatrix, ctas: int, warps_per_cta: int, stage_bytes: int) -> dict:
+    """Host-only plan of the batch-1 panel layout, copied out for inspection (see csb.h)."""
+    lib.csb_panel_dump.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, C.c_int64, _P, C.c_int64]
+    lib.csb_panel_dump.restype = C.c_int
+    info = np.zeros(8, np.int64)
+    _check(lib.csb_panel_dump(A.handle, ctas, warps_per_cta, stage_bytes, info.ctypes.data, None, 0, None, 0))
+    panels = np.zeros(max(int(info[1]), 1), np.uint8)
+    cta = np.zeros((max(int(info[0]), 1), 4), np.uint32)
+    _check(lib.csb_panel_dump(A.handle, ctas, warps_per_cta, stage_bytes, info.ctypes.data, panels.ctypes.data, panels.size,
+                              cta.ctypes.data, cta.shape[0]))
+    return {"ctas": int(info[0]), "bytes": int(info[1]), "max_meta": int(info[3]),
+            "max_xg": int(info[4]), "max_rows": int(info[5]), "balance": info[6] / 1e6, "warp_balance": info[7] / 1e6,
+            "panels": panels[: int(info[1])], "cta": cta[: int(info[0])]}
+
+
 def csb_spmv(A: CsbMatrix, x, y, stream=None) -> None:
     _check(lib.csb_spmv(A.handle, _ptr(x), _ptr(y), _stream(stream)))
 

@@ -63,7 +63,7 @@ int csb_encode(const float* dense, int64_t rows, int64_t cols, int64_t ld, int b
     int rc = encode_host(dense, rows, cols, ld, block_r, block_c, row_keep, col_keep, val_dtype, A);
     if (rc == CSB_OK) rc = validate_host(A);
     if (rc == CSB_OK && device >= 0) {
-        try { rc = plan_product(A); }
+        try { rc = plan_product(A); if (rc == CSB_OK) rc = plan_panels(A); }
         catch (const std::bad_alloc&) { set_error("out of host memory while planning"); rc = CSB_ERR_ALLOC; }
     }
     if (rc != CSB_OK) { csb_free(A); return rc; }
@@ -129,10 +129,38 @@ int csb_plan_dump(const csb_matrix_t* A, int ctas, int warps_per_cta, int stage_
     return CSB_OK;
 }
 
+int csb_panel_dump(const csb_matrix_t* A, int ctas, int warps_per_cta, int stage_bytes, int64_t* info_out,
+                   uint8_t* panels_out, int64_t panels_cap, uint32_t* cta_out, int64_t cta_cap) {
+    clear_error();
+    if (!A || !info_out || ctas < 1 || warps_per_cta < 1 || warps_per_cta > 32) { set_error("csb_panel_dump: bad argument"); return CSB_ERR_INVALID_ARG; }
+    PanelHostPlan H;
+    int rc;
+    try { rc = plan_panels_host(A, ctas, warps_per_cta, stage_bytes, 16384, 8192 / warps_per_cta, &H); }
+    catch (const std::bad_alloc&) { set_error("out of host memory while planning"); return CSB_ERR_ALLOC; }
+    if (rc == 1) { set_error("the panel layout does not apply to this matrix (fp16 values, block_c <= 128, cols <= 16384, power-of-two stage >= 8192)"); return CSB_ERR_UNSUPPORTED; }
+    if (rc != CSB_OK) return rc;
+    info_out[0] = (int64_t)H.cta.size(); info_out[1] = (int64_t)H.bytes.size(); info_out[2] = 0;
+    info_out[3] = (int64_t)H.max_meta; info_out[4] = (int64_t)H.max_xg; info_out[5] = (int64_t)H.max_rows;
+    info_out[6] = (int64_t)(H.balance * 1e6); info_out[7] = (int64_t)(H.warp_balance * 1e6);
+    if (panels_out) {
+        if (panels_cap < (int64_t)H.bytes.size()) { set_error("panel buffer too small"); return CSB_ERR_INVALID_ARG; }
+        std::memcpy(panels_out, H.bytes.data(), H.bytes.size());
+    }
+    if (cta_out) {
+        if (cta_cap < (int64_t)H.cta.size()) { set_error("CTA table too small"); return CSB_ERR_INVALID_ARG; }
+        for (size_t c = 0; c < H.cta.size(); ++c) {
+            cta_out[4 * c] = H.cta[c].off16; cta_out[4 * c + 1] = H.cta[c].meta_bytes;
+            cta_out[4 * c + 2] = H.cta[c].value_bytes; cta_out[4 * c + 3] = H.cta[c].n_rows;
+        }
+    }
+    return CSB_OK;
+}
+
 void csb_free(csb_matrix_t* A) {
     if (!A) return;
     drop_rnn_plans(A);
     free_mma(A);
+    free_panels(A);
     free_product(A);
     delete A;
 }
@@ -149,6 +177,7 @@ int csb_spmm(const csb_matrix_t* A, const float* X, int64_t ldx, int batch, floa
         const int rc = launch_spmm_mma(A, X, ldx, batch, Y, ldy, stream);
         if (rc != 1) return rc;                       // 1: the tensor-core plan does not fit this matrix
     }
+    if (batch == 1 && A->panel && A->panel->built) return launch_panels(A, X, Y, stream);
     return launch_product(A, X, ldx, batch, Y, ldy, stream);
 }
 

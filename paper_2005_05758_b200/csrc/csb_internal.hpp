@@ -106,6 +106,7 @@ struct ProductPlan {
 struct Planner;                            // csb_plan.cpp
 struct RnnPlan;                            // csb_rnn.cu
 struct MmaPlan;                            // tensor-core SpMM plan (below)
+struct PanelPlan;                          // panel layout of the batch-1 product (below)
 
 }  // namespace csb
 
@@ -127,6 +128,7 @@ struct csb_matrix {
     csb::ProductPlan product;
     mutable csb::MmaPlan* mma = nullptr;   // tensor-core SpMM plan, built lazily
     mutable std::mutex mma_mu;
+    csb::PanelPlan* panel = nullptr;       // panel layout for batch 1 (fp16 values), or NULL
     int sm_count = 0;
     size_t smem_optin = 0;
     uint64_t uid = 0;                      // identity for the recurrent-plan cache
@@ -221,6 +223,56 @@ struct MmaPlan {                           // device side, built on the first ba
 int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream);
 bool spmm_mma_applicable(const csb_matrix* A, int batch);
 void free_mma(csb_matrix* A);
+
+// ---- panel layout of the batch-1 product (csb_panel_plan.cpp, csb_panel.cu) ----
+enum { kMaxPanelCtas = 192 };
+struct PanelItem {          // one item: up to 32 kept rows of a block, all its kept columns
+    uint32_t off16;         // where its values start in the panel's value stream, 16-byte units
+    uint16_t xoff4;         // the block's gathered inputs, in units of four floats
+    int16_t zoff;           // block-row's first row minus the panel's first row (may be negative)
+    uint16_t roff;          // the item's row indices (in-block, one byte each) inside the panel's index bytes
+    uint8_t m;              // kept rows in the item, 1..32
+    uint8_t logp;           // log2 of the lane stride P, the smallest power of two >= m
+    uint16_t n;             // kept columns, 1..block_c
+    uint16_t pad;
+};
+static_assert(sizeof(PanelItem) == 16, "descriptor is one 16-byte word");
+struct PanelGather {        // one block whose kept inputs the CTA gathers
+    uint16_t xbase;         // first column of the block
+    uint16_t n;             // kept columns
+    uint32_t xoff;          // where its indices (bytes) and its gathered inputs (floats) start; multiple of 4
+};
+static_assert(sizeof(PanelGather) == 8, "two per 16-byte word");
+struct PanelHeader {        // start of a panel's meta part; offsets are from the panel's start
+    uint32_t n_items, n_gather, n_xg, n_stages;
+    uint32_t value_bytes, ridx_bytes, row0, n_rows;
+    uint32_t warp_off, items_off, gather_off, expect_off;
+    uint32_t cidx_off, ridx_off, pad[2];
+};
+static_assert(sizeof(PanelHeader) == 64, "header is four 16-byte words");
+struct PanelCta { uint32_t off16, meta_bytes, value_bytes, n_rows; };
+struct PanelHostPlan {
+    std::vector<uint8_t> bytes;            // all panels, each aligned to 128 bytes
+    std::vector<PanelCta> cta;
+    int warps = 0, stage_bytes = 0;
+    size_t max_meta = 0, max_xg = 0, max_rows = 0;
+    double balance = 1.0, warp_balance = 1.0;
+};
+// Returns CSB_OK, or 1 when the matrix does not suit the panel path (the caller keeps the other one).
+int plan_panels_host(const csb_matrix* A, int ctas, int warps, int stage_bytes, int max_xg_floats, int max_rows,
+                     PanelHostPlan* out);
+struct PanelPlan {                         // device side
+    bool built = false;
+    int ctas = 0, warps = 0, stage_bytes = 0, log2_ring = 0, max_rows = 0, max_xg = 0, max_meta = 0;
+    size_t smem_bytes = 0;
+    uint8_t* d_panels = nullptr;
+    std::vector<PanelCta> cta;
+    int64_t stream_bytes = 0;
+    double balance = 1.0, warp_balance = 1.0;
+};
+int plan_panels(csb_matrix* A);            // after plan_product; leaves A->panel NULL when the path does not apply
+void free_panels(csb_matrix* A);
+int launch_panels(const csb_matrix* A, const float* x, float* y, void* stream);
 
 // csb_product.cu
 int plan_product(csb_matrix* A);           // plans, uploads, fills A->product

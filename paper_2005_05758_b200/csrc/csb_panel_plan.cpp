@@ -1,0 +1,265 @@
+// Host planner of the panel layout: the device form of a CSB matrix that the batch-1
+// product (SpMV) streams.
+//
+// The paper's CSB-Engine walks the blocks of a matrix in row-major order and hides their
+// uneven sizes with compile-time workload sharing (Sections 4.3.1, 5.2).  Here the output
+// rows are cut into one contiguous range per CTA of a persistent grid, of about equal modelled
+// cost, and a CTA gets everything that lands in its rows: of every block that has kept rows in
+// the range, those rows with all the block's kept columns.  Ranges do not follow block-row
+// borders (a block-row's kept rows may go to two or more CTAs), so every output row is written
+// by exactly one CTA and nothing has to be joined across CTAs.  What a CTA streams is a *panel*:
+//
+//   meta    PanelHeader, per-warp item ranges, item descriptors, gather descriptors, per-stage
+//           item counts, column indices, row indices
+//   values  the kernel-matrix rows of the panel's items back to back, fetched by the CTA in
+//           fixed-size stages through one shared-memory ring
+//
+// An item is at most 32 kept rows of one block with all its kept columns.  Its values are the
+// canonical row-major kernel-matrix rows re-tiled so that a lane reads 16 bytes = 8 consecutive
+// kept columns of one kept row: [octet o][row r][8], then the 4-, 2- and 1-column remainders
+// as [r][4], [r][2], [r][1].  No padding inside an item; items are padded to 16 bytes.
+//
+// The gathered input of a block (its kept columns of x) is built once per CTA in shared
+// memory, so the multiply loop reads it with vector loads.  A panel's items are laid out
+// longest first and dealt to the CTA's warps in that order, each to the warp with the least
+// work so far; the deal is part of the plan, so the summation order is fixed.
+#include <algorithm>
+#include <cstdlib>
+
+#include "csb_internal.hpp"
+
+namespace csb {
+
+static inline size_t pad_to(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline int log2_ceil(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
+
+// Modelled time of one item on one SM, in issue slots of one warp: a fixed part per item, the
+// octet steps of the multiply loop, the remainder columns and the joining shuffles.
+static double panel_item_cost(int mi, int n) {
+    const int S = 32 >> log2_ceil(mi);
+    const int steps = ((n >> 3) + S - 1) / S;
+    return 110.0 + 19.0 * steps + ((n & 7) ? 25.0 : 0.0) + 3.0 * log2_ceil(S);
+}
+
+struct PanelItemSrc {
+    int64_t block;
+    int r0, mi;            // kept-row range [r0, r0 + mi) of the block's kept-row list
+    size_t bytes;          // padded value bytes
+    double cost;
+    uint32_t xoff;         // the block's place in the gathered inputs
+};
+
+int plan_panels_host(const csb_matrix* A, int ctas, int warps, int stage_bytes, int max_xg_floats, int max_rows,
+                     PanelHostPlan* out) {
+    *out = PanelHostPlan{};
+    if (A->val_dtype != CSB_F16) return 1;
+    if (A->block_c > 128 || A->cols > 16384) return 1;
+    if (stage_bytes < 8192 || (stage_bytes & (stage_bytes - 1))) return 1;
+    const int BR = A->block_r, BC = A->block_c;
+
+    // ---- which blocks keep a given output row (blocks without kept columns store nothing)
+    std::vector<uint32_t> rb_begin(A->rows + 1, 0);
+    size_t total_bytes = 0;
+    for (int64_t b = 0; b < A->nblk; ++b) {
+        const int m = A->m[b], n = A->n[b];
+        if (m == 0 || n == 0) continue;
+        const uint8_t* ri = A->row_idx.data() + A->ridx_off[b];
+        for (int r = 0; r < m; ++r) ++rb_begin[(b / A->nbc) * BR + ri[r] + 1];
+        total_bytes += (size_t)m * n * 2;
+    }
+    for (int64_t r = 0; r < A->rows; ++r) rb_begin[r + 1] += rb_begin[r];
+    std::vector<uint32_t> rb(rb_begin[A->rows]);
+    {
+        std::vector<uint32_t> fill(rb_begin.begin(), rb_begin.end() - 1);
+        for (int64_t b = 0; b < A->nblk; ++b) {
+            const int m = A->m[b], n = A->n[b];
+            if (m == 0 || n == 0) continue;
+            const uint8_t* ri = A->row_idx.data() + A->ridx_off[b];
+            for (int r = 0; r < m; ++r) rb[fill[(b / A->nbc) * BR + ri[r]]++] = (uint32_t)b;
+        }
+    }
+    int n_ctas = (int)std::min<int64_t>(ctas, std::max<int64_t>(1, (int64_t)total_bytes / 8192));
+    n_ctas = (int)std::min<int64_t>(std::min<int64_t>(n_ctas, (int64_t)kMaxPanelCtas), A->rows);
+
+    // ---- one contiguous row range per CTA.  The cost of a range is the cost of its items, and an
+    // item's fixed part is paid again by every CTA that holds rows of the block, so the cost is
+    // followed row by row: rows are packed into a CTA until a limit T would be passed, and T is
+    // the smallest limit (by bisection) that needs no more than n_ctas CTAs.
+    std::vector<uint16_t> cnt(A->nblk, 0);                 // rows of the block in the CTA being filled
+    auto block_cost = [&](int m, int n) { double c = 0.0; for (int r0 = 0; r0 < m; r0 += 32) c += panel_item_cost(std::min(32, m - r0), n); return c; };
+    auto pack = [&](double T, std::vector<int64_t>* cuts, double* worst) -> int {
+        int used = 1;
+        double cur = 0.0;
+        *worst = 0.0;
+        int64_t start = 0;
+        if (cuts) { cuts->assign(1, 0); }
+        auto reset = [&](int64_t from, int64_t to) { for (int64_t r = from; r < to; ++r) for (uint32_t i = rb_begin[r]; i < rb_begin[r + 1]; ++i) cnt[rb[i]] = 0; };
+        for (int64_t r = 0; r < A->rows; ++r) {
+            double delta = 0.0;
+            for (uint32_t i = rb_begin[r]; i < rb_begin[r + 1]; ++i) { const uint32_t b = rb[i]; delta += block_cost(cnt[b] + 1, A->n[b]) - block_cost(cnt[b], A->n[b]); }
+            if ((cur > 0.0 && cur + delta > T) || r - start >= max_rows) {
+                *worst = std::max(*worst, cur);
+                reset(start, r);
+                start = r; cur = 0.0; ++used;
+                if (cuts) cuts->push_back(r);
+                delta = 0.0;
+                for (uint32_t i = rb_begin[r]; i < rb_begin[r + 1]; ++i) delta += block_cost(1, A->n[rb[i]]);
+            }
+            for (uint32_t i = rb_begin[r]; i < rb_begin[r + 1]; ++i) ++cnt[rb[i]];
+            cur += delta;
+        }
+        *worst = std::max(*worst, cur);
+        reset(start, A->rows);
+        if (cuts) cuts->push_back(A->rows);
+        return used;
+    };
+    std::vector<int64_t> cut;
+    {
+        double worst = 0.0, lo = 0.0, hi = 0.0;
+        pack(1e300, nullptr, &hi);                         // everything in one CTA: an upper bound
+        hi = std::max(hi, 1.0);
+        for (int it = 0; it < 40 && hi - lo > 1e-3 * hi; ++it) {
+            const double mid = 0.5 * (lo + hi);
+            if (pack(mid, nullptr, &worst) <= n_ctas) hi = mid; else lo = mid;
+        }
+        n_ctas = pack(hi, &cut, &worst);
+        if (n_ctas > (int)kMaxPanelCtas) return 1;        // only when max_rows forces more ranges than the grid has
+    }
+
+    out->warps = warps;
+    out->stage_bytes = stage_bytes;
+    out->cta.resize(n_ctas);
+    double max_cta_cost = 0.0, max_warp_cost = 0.0, sum_cta_cost = 0.0;
+    for (int c = 0; c < n_ctas; ++c) {
+        const int64_t R0 = cut[c], R1 = cut[c + 1];
+        if (R1 - R0 > max_rows) return 1;
+        std::vector<PanelItemSrc> items;
+        std::vector<PanelItem> desc;
+        std::vector<PanelGather> gath;
+        std::vector<uint8_t> cidx, ridx, values;
+        for (int64_t bi = R0 / BR; bi < A->nbr && bi * BR < R1; ++bi) {
+            const int lo = (int)std::max<int64_t>(0, R0 - bi * BR), hi = (int)std::min<int64_t>(BR, R1 - bi * BR);   // in-block rows [lo, hi)
+            for (int64_t bj = 0; bj < A->nbc; ++bj) {
+                const int64_t b = bi * A->nbc + bj;
+                const int m = A->m[b], n = A->n[b];
+                if (m == 0 || n == 0) continue;
+                const uint8_t* ri = A->row_idx.data() + A->ridx_off[b];
+                const int ra = (int)(std::lower_bound(ri, ri + m, lo) - ri), rb = (int)(std::lower_bound(ri, ri + m, hi) - ri);
+                if (ra == rb) continue;
+                PanelGather g{};
+                g.xbase = (uint16_t)(bj * BC); g.n = (uint16_t)n; g.xoff = (uint32_t)cidx.size();
+                gath.push_back(g);
+                const uint8_t* ci = A->col_idx.data() + A->cidx_off[b];
+                cidx.insert(cidx.end(), ci, ci + n);
+                while (cidx.size() & 3) cidx.push_back(0);
+                for (int r0 = ra; r0 < rb; r0 += 32) {
+                    PanelItemSrc it{};
+                    it.block = b; it.r0 = r0; it.mi = std::min(32, rb - r0);
+                    it.bytes = pad_to((size_t)it.mi * n * 2, 16);
+                    it.cost = panel_item_cost(it.mi, n);
+                    it.xoff = g.xoff;
+                    items.push_back(it);
+                }
+            }
+        }
+        // The value stream holds the items longest first: dealt in that order to the least loaded
+        // warp they leave the warps with nearly equal work, and the short ones fill in at the end.
+        std::stable_sort(items.begin(), items.end(), [](const PanelItemSrc& x, const PanelItemSrc& y) { return x.cost > y.cost; });
+        for (const PanelItemSrc& it : items) {
+            const int64_t b = it.block, bi = b / A->nbc;
+            const int n = A->n[b];
+            const uint8_t* ri = A->row_idx.data() + A->ridx_off[b];
+            PanelItem d{};
+            d.off16 = (uint32_t)(values.size() / 16);
+            d.xoff4 = (uint16_t)(it.xoff / 4);
+            d.zoff = (int16_t)(bi * BR - R0);
+            d.roff = (uint16_t)ridx.size();
+            d.m = (uint8_t)it.mi; d.logp = (uint8_t)log2_ceil(it.mi);
+            d.n = (uint16_t)n; d.pad = 0;
+            ridx.insert(ridx.end(), ri + it.r0, ri + it.r0 + it.mi);
+            // values: [octet][row][8], then [row][4], [row][2], [row][1]
+            const uint8_t* v = A->val.data() + (A->val_off[b] + (uint64_t)it.r0 * n) * 2;
+            const size_t base = values.size();
+            values.resize(base + it.bytes, 0);
+            uint8_t* p = values.data() + base;
+            const int noct = n >> 3;
+            for (int o = 0; o < noct; ++o)
+                for (int r = 0; r < it.mi; ++r, p += 16) std::memcpy(p, v + ((size_t)r * n + 8 * o) * 2, 16);
+            int k = noct * 8;
+            for (int w = 4; w >= 1; w >>= 1)
+                if (n & w) {
+                    for (int r = 0; r < it.mi; ++r, p += 2 * w) std::memcpy(p, v + ((size_t)r * n + k) * 2, 2 * w);
+                    k += w;
+                }
+            desc.push_back(d);
+        }
+        if (cidx.size() > (size_t)max_xg_floats || cidx.size() / 4 > 0xffff || ridx.size() > 0xffff || items.size() > 0xffff ||
+            values.size() / 16 > 0xffffffffull)
+            return 1;                                            // beyond the kernel's limits: the caller keeps the other path
+        // items per stage (an item that straddles a boundary counts on both sides)
+        const size_t n_stages = (values.size() + stage_bytes - 1) / stage_bytes;
+        std::vector<uint16_t> expect(n_stages, 0);
+        for (size_t i = 0; i < items.size(); ++i) {
+            const size_t off = (size_t)desc[i].off16 * 16;
+            const size_t s0 = off / stage_bytes, s1 = (off + items[i].bytes - 1) / stage_bytes;
+            for (size_t s = s0; s <= s1; ++s) ++expect[s];
+        }
+        // deal items to warps in stream order, each to the least loaded warp
+        std::vector<double> load(warps, 0.0);
+        std::vector<std::vector<uint32_t>> per_warp(warps);
+        for (size_t i = 0; i < items.size(); ++i) {
+            const int w = (int)(std::min_element(load.begin(), load.end()) - load.begin());
+            per_warp[w].push_back((uint32_t)i);
+            load[w] += items[i].cost;
+        }
+        double cta_cost = 0.0;
+        for (int w = 0; w < warps; ++w) { cta_cost += load[w]; max_warp_cost = std::max(max_warp_cost, load[w]); }
+        sum_cta_cost += cta_cost;
+        max_cta_cost = std::max(max_cta_cost, cta_cost);
+
+        // ---- emit the panel
+        PanelHeader h{};
+        h.n_items = (uint32_t)items.size(); h.n_gather = (uint32_t)gath.size(); h.n_xg = (uint32_t)cidx.size();
+        h.n_stages = (uint32_t)n_stages; h.value_bytes = (uint32_t)values.size(); h.ridx_bytes = (uint32_t)ridx.size();
+        h.row0 = (uint32_t)R0; h.n_rows = (uint32_t)(R1 - R0);
+        size_t off = sizeof(PanelHeader);
+        h.warp_off = (uint32_t)off; off = pad_to(off + (size_t)(warps + 1) * 2, 16);
+        h.items_off = (uint32_t)off; off += (size_t)h.n_items * sizeof(PanelItem);
+        h.gather_off = (uint32_t)off; off = pad_to(off + gath.size() * sizeof(PanelGather), 16);
+        h.expect_off = (uint32_t)off; off = pad_to(off + n_stages * 2, 16);
+        h.cidx_off = (uint32_t)off; off = pad_to(off + cidx.size(), 16);
+        h.ridx_off = (uint32_t)off; off = pad_to(off + ridx.size(), 128);
+        const size_t meta_bytes = off;
+        const size_t base = pad_to(out->bytes.size(), 128);
+        out->bytes.resize(base + meta_bytes + pad_to(values.size(), 128), 0);
+        uint8_t* p = out->bytes.data() + base;
+        std::memcpy(p, &h, sizeof h);
+        {
+            uint16_t* wb = reinterpret_cast<uint16_t*>(p + h.warp_off);
+            PanelItem* di = reinterpret_cast<PanelItem*>(p + h.items_off);
+            uint32_t pos = 0;
+            for (int w = 0; w < warps; ++w) {
+                wb[w] = (uint16_t)pos;
+                for (uint32_t j : per_warp[w]) di[pos++] = desc[j];
+            }
+            wb[warps] = (uint16_t)pos;
+        }
+        if (!gath.empty()) std::memcpy(p + h.gather_off, gath.data(), gath.size() * sizeof(PanelGather));
+        if (n_stages) std::memcpy(p + h.expect_off, expect.data(), n_stages * 2);
+        if (!cidx.empty()) std::memcpy(p + h.cidx_off, cidx.data(), cidx.size());
+        if (!ridx.empty()) std::memcpy(p + h.ridx_off, ridx.data(), ridx.size());
+        if (!values.empty()) std::memcpy(p + meta_bytes, values.data(), values.size());
+        PanelCta& ct = out->cta[c];
+        ct.off16 = (uint32_t)(base / 16); ct.meta_bytes = (uint32_t)meta_bytes; ct.value_bytes = (uint32_t)values.size();
+        ct.n_rows = (uint32_t)(R1 - R0);
+        out->max_meta = std::max(out->max_meta, meta_bytes);
+        out->max_xg = std::max(out->max_xg, cidx.size());
+        out->max_rows = std::max<size_t>(out->max_rows, (size_t)(R1 - R0));
+    }
+    if (out->bytes.size() / 16 > 0xffffffffull) return 1;
+    out->balance = max_cta_cost > 0.0 ? (sum_cta_cost / n_ctas) / max_cta_cost : 1.0;
+    out->warp_balance = max_warp_cost > 0.0 ? (sum_cta_cost / ((double)n_ctas * warps)) / max_warp_cost : 1.0;
+    return CSB_OK;
+}
+
+}  // namespace csb

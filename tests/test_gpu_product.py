@@ -12,6 +12,18 @@ pytestmark = pytest.mark.gpu
 RTOL = {"f16": 2e-3, "f32": 1e-5}   # max relative error per output allowed for each storage type
 
 
+@pytest.fixture(autouse=True, params=["panel", "stream"])
+def spmv_path(request, monkeypatch):
+    """Batch-1 products of fp16 matrices have two kernels: the panel kernel (default) and the
+    per-warp stream kernel that also serves fp32 values and small batches.  Every case runs on both;
+    the choice is made when the matrix is encoded."""
+    if request.param == "stream":
+        monkeypatch.setenv("CSB_NO_PANEL", "1")
+    else:
+        monkeypatch.delenv("CSB_NO_PANEL", raising=False)
+    return request.param
+
+
 def check_product(got, want, scale, vd):
     """|got - want| <= rtol * max(|want|, 1e-2 * sum|w||x|): relative error per output, with
     the forward-error scale of the row as the floor where the exact output is near zero."""
@@ -36,7 +48,7 @@ def run_case(mat, X, opts=None, repeat=2):
             binding.csb_spmm(A, Xd, Y)
         torch.cuda.synchronize()
         outs.append(Y.cpu().numpy())
-    assert np.array_equal(outs[0], outs[1]), "two runs differ bitwise: summation order is not fixed"
+    assert all(np.array_equal(outs[0], o) for o in outs[1:]), "two runs differ bitwise: summation order is not fixed"
     args = (mat.dense, mat.block_r, mat.block_c, mat.row_keep, mat.col_keep, mat.val_dtype)
     check_product(outs[0], O.spmm(*args, X), O.abs_scale(*args, X), mat.val_dtype)
     info = A.info()
@@ -101,6 +113,18 @@ def test_schedules_agree(opts):
     full = dict(ctas=0, warps_per_cta=0, stage_bytes=0, stages=0)
     full.update(opts)
     run_case(w.matrix, w.X, full)
+
+
+@pytest.mark.parametrize("ctas,stage,ring", [(4, 8192, 14), (16, 8192, 15), (148, 16384, 15)])
+def test_panel_ring_is_refilled_many_times(monkeypatch, spmv_path, ctas, stage, ring):
+    # few CTAs and a ring of two or four small stages: every slot is refilled dozens of times and
+    # warps run far ahead of each other, which is what the refill protocol has to survive
+    if spmv_path != "panel":
+        pytest.skip("the ring belongs to the panel kernel")
+    monkeypatch.setenv("CSB_PANEL_STAGE", str(stage))
+    monkeypatch.setenv("CSB_PANEL_RING_LOG2", str(ring))
+    w = workloads.make_spmv_workload(21, 2048, 4096, 64, 64, "lognormal", rate=5.0, batch=1, w_std=0.05)
+    run_case(w.matrix, w.X, dict(ctas=ctas, warps_per_cta=0, stage_bytes=0, stages=0), repeat=3)
 
 
 def test_cfg4_full_size_sampled():
