@@ -247,7 +247,7 @@ struct PanelHeader {        // start of a panel's meta part; offsets are from th
     uint32_t n_items, n_gather, n_xg, n_stages;
     uint32_t value_bytes, ridx_bytes, row0, n_rows;
     uint32_t warp_off, items_off, gather_off, expect_off;
-    uint32_t cidx_off, ridx_off, pad[2];
+    uint32_t cidx_off, ridx_off, list_off, n_bundles;
 };
 static_assert(sizeof(PanelHeader) == 64, "header is four 16-byte words");
 struct PanelCta { uint32_t off16, meta_bytes, value_bytes, n_rows; };

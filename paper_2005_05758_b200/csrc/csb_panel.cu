@@ -13,10 +13,12 @@
 //   * the panel's values flow through one shared-memory ring in fixed-size stages.  Whoever
 //     finishes the last item of a stage refills its slot, so there is no producer thread and
 //     nobody waits for a slower neighbour;
-//   * a warp takes one item at a time (up to 32 kept rows of a block).  A lane owns one kept
-//     row and reads 16 bytes = 8 kept columns per step; when the item has 16 or fewer rows the
-//     lanes split the columns 2-, 4-, ... ways and a few shuffles join them.  Products are
-//     accumulated with packed fp32 multiply-adds;
+//   * a warp takes one bundle at a time: one item (up to 32 kept rows of a block) on all its
+//     lanes, or two items of at most 16 rows / four of at most 8 rows side by side on lane
+//     groups of 16 / 8, so that the fixed work per item is shared.  A lane owns one kept row
+//     and reads 16 bytes = 8 kept columns per step; lanes left over in a group split the
+//     columns 2-, 4-, ... ways and a few shuffles join them.  Products are accumulated with
+//     packed fp32 multiply-adds;
 //   * every warp adds into its own copy of the CTA's output rows; at the end the CTA adds the
 //     copies in warp order and stores y.  The deal of items to warps is part of the plan, so
 //     the result does not depend on timing.
@@ -191,8 +193,9 @@ __global__ void __launch_bounds__(1024, 1) csb_panel_kernel(const __grid_constan
         __syncthreads();
         PANEL_STAMP(3);
 
-        // ---- this warp's items
+        // ---- this warp's bundles: one item on all 32 lanes, or two / four small ones side by side
         const uint16_t* wb = reinterpret_cast<const uint16_t*>(meta + H->warp_off);
+        const uint16_t* wlist = reinterpret_cast<const uint16_t*>(meta + H->list_off);
         const uint4* items = reinterpret_cast<const uint4*>(meta + H->items_off);
         const uint16_t* expect = reinterpret_cast<const uint16_t*>(meta + H->expect_off);
         const uint8_t* ridx = meta + H->ridx_off;
@@ -200,21 +203,21 @@ __global__ void __launch_bounds__(1024, 1) csb_panel_kernel(const __grid_constan
         float* zs = zs_all + (size_t)warp * a.max_rows;
         const uint32_t i_end = wb[warp + 1];
         uint32_t idx = wb[warp];
-        uint4 d = idx < i_end ? items[idx] : make_uint4(0u, 0u, 0u, 0u);
+        uint32_t e = idx < i_end ? wlist[idx] : 0u;
         for (; idx < i_end; ++idx) {
+            const int logg = (int)(e >> 14);
+            const int gl = lane & ((32 >> logg) - 1), grp = lane >> (5 - logg);
+            const uint4 d = items[(e & 0x3fffu) + grp];
+            if (idx + 1 < i_end) e = wlist[idx + 1];          // on its way while this bundle is worked on
             const uint32_t off = d.x << 4;
             const uint32_t xoff4 = d.y & 0xffffu, roff = d.z & 0xffffu;
             const int zoff = (int)(int16_t)(d.y >> 16);
             const int m = (int)((d.z >> 16) & 0xffu), logp = (int)(d.z >> 24), n = (int)(d.w & 0xffffu);
-            // the next descriptor and this lane's row index are on their way while the item is worked on
-            if (idx + 1 < i_end) d = items[idx + 1];
-            const int my_row = zoff + (int)ridx[roff + (lane < m ? lane : 0)];
-            const uint32_t s0 = off >> a.log2_stage, s1 = (off + (uint32_t)(m * n * 2) - 1u) >> a.log2_stage;
-            bool ok = panel_wait_stage(full, issued, s0, a.log2_slots, s_dead);
-            if (ok && s1 != s0) ok = panel_wait_stage(full, issued, s1, a.log2_slots, s_dead);
-            if (__any_sync(0xffffffffu, !ok)) { *s_dead = 1u; break; }
+            const int my_row = zoff + (int)ridx[roff + (gl < m ? gl : 0)];
+            const uint32_t st = off >> a.log2_stage;          // the same for every member of the bundle
+            if (__any_sync(0xffffffffu, !panel_wait_stage(full, issued, st, a.log2_slots, s_dead))) { *s_dead = 1u; break; }
 
-            const int r = lane & ((1 << logp) - 1), sub = lane >> logp, S = 32 >> logp;
+            const int r = gl & ((1 << logp) - 1), sub = gl >> logp, S = 32 >> (logg + logp);
             const int noct = n >> 3;
             float2 a0 = make_float2(0.f, 0.f), a1 = make_float2(0.f, 0.f);
             float2 b0 = make_float2(0.f, 0.f), b1 = make_float2(0.f, 0.f);
@@ -248,51 +251,60 @@ __global__ void __launch_bounds__(1024, 1) csb_panel_kernel(const __grid_constan
                 }
             }
             float acc = 0.f;
-            if (n & 7) {
+            if ((n & 7) && gl < m) {
                 // the last n % 8 columns: [row][4], [row][2], [row][1] behind the octets
                 uint32_t tb = off + ((uint32_t)(noct * m) << 4);
                 const float* xt = xg + 4 * xoff4 + 8 * noct;
-                if (lane < m) {
-                    if (n & 4) {
-                        const uint2 w = *reinterpret_cast<const uint2*>(ring + ((tb + 8u * lane) & ring_mask));
-                        const float4 x0 = *reinterpret_cast<const float4*>(xt);
-                        b0 = ffma2(h2f2(w.x), make_float2(x0.x, x0.y), b0);
-                        b1 = ffma2(h2f2(w.y), make_float2(x0.z, x0.w), b1);
-                        tb += 8u * m; xt += 4;
-                    }
-                    if (n & 2) {
-                        const uint32_t w = *reinterpret_cast<const uint32_t*>(ring + ((tb + 4u * lane) & ring_mask));
-                        const float2 x0 = *reinterpret_cast<const float2*>(xt);
-                        a0 = ffma2(h2f2(w), x0, a0);
-                        tb += 4u * m; xt += 2;
-                    }
-                    if (n & 1) {
-                        const __half w = *reinterpret_cast<const __half*>(ring + ((tb + 2u * lane) & ring_mask));
-                        acc = __half2float(w) * xt[0];
-                    }
+                if (n & 4) {
+                    const uint2 w = *reinterpret_cast<const uint2*>(ring + ((tb + 8u * gl) & ring_mask));
+                    const float4 x0 = *reinterpret_cast<const float4*>(xt);
+                    b0 = ffma2(h2f2(w.x), make_float2(x0.x, x0.y), b0);
+                    b1 = ffma2(h2f2(w.y), make_float2(x0.z, x0.w), b1);
+                    tb += 8u * m; xt += 4;
+                }
+                if (n & 2) {
+                    const uint32_t w = *reinterpret_cast<const uint32_t*>(ring + ((tb + 4u * gl) & ring_mask));
+                    const float2 x0 = *reinterpret_cast<const float2*>(xt);
+                    a0 = ffma2(h2f2(w), x0, a0);
+                    tb += 4u * m; xt += 2;
+                }
+                if (n & 1) {
+                    const __half w = *reinterpret_cast<const __half*>(ring + ((tb + 2u * gl) & ring_mask));
+                    acc = __half2float(w) * xt[0];
                 }
             }
             acc += ((a0.x + a1.x) + (b0.x + b1.x)) + ((a0.y + a1.y) + (b0.y + b1.y));
-            // join the lanes that split the columns of a row (fixed tree)
-            for (int o = 16; o >= (1 << logp); o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-            if (lane < m) zs[my_row] += acc;
+            // join the lanes that split the columns of a row (fixed tree inside the lane group)
+            if (logg == 0) {
+                for (int o = 16; o >= (1 << logp); o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+                if (lane < m) zs[my_row] += acc;
+            } else {
+                const int pmin = (int)__reduce_min_sync(0xffffffffu, 1u << logp);
+                for (int o = 16 >> logg; o >= pmin; o >>= 1) {
+                    const float t = __shfl_xor_sync(0xffffffffu, acc, o);
+                    if (o >= (1 << logp)) acc += t;
+                }
+                // members of a bundle may add into the same output: one lane group at a time
+                for (int g = 0; g < (1 << logg); ++g) {
+                    if (grp == g && gl < m) zs[my_row] += acc;
+                    __syncwarp();
+                }
+            }
             __syncwarp();
-            // ---- this item is done with its stage(s); the last one out refills the slot
+            // ---- the bundle is done with its stage; the last one out refills the slot
             if (lane == 0) {
                 __threadfence_block();
-                for (uint32_t st = s0; st <= s1; ++st) {
-                    const uint32_t slot = st & (slots - 1u);
-                    if (atomicAdd(&done[slot], 1u) + 1u == (uint32_t)expect[st]) {
-                        *reinterpret_cast<volatile uint32_t*>(&done[slot]) = 0u;
-                        const uint32_t nx = st + slots;
-                        if (nx < n_stages) {
-                            __threadfence_block();
-                            fence_proxy_async_all();
-                            const uint32_t bytes = min(SB, value_bytes - (nx << a.log2_stage));
-                            issued[slot] = issued[slot] + 1u;
-                            mbar_expect_tx(&full[slot], bytes);
-                            bulk_g2s(ring + ((size_t)slot << a.log2_stage), values + ((size_t)nx << a.log2_stage), bytes, &full[slot]);
-                        }
+                const uint32_t slot = st & (slots - 1u);
+                if (atomicAdd(&done[slot], 1u) + 1u == (uint32_t)expect[st]) {
+                    *reinterpret_cast<volatile uint32_t*>(&done[slot]) = 0u;
+                    const uint32_t nx = st + slots;
+                    if (nx < n_stages) {
+                        __threadfence_block();
+                        fence_proxy_async_all();
+                        const uint32_t bytes = min(SB, value_bytes - (nx << a.log2_stage));
+                        issued[slot] = issued[slot] + 1u;
+                        mbar_expect_tx(&full[slot], bytes);
+                        bulk_g2s(ring + ((size_t)slot << a.log2_stage), values + ((size_t)nx << a.log2_stage), bytes, &full[slot]);
                     }
                 }
             }

@@ -33,12 +33,25 @@ namespace csb {
 static inline size_t pad_to(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static inline int log2_ceil(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
 
-// Modelled time of one item on one SM, in issue slots of one warp: a fixed part per item, the
-// octet steps of the multiply loop, the remainder columns and the joining shuffles.
+// How many items of this height share a warp: one with more than 16 rows, two with 9..16, four
+// with 8 or fewer (log2 of that number).
+static inline int panel_item_logg(int mi) { return mi > 16 ? 0 : mi > 8 ? 1 : 2; }
+// Loop steps of an item: its column octets divided among the lane sub-groups of its lane group.
+static inline int panel_item_steps(int mi, int n) {
+    const int gw = 32 >> panel_item_logg(mi), S = gw >> log2_ceil(mi);
+    return ((n >> 3) + S - 1) / S;
+}
+// Modelled issue slots, from instruction counts of the kernel on matrices with a fixed number
+// of kept lines per block: a fixed part per bundle, and per member its loop steps, remainder
+// columns and joining shuffles.
+constexpr double kPanelBundleFixed = 110.0;
+static double panel_member_cost(int mi, int n) {
+    const int gw = 32 >> panel_item_logg(mi), S = gw >> log2_ceil(mi);
+    return 28.0 * panel_item_steps(mi, n) + ((n & 7) ? 34.0 : 0.0) + 8.0 * log2_ceil(S);
+}
+// Cost of an item as seen by the row cut: its share of a bundle.
 static double panel_item_cost(int mi, int n) {
-    const int S = 32 >> log2_ceil(mi);
-    const int steps = ((n >> 3) + S - 1) / S;
-    return 110.0 + 19.0 * steps + ((n & 7) ? 25.0 : 0.0) + 3.0 * log2_ceil(S);
+    return (kPanelBundleFixed + panel_member_cost(mi, n)) / (double)(1 << panel_item_logg(mi)) + 10.0;
 }
 
 struct PanelItemSrc {
@@ -162,68 +175,121 @@ int plan_panels_host(const csb_matrix* A, int ctas, int warps, int stage_bytes, 
                 }
             }
         }
-        // The value stream holds the items longest first: dealt in that order to the least loaded
-        // warp they leave the warps with nearly equal work, and the short ones fill in at the end.
-        std::stable_sort(items.begin(), items.end(), [](const PanelItemSrc& x, const PanelItemSrc& y) { return x.cost > y.cost; });
-        for (const PanelItemSrc& it : items) {
-            const int64_t b = it.block, bi = b / A->nbc;
-            const int n = A->n[b];
-            const uint8_t* ri = A->row_idx.data() + A->ridx_off[b];
-            PanelItem d{};
-            d.off16 = (uint32_t)(values.size() / 16);
-            d.xoff4 = (uint16_t)(it.xoff / 4);
-            d.zoff = (int16_t)(bi * BR - R0);
-            d.roff = (uint16_t)ridx.size();
-            d.m = (uint8_t)it.mi; d.logp = (uint8_t)log2_ceil(it.mi);
-            d.n = (uint16_t)n; d.pad = 0;
-            ridx.insert(ridx.end(), ri + it.r0, ri + it.r0 + it.mi);
-            // values: [octet][row][8], then [row][4], [row][2], [row][1]
-            const uint8_t* v = A->val.data() + (A->val_off[b] + (uint64_t)it.r0 * n) * 2;
-            const size_t base = values.size();
-            values.resize(base + it.bytes, 0);
-            uint8_t* p = values.data() + base;
-            const int noct = n >> 3;
-            for (int o = 0; o < noct; ++o)
-                for (int r = 0; r < it.mi; ++r, p += 16) std::memcpy(p, v + ((size_t)r * n + 8 * o) * 2, 16);
-            int k = noct * 8;
-            for (int w = 4; w >= 1; w >>= 1)
-                if (n & w) {
-                    for (int r = 0; r < it.mi; ++r, p += 2 * w) std::memcpy(p, v + ((size_t)r * n + k) * 2, 2 * w);
-                    k += w;
+        if (items.size() > 0x3fff) return 1;
+        // ---- bundles: items of 16 or fewer rows go through a warp two at a time, of 8 or fewer
+        // four at a time (each on its own group of lanes), so the fixed work per item is shared.
+        // Members of a bundle are picked with about the same number of loop steps.
+        struct Bundle { std::vector<uint32_t> members; int logg; double cost; size_t bytes; };
+        std::vector<Bundle> bundles;
+        for (int logg = 0; logg <= 2; ++logg) {
+            std::vector<uint32_t> cls;
+            for (uint32_t i = 0; i < items.size(); ++i) if (panel_item_logg(items[i].mi) == logg) cls.push_back(i);
+            std::stable_sort(cls.begin(), cls.end(), [&](uint32_t x, uint32_t y) {
+                return panel_item_steps(items[x].mi, A->n[items[x].block]) > panel_item_steps(items[y].mi, A->n[items[y].block]); });
+            for (size_t k = 0; k < cls.size(); k += (size_t)1 << logg) {
+                Bundle bu{};
+                bu.logg = logg;
+                double worst = 0.0;
+                for (size_t j = k; j < std::min(cls.size(), k + ((size_t)1 << logg)); ++j) {
+                    bu.members.push_back(cls[j]);
+                    bu.bytes += items[cls[j]].bytes;
+                    worst = std::max(worst, panel_member_cost(items[cls[j]].mi, A->n[items[cls[j]].block]));
                 }
-            desc.push_back(d);
+                bu.cost = kPanelBundleFixed + worst + 10.0 * (double)bu.members.size();
+                bundles.push_back(std::move(bu));
+            }
         }
-        if (cidx.size() > (size_t)max_xg_floats || cidx.size() / 4 > 0xffff || ridx.size() > 0xffff || items.size() > 0xffff ||
-            values.size() / 16 > 0xffffffffull)
-            return 1;                                            // beyond the kernel's limits: the caller keeps the other path
-        // items per stage (an item that straddles a boundary counts on both sides)
-        const size_t n_stages = (values.size() + stage_bytes - 1) / stage_bytes;
+        // longest first, then packed into stages (first fit), so that no bundle straddles a stage
+        std::stable_sort(bundles.begin(), bundles.end(), [](const Bundle& x, const Bundle& y) { return x.cost > y.cost; });
+        std::vector<std::vector<uint32_t>> stage_of;          // bundles of every stage, in placement order
+        std::vector<size_t> fill;
+        for (uint32_t k = 0; k < bundles.size(); ++k) {
+            if (bundles[k].bytes > (size_t)stage_bytes) return 1;
+            size_t st = 0;
+            while (st < fill.size() && fill[st] + bundles[k].bytes > (size_t)stage_bytes) ++st;
+            if (st == fill.size()) { fill.push_back(0); stage_of.emplace_back(); }
+            fill[st] += bundles[k].bytes;
+            stage_of[st].push_back(k);
+        }
+        const size_t n_stages = fill.size();
         std::vector<uint16_t> expect(n_stages, 0);
-        for (size_t i = 0; i < items.size(); ++i) {
-            const size_t off = (size_t)desc[i].off16 * 16;
-            const size_t s0 = off / stage_bytes, s1 = (off + items[i].bytes - 1) / stage_bytes;
-            for (size_t s = s0; s <= s1; ++s) ++expect[s];
-        }
-        // deal items to warps in stream order, each to the least loaded warp
+        // emit the values stage by stage and deal the bundles, in stream order, to the least loaded warp
         std::vector<double> load(warps, 0.0);
         std::vector<std::vector<uint32_t>> per_warp(warps);
-        for (size_t i = 0; i < items.size(); ++i) {
-            const int w = (int)(std::min_element(load.begin(), load.end()) - load.begin());
-            per_warp[w].push_back((uint32_t)i);
-            load[w] += items[i].cost;
+        desc.assign(items.size(), PanelItem{});
+        for (size_t st = 0; st < n_stages; ++st) {
+            values.resize(st * (size_t)stage_bytes, 0);         // the previous stage is padded to its end
+            expect[st] = (uint16_t)stage_of[st].size();
+            for (uint32_t k : stage_of[st]) {
+                const int w = (int)(std::min_element(load.begin(), load.end()) - load.begin());
+                per_warp[w].push_back(k);
+                load[w] += bundles[k].cost;
+                for (uint32_t i : bundles[k].members) {
+                    const PanelItemSrc& it = items[i];
+                    const int64_t b = it.block, bi = b / A->nbc;
+                    const int n = A->n[b];
+                    const uint8_t* ri = A->row_idx.data() + A->ridx_off[b];
+                    PanelItem& d = desc[i];
+                    d.off16 = (uint32_t)(values.size() / 16);
+                    d.xoff4 = (uint16_t)(it.xoff / 4);
+                    d.zoff = (int16_t)(bi * BR - R0);
+                    d.roff = (uint16_t)ridx.size();
+                    d.m = (uint8_t)it.mi; d.logp = (uint8_t)log2_ceil(it.mi);
+                    d.n = (uint16_t)n; d.pad = 0;
+                    ridx.insert(ridx.end(), ri + it.r0, ri + it.r0 + it.mi);
+                    // values: [octet][row][8], then [row][4], [row][2], [row][1]
+                    const uint8_t* v = A->val.data() + (A->val_off[b] + (uint64_t)it.r0 * n) * 2;
+                    const size_t base = values.size();
+                    values.resize(base + it.bytes, 0);
+                    uint8_t* p = values.data() + base;
+                    const int noct = n >> 3;
+                    for (int o = 0; o < noct; ++o)
+                        for (int r = 0; r < it.mi; ++r, p += 16) std::memcpy(p, v + ((size_t)r * n + 8 * o) * 2, 16);
+                    int kk = noct * 8;
+                    for (int w2 = 4; w2 >= 1; w2 >>= 1)
+                        if (n & w2) {
+                            for (int r = 0; r < it.mi; ++r, p += 2 * w2) std::memcpy(p, v + ((size_t)r * n + kk) * 2, 2 * w2);
+                            kk += w2;
+                        }
+                }
+            }
         }
+        if (cidx.size() > (size_t)max_xg_floats || cidx.size() / 4 > 0xffff || ridx.size() > 0xffff || values.size() / 16 > 0xffffffffull)
+            return 1;                                            // beyond the kernel's limits: the caller keeps the other path
         double cta_cost = 0.0;
         for (int w = 0; w < warps; ++w) { cta_cost += load[w]; max_warp_cost = std::max(max_warp_cost, load[w]); }
         sum_cta_cost += cta_cost;
         max_cta_cost = std::max(max_cta_cost, cta_cost);
+        // descriptors in the order the warps take them: a bundle's members side by side, missing
+        // members as empty descriptors (no rows, no columns) that point at the bundle's stage
+        std::vector<PanelItem> table;
+        std::vector<uint16_t> wlist, wbegin(warps + 1, 0);
+        for (int w = 0; w < warps; ++w) {
+            wbegin[w] = (uint16_t)wlist.size();
+            for (uint32_t k : per_warp[w]) {
+                const Bundle& bu = bundles[k];
+                if (table.size() > 0x3fff - 4) return 1;
+                wlist.push_back((uint16_t)(table.size() | ((size_t)bu.logg << 14)));
+                for (int g = 0; g < (1 << bu.logg); ++g) {
+                    if (g < (int)bu.members.size()) { table.push_back(desc[bu.members[g]]); continue; }
+                    PanelItem e{};
+                    e.off16 = desc[bu.members[0]].off16;
+                    e.logp = (uint8_t)(5 - bu.logg);
+                    table.push_back(e);
+                }
+            }
+        }
+        wbegin[warps] = (uint16_t)wlist.size();
+        if (wlist.size() > 0xffff) return 1;
 
         // ---- emit the panel
         PanelHeader h{};
-        h.n_items = (uint32_t)items.size(); h.n_gather = (uint32_t)gath.size(); h.n_xg = (uint32_t)cidx.size();
+        h.n_items = (uint32_t)table.size(); h.n_bundles = (uint32_t)wlist.size(); h.n_gather = (uint32_t)gath.size(); h.n_xg = (uint32_t)cidx.size();
         h.n_stages = (uint32_t)n_stages; h.value_bytes = (uint32_t)values.size(); h.ridx_bytes = (uint32_t)ridx.size();
         h.row0 = (uint32_t)R0; h.n_rows = (uint32_t)(R1 - R0);
         size_t off = sizeof(PanelHeader);
         h.warp_off = (uint32_t)off; off = pad_to(off + (size_t)(warps + 1) * 2, 16);
+        h.list_off = (uint32_t)off; off = pad_to(off + wlist.size() * 2, 16);
         h.items_off = (uint32_t)off; off += (size_t)h.n_items * sizeof(PanelItem);
         h.gather_off = (uint32_t)off; off = pad_to(off + gath.size() * sizeof(PanelGather), 16);
         h.expect_off = (uint32_t)off; off = pad_to(off + n_stages * 2, 16);
@@ -234,16 +300,9 @@ int plan_panels_host(const csb_matrix* A, int ctas, int warps, int stage_bytes, 
         out->bytes.resize(base + meta_bytes + pad_to(values.size(), 128), 0);
         uint8_t* p = out->bytes.data() + base;
         std::memcpy(p, &h, sizeof h);
-        {
-            uint16_t* wb = reinterpret_cast<uint16_t*>(p + h.warp_off);
-            PanelItem* di = reinterpret_cast<PanelItem*>(p + h.items_off);
-            uint32_t pos = 0;
-            for (int w = 0; w < warps; ++w) {
-                wb[w] = (uint16_t)pos;
-                for (uint32_t j : per_warp[w]) di[pos++] = desc[j];
-            }
-            wb[warps] = (uint16_t)pos;
-        }
+        std::memcpy(p + h.warp_off, wbegin.data(), wbegin.size() * 2);
+        if (!wlist.empty()) std::memcpy(p + h.list_off, wlist.data(), wlist.size() * 2);
+        if (!table.empty()) std::memcpy(p + h.items_off, table.data(), table.size() * sizeof(PanelItem));
         if (!gath.empty()) std::memcpy(p + h.gather_off, gath.data(), gath.size() * sizeof(PanelGather));
         if (n_stages) std::memcpy(p + h.expect_off, expect.data(), n_stages * 2);
         if (!cidx.empty()) std::memcpy(p + h.cidx_off, cidx.data(), cidx.size());

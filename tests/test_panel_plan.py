@@ -11,7 +11,7 @@ from oracle import csb_oracle as O
 from paper_2005_05758_b200 import binding
 
 HDR = ("n_items", "n_gather", "n_xg", "n_stages", "value_bytes", "ridx_bytes", "row0", "n_rows",
-       "warp_off", "items_off", "gather_off", "expect_off", "cidx_off", "ridx_off")
+       "warp_off", "items_off", "gather_off", "expect_off", "cidx_off", "ridx_off", "list_off", "n_bundles")
 
 
 def decode(plan, rows, cols, block_r, warps, stage):
@@ -25,16 +25,17 @@ def decode(plan, rows, cols, block_r, warps, stage):
         assert meta_bytes <= plan["max_meta"]
         meta = blob[base:base + meta_bytes]
         vals = blob[base + meta_bytes:base + meta_bytes + value_bytes]
-        h = dict(zip(HDR, (int(v) for v in meta[:56].view(np.uint32))))
+        h = dict(zip(HDR, (int(v) for v in meta[:64].view(np.uint32))))
         assert h["value_bytes"] == value_bytes and h["n_rows"] == n_rows <= plan["max_rows"]
         assert h["n_stages"] == -(-value_bytes // stage)
         assert h["n_xg"] % 4 == 0 and h["n_xg"] <= plan["max_xg"]
-        for k in ("items_off", "gather_off", "expect_off", "cidx_off", "ridx_off"):
+        for k in ("items_off", "gather_off", "expect_off", "cidx_off", "ridx_off", "list_off"):
             assert h[k] % 16 == 0, k
         row0 = h["row0"]
         ranges.append((row0, row0 + n_rows))
         wb = meta[h["warp_off"]:h["warp_off"] + 2 * (warps + 1)].view(np.uint16).astype(int)
-        assert wb[0] == 0 and wb[-1] == h["n_items"] and (np.diff(wb) >= 0).all()
+        assert wb[0] == 0 and wb[-1] == h["n_bundles"] and (np.diff(wb) >= 0).all()
+        wlist = meta[h["list_off"]:h["list_off"] + 2 * h["n_bundles"]].view(np.uint16).astype(int)
         items = meta[h["items_off"]:h["items_off"] + 16 * h["n_items"]]
         gath = meta[h["gather_off"]:h["gather_off"] + 8 * h["n_gather"]]
         expect = meta[h["expect_off"]:h["expect_off"] + 2 * h["n_stages"]].view(np.uint16).astype(int)
@@ -52,57 +53,74 @@ def decode(plan, rows, cols, block_r, warps, stage):
         assert pos == h["n_xg"] and xg_col.max(initial=0) < cols
         touched = np.zeros(h["n_stages"], int)
         spans = []
+        seen_desc = 0
         for w in range(warps):
-            last_off = -1
-            for i in range(wb[w], wb[w + 1]):
-                d = items[16 * i:16 * i + 16]
-                off = int(d[0:4].view(np.uint32)[0]) * 16
-                xoff4, roff = int(d[4:6].view(np.uint16)[0]), int(d[8:10].view(np.uint16)[0])
-                zoff = int(d[6:8].view(np.int16)[0])
-                m, logp = int(d[10]), int(d[11])
-                n = int(d[12:14].view(np.uint16)[0])
-                assert 1 <= m <= 32 and 1 <= n and (1 << logp) >= m and ((1 << logp) < 2 * m)
-                assert off > last_off, "a warp takes its items in stream order"
-                last_off = off
-                nbytes = m * n * 2
-                assert off + nbytes <= value_bytes and nbytes <= stage
-                s0, s1 = off // stage, (off + nbytes - 1) // stage
-                assert s1 - s0 <= 1
-                touched[s0:s1 + 1] += 1
-                spans.append((off, off + ((nbytes + 15) & ~15)))
-                assert (row0 + zoff) % block_r == 0, "zoff is the block-row's first row relative to the panel's"
-                rr = zoff + ridx[roff:roff + m]
-                assert (np.diff(rr) > 0).all() and rr.min() >= 0 and rr.max() < n_rows
-                cc = xg_col[4 * xoff4:4 * xoff4 + n]
-                assert (cc >= 0).all() and (np.diff(cc) > 0).all(), "kept columns of a block are ascending"
-                v = vals[off:off + nbytes].view(np.float16).astype(np.float64)
-                noct = n >> 3
-                # what the lanes read: lane (sub, r) takes octets sub, sub + S, ... of row r
-                P = 1 << logp
-                S = 32 // P
-                got = np.zeros((m, n))
-                for lane in range(32):
-                    r, sub = lane & (P - 1), lane >> logp
-                    if r >= m:
+            last_stage = -1
+            for e in wlist[wb[w]:wb[w + 1]]:
+                logg, first = e >> 14, e & 0x3FFF
+                G, GW = 1 << logg, 32 >> logg
+                assert first == seen_desc, "descriptors sit in the order the warps take them"
+                seen_desc += G
+                stages = set()
+                real = 0
+                for grp in range(G):
+                    d = items[16 * (first + grp):16 * (first + grp) + 16]
+                    off = int(d[0:4].view(np.uint32)[0]) * 16
+                    xoff4, roff = int(d[4:6].view(np.uint16)[0]), int(d[8:10].view(np.uint16)[0])
+                    zoff = int(d[6:8].view(np.int16)[0])
+                    m, logp = int(d[10]), int(d[11])
+                    n = int(d[12:14].view(np.uint16)[0])
+                    stages.add(off // stage)
+                    P = 1 << logp
+                    assert P <= GW
+                    if m == 0:                          # a missing member: no rows, no columns, same stage
+                        assert n == 0 and grp > 0 and P == GW
                         continue
-                    for o in range(sub, noct, S):
-                        q = (o * m + r) * 8
-                        got[r, 8 * o:8 * o + 8] = v[q:q + 8]
-                tb, k = noct * m * 8, noct * 8
-                for wdt in (4, 2, 1):
-                    if n & wdt:
-                        for r in range(m):
-                            got[r, k:k + wdt] = v[tb + r * wdt:tb + r * wdt + wdt]
-                        tb += m * wdt
-                        k += wdt
-                for r in range(m):
-                    dense[row0 + rr[r], cc] = got[r]
-                    count[row0 + rr[r], cc] += 1
-        assert np.array_equal(touched, expect), "per-stage item counts are what the refill protocol waits for"
+                    real += 1
+                    assert 1 <= m <= GW and 1 <= n and P >= m and P < 2 * m
+                    assert (m > 16) == (logg == 0) and (m <= 8) == (logg == 2), "items are bundled by height"
+                    nbytes = m * n * 2
+                    assert off + nbytes <= value_bytes
+                    assert off // stage == (off + nbytes - 1) // stage, "no item straddles a stage"
+                    spans.append((off, off + ((nbytes + 15) & ~15)))
+                    assert (row0 + zoff) % block_r == 0, "zoff is the block-row's first row relative to the panel's"
+                    rr = zoff + ridx[roff:roff + m]
+                    assert (np.diff(rr) > 0).all() and rr.min() >= 0 and rr.max() < n_rows
+                    cc = xg_col[4 * xoff4:4 * xoff4 + n]
+                    assert (cc >= 0).all() and (np.diff(cc) > 0).all(), "kept columns of a block are ascending"
+                    v = vals[off:off + nbytes].view(np.float16).astype(np.float64)
+                    noct = n >> 3
+                    # what the lanes of the group read: lane (sub, r) takes octets sub, sub + S, ... of row r
+                    S = GW // P
+                    got = np.zeros((m, n))
+                    for gl in range(GW):
+                        r, sub = gl & (P - 1), gl >> logp
+                        if r >= m:
+                            continue
+                        for o in range(sub, noct, S):
+                            q = (o * m + r) * 8
+                            got[r, 8 * o:8 * o + 8] = v[q:q + 8]
+                    tb, k = noct * m * 8, noct * 8
+                    for wdt in (4, 2, 1):
+                        if n & wdt:
+                            for r in range(m):
+                                got[r, k:k + wdt] = v[tb + r * wdt:tb + r * wdt + wdt]
+                            tb += m * wdt
+                            k += wdt
+                    for r in range(m):
+                        dense[row0 + rr[r], cc] = got[r]
+                        count[row0 + rr[r], cc] += 1
+                assert real >= 1 and len(stages) == 1, "a bundle sits in one stage"
+                st = stages.pop()
+                assert st >= last_stage, "a warp takes its bundles in stream order"
+                last_stage = st
+                touched[st] += 1
+        assert seen_desc == h["n_items"]
+        assert np.array_equal(touched, expect), "per-stage bundle counts are what the refill protocol waits for"
         spans.sort()
         pos = 0
-        for a, b in spans:                                # items tile the value stream without gaps or overlap
-            assert a == pos
+        for a, b in spans:                                # items tile the value stream; gaps only up to a stage's end
+            assert a == pos or (a > pos and a % stage == 0 and a - pos < stage)
             pos = b
         assert pos == value_bytes
     return dense, count, ranges
