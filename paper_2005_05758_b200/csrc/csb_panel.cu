@@ -81,6 +81,10 @@ __device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
 }
 __device__ __forceinline__ float2 h2f2(uint32_t w) { return __half22float2(*reinterpret_cast<const __half2*>(&w)); }
 
+// Blocks until the grids this one depends on (the work in front of it on the stream) have
+// completed and their writes are visible; returns at once for an ordinary launch.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Wait for a phase; gives up after the wall-clock bound or as soon as another warp of the CTA
 // has given up.
 __device__ __forceinline__ bool panel_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* dead) {
@@ -136,6 +140,11 @@ __global__ void __launch_bounds__(1024, 1) csb_panel_kernel(const __grid_constan
     volatile uint32_t* s_dead = reinterpret_cast<volatile uint32_t*>(smem + L.dead);
 
     const bool x_bulk = (reinterpret_cast<uintptr_t>(a.x) & 15) == 0 && (a.cols & 3) == 0;
+    // Launched with programmatic stream serialization, this grid may start while the kernel in
+    // front of it on the stream is still draining: whatever comes next may be scheduled as early
+    // as the hardware likes, and this grid touches x and y only behind grid_dependency_wait().
+    // The panels are written once at plan time, so their copies go out before that wait.
+    asm volatile("griddepcontrol.launch_dependents;");
     PANEL_STAMP(0);
     // the first copies go out from separate lanes of warp 0, each with the barrier it set up itself:
     // lane s < slots takes stage s, the next two lanes take the bookkeeping and x
@@ -145,17 +154,11 @@ __global__ void __launch_bounds__(1024, 1) csb_panel_kernel(const __grid_constan
         if (s < slots) { done[s] = 0u; issued[s] = 0u; }
         if (s == slots) *s_dead = 0u;
         mbar_fence_init();
-        // bookkeeping and x first: everything else waits for them, the values are needed later
+        // the bookkeeping first (everything else waits for it), then the values, then x, which
+        // may still be being written by the kernel in front
         if (s == slots) {
             mbar_expect_tx(metabar, meta_bytes);
             bulk_g2s(smem + L.meta, panel, meta_bytes, metabar);
-        } else if (s == slots + 1u) {
-            if (x_bulk) {
-                const uint32_t xb = (uint32_t)a.cols * 4u;
-                mbar_expect_tx(xbar, xb);
-                for (uint32_t off = 0; off < xb; off += 16384u)
-                    bulk_g2s(smem + L.xs + off, reinterpret_cast<const uint8_t*>(a.x) + off, min(16384u, xb - off), xbar);
-            }
         }
         __syncwarp(slots + 2u >= 32u ? 0xffffffffu : (1u << (slots + 2u)) - 1u);
         if (s < slots && s < n_stages) {
@@ -164,10 +167,19 @@ __global__ void __launch_bounds__(1024, 1) csb_panel_kernel(const __grid_constan
             mbar_expect_tx(&full[s], bytes);
             bulk_g2s(ring + ((size_t)s << a.log2_stage), values + ((size_t)s << a.log2_stage), bytes, &full[s]);
         }
+        if (s == slots + 1u && x_bulk) {
+            grid_dependency_wait();
+            const uint32_t xb = (uint32_t)a.cols * 4u;
+            mbar_expect_tx(xbar, xb);
+            for (uint32_t off = 0; off < xb; off += 16384u)
+                bulk_g2s(smem + L.xs + off, reinterpret_cast<const uint8_t*>(a.x) + off, min(16384u, xb - off), xbar);
+        }
     }
     for (int i = threadIdx.x; i < W * a.max_rows; i += blockDim.x) zs_all[i] = 0.f;
-    if (!x_bulk)
+    if (!x_bulk) {
+        grid_dependency_wait();
         for (int i = threadIdx.x; i < a.cols; i += blockDim.x) xs[i] = __ldg(a.x + i);
+    }
     __syncthreads();                                       // barriers initialised, counters and sums cleared
     PANEL_STAMP(1);
 
@@ -427,8 +439,19 @@ int launch_panels(const csb_matrix* A, const float* x, float* y, void* stream) {
     a.clocks = d_clocks;
     g_panel_clocks = d_clocks;
 #endif
-    csb_panel_kernel<<<P.ctas, P.warps * 32, P.smem_bytes, (cudaStream_t)stream>>>(a);
-    const cudaError_t e = cudaGetLastError();
+    // Programmatic stream serialization lets this grid's start-up (barriers, first copies of the
+    // panels) overlap the end of the kernel in front of it; the kernel orders itself behind that
+    // kernel before it touches x or y.  CSB_PANEL_PDL=0 asks for an ordinary launch.
+    static const int use_pdl = env_int("CSB_PANEL_PDL", 1);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)P.ctas); cfg.blockDim = dim3((unsigned)P.warps * 32u);
+    cfg.dynamicSmemBytes = P.smem_bytes; cfg.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = use_pdl ? 1u : 0u;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, csb_panel_kernel, a);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (prev != A->device) cudaSetDevice(prev);
     if (e != cudaSuccess) { set_error("panel kernel launch failed: %s", cudaGetErrorString(e)); return CSB_ERR_CUDA; }
     return CSB_OK;
