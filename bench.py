@@ -35,10 +35,10 @@ WORKLOAD = "cfg5: 2-layer LSTM, I=H=2048, 8192x4096 CSB weights, 64x64 blocks, ~
 
 
 # dram__bytes_read + dram__bytes_write per launch from the ncu captures summarised under profiles/
-# (csb_rnn_kernel_cfg5.md: T = 512 launch; csb_product_kernel_cfg4_rate4_b1.md).  They describe the
+# (csb_rnn_kernel_cfg5.md: T = 512 launch; csb_panel_kernel_cfg4_rate4_b1.md).  They describe the
 # kernels as committed with those summaries; set to None when a kernel or its layout changes.
 RNN_DRAM_BYTES_PER_LAUNCH = 20288768 + 11008
-SPMV4X_DRAM_BYTES_PER_LAUNCH = 35873280
+SPMV4X_DRAM_BYTES_PER_LAUNCH = 36163584
 
 
 def peaks():
@@ -261,7 +261,9 @@ def spmv_sweep(binding, torch, dev, rates, batch, reps=10, with_cpu=False):
         m = w.matrix
         A0 = binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, dev)
         info = A0.info()
-        ncopy = max(2, int(160e6 // max(info["device_stream_bytes"], 1)) + 1)
+        panel = batch == 1 and info["panel_ctas"] > 0      # which kernel serves this batch size
+        stream_bytes = info["panel_stream_bytes"] if panel else info["device_stream_bytes"]
+        ncopy = max(2, int(160e6 // max(stream_bytes, 1)) + 1)
         As = [A0] + [binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, dev)
                      for _ in range(ncopy - 1)]
         X = torch.from_numpy(w.X).cuda()
@@ -314,7 +316,9 @@ def spmv_sweep(binding, torch, dev, rates, batch, reps=10, with_cpu=False):
                     "GBps": round(alg / us / 1e3, 1), "frac_hbm_measured": round(alg / us / 1e3 / hbm, 4),
                     "frac_hbm_8TBps": round(alg / us / 1e3 / 8000.0, 4), "GFLOPs": round(2 * info["nnz"] * batch / us / 1e3, 1),
                     "us_warm_l2": round(us_warm, 3), "GBps_warm_l2": round(alg / us_warm / 1e3, 1),
-                    "balance": round(info["balance"], 3), "copies": ncopy})
+                    "balance": round(info["panel_balance"] if panel else info["balance"], 3), "copies": ncopy,
+                    "kernel": "csb_panel_kernel" if panel else "csb_product_kernel / csb_spmm_mma_kernel",
+                    "streamed_bytes": stream_bytes})
         if with_cpu and rate == rates[0]:
             out[-1]["cpu_csb_loops"] = cpu_csb_loops(m, w.X[0])
         for a in As:
@@ -457,10 +461,12 @@ def main():
         for r in line["spmv"]:
             r["frac_l2_warm"] = round(r["GBps_warm_l2"] / l2, 4)
         best = max(line["spmv"], key=lambda r: r["frac_hbm_measured"])
-        line["roofline_spmv"] = {"kernel": "csb_product_kernel<half,1>", "bound": "hbm", "achieved": best["GBps"], "peak": hbm,
+        line["roofline_spmv"] = {"kernel": best["kernel"], "bound": "hbm", "achieved": best["GBps"], "peak": hbm,
                                  "peak_kind": peak_kind, "unit": "GB/s", "frac": best["frac_hbm_measured"],
                                  "traffic": SPMV4X_DRAM_BYTES_PER_LAUNCH if best["rate"] == 4.0 else None,
-                                 "workload": "cfg4 8192x8192, 64x64 blocks, rate %gx, batch 1, cold (rotating copies > L2)" % best["rate"]}
+                                 "workload": "cfg4 8192x8192, 64x64 blocks, rate %gx, batch 1, cold (rotating copies > L2)" % best["rate"],
+                                 "launch": "back-to-back launches of one CUDA graph; the kernel is launched with programmatic stream "
+                                           "serialization, so a launch's start-up overlaps the end of the one in front (CSB_PANEL_PDL=0 turns it off)"}
     if rank == 0 and "spmm" in sections:
         line["spmm"] = []
         for bsz in [int(b) for b in args.spmm_batches.split(",")]:

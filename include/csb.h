@@ -87,6 +87,10 @@ typedef struct csb_info {
     int64_t device_stream_bytes; /* bytes of the private device layout actually streamed    */
     int32_t plan_ctas, plan_warps;
     double balance;              /* mean / max of the per-warp scheduled cost (1 = perfect) */
+    /* the panel layout that csb_spmv streams for fp16 matrices (all zero when it does not apply) */
+    int64_t panel_stream_bytes;  /* bytes of all panels (bookkeeping + values)              */
+    int32_t panel_ctas, panel_warps;
+    double panel_balance;        /* mean / max of the per-CTA modelled cost                 */
 } csb_info_t;
 
 /*
@@ -126,6 +130,11 @@ void csb_free(csb_matrix_t* A);
  *   become exactly 0).  fp32 accumulation, fixed summation order (bit-reproducible).
  * Asynchronous on `stream`.  Calls on the same handle must not overlap on the GPU: they share
  * the handle's scratch for partial block-row sums.
+ * Matrices with fp16 values (block_c <= 128, cols <= 16384) run the panel kernel: every CTA owns
+ * a range of output rows, so it needs no scratch.  That kernel is launched with programmatic
+ * stream serialization: its start-up overlaps the end of the work in front of it on `stream`,
+ * and it waits for that work before it reads x or writes y (set CSB_PANEL_PDL=0 in the
+ * environment for an ordinary launch, CSB_NO_PANEL=1 at encode time for the other kernel).
  */
 int csb_spmv(const csb_matrix_t* A, const float* x, float* y, void* stream);
 
@@ -168,7 +177,8 @@ int csb_spmm(const csb_matrix_t* A, const float* X, int64_t ldx, int batch, floa
  * written before it is read.  The array is shared by ALL handles and keeps the last call's
  * contents: two calls of this function that overlap on the GPU (different streams, or different
  * host threads without ordering between their streams) race on it and give wrong results.  Calls
- * queued on one stream are safe.  Results equal csb_spmv's bit for bit.
+ * queued on one stream are safe.  Results equal those of csb_spmv's stream kernel bit for bit
+ * (csb_spmv itself may run the panel kernel, whose summation order differs).
  * Errors: INVALID_ARG (null), UNSUPPORTED (host-only handle, limits, device ordinal > 63),
  * TIMEOUT (an earlier product on the handle gave up a bounded wait), CUDA.
  */

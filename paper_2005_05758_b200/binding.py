@@ -40,7 +40,9 @@ class csb_view_t(C.Structure):
 class csb_info_t(C.Structure):
     _fields_ = [("nnz", C.c_int64), ("pruning_rate", C.c_double), ("nio", C.c_double),
                 ("algorithmic_bytes", C.c_int64), ("device_stream_bytes", C.c_int64),
-                ("plan_ctas", C.c_int32), ("plan_warps", C.c_int32), ("balance", C.c_double)]
+                ("plan_ctas", C.c_int32), ("plan_warps", C.c_int32), ("balance", C.c_double),
+                ("panel_stream_bytes", C.c_int64), ("panel_ctas", C.c_int32), ("panel_warps", C.c_int32),
+                ("panel_balance", C.c_double)]
 
 
 _P = C.c_void_p

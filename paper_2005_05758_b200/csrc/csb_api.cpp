@@ -94,6 +94,11 @@ int csb_info(const csb_matrix_t* A, csb_info_t* o) {
     o->plan_ctas = A->product.ctas;
     o->plan_warps = A->product.warps;
     o->balance = A->product.balance;
+    o->panel_stream_bytes = 0; o->panel_ctas = 0; o->panel_warps = 0; o->panel_balance = 0.0;
+    if (A->panel && A->panel->built) {
+        o->panel_stream_bytes = A->panel->stream_bytes; o->panel_ctas = A->panel->ctas;
+        o->panel_warps = A->panel->warps; o->panel_balance = A->panel->balance;
+    }
     return CSB_OK;
 }
 
