@@ -199,6 +199,10 @@ int csb_spmv_static_scratch(const csb_matrix_t* A, const float* x, float* y, voi
  *            through device staging buffers on `stream` and waits for the result.
  * The first call for a given (W..., B) builds and caches the time-loop schedule and its
  * device state (allocates, synchronises); later calls reuse it.  T = 0 or B = 0 is a no-op.
+ * With B >= 16, fp16 values and block_r <= 64 the sequence is not run by the persistent kernel
+ * but step by step: per layer and step the batched product on tensor cores (as csb_spmm, same
+ * input-range rule) and one kernel with the gate arithmetic; same results within rounding, same
+ * arguments and flags (CSB_RNN_NO_STEPWISE=1 in the environment keeps the persistent kernel).
  * Errors: SHAPE (rows != 4H, cols != I_l + H, layers disagree), LAUNCH (grid cannot be
  * co-resident; nothing was launched), TIMEOUT (the bounded grid barrier gave up; outputs are
  * undefined, the context stays usable), CUDA.

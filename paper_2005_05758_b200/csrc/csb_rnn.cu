@@ -457,6 +457,7 @@ static unsigned long long g_barrier_ns = 2000ull * 1000ull * 1000ull;
 static unsigned int g_barrier_extra = 0;
 
 void drop_rnn_plans(const csb_matrix* A) {
+    drop_step_plans(A);
     std::lock_guard<std::mutex> lk(g_rnn_mu);
     int prev = 0;
     cudaGetDevice(&prev);
@@ -609,6 +610,12 @@ static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const flo
     CSB_CUDA(cudaGetDevice(&prev));
     CSB_CUDA(cudaSetDevice(W[0]->device));
     struct Restore { int d; ~Restore() { cudaSetDevice(d); } } restore{prev};
+
+    // LSTM at batch >= 16 with fp16 values: step by step, the products on tensor cores
+    if (rnn_stepwise_wanted(gates, L, W, B)) {
+        const int rc = rnn_forward_stepwise(L, W, bias, x, T, B, H, in_size, h0, c0, y, hT, cT, flags, stream);
+        if (rc != 1) return rc;
+    }
 
     RnnPlan* P = nullptr;
     {

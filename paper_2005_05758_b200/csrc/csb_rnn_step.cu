@@ -1,0 +1,200 @@
+// LSTM layers at larger batch, one timestep at a time on tensor cores.
+//
+// With a batch of 16 or more the per-step product of Section 2.1, W . [u_t ; h_{t-1}] for all
+// batch columns at once, is a dense contraction per block (kernel matrix times gathered inputs),
+// which the batched product kernel runs on tensor cores.  The persistent time-loop kernel keeps
+// that product on CUDA cores, so for these batches a step is issued as separate launches instead:
+// the batched product (pack + tensor-core kernel) of every layer, then one small kernel with the
+// gate arithmetic, which also routes h_t to where the next products read it.  The products of a
+// layer read one buffer V_l = [u_t ; h_{t-1}] of shape [B, I_l + H]; the gate kernel of layer l
+// writes h_t into the right part of V_l (for step t + 1) and into the left part of V_{l+1} (the
+// layer above, same step) or into y, and the gate kernel of layer 0 also moves x_{t+1} in.
+#include <algorithm>
+#include <list>
+#include <memory>
+#include <mutex>
+
+#include "csb_internal.hpp"
+
+namespace csb {
+
+#define CSB_CUDA(call)                                                                     \
+    do {                                                                                   \
+        cudaError_t e_ = (call);                                                           \
+        if (e_ != cudaSuccess) {                                                           \
+            set_error("%s failed: %s", #call, cudaGetErrorString(e_));                     \
+            return e_ == cudaErrorMemoryAllocation ? CSB_ERR_ALLOC : CSB_ERR_CUDA;         \
+        }                                                                                  \
+    } while (0)
+
+struct StepPlan {
+    std::vector<uint64_t> uids;
+    int L = 0, B = 0, H = 0, device = -1;
+    int in_size[kMaxLayers] = {};
+    float* d_v[kMaxLayers] = {};       // [B, in_size[l] + H] per layer
+    float* d_z = nullptr;              // [B, 4H] pre-activations of the layer being worked on
+    float* d_c = nullptr;              // [L, B, H] cell state
+    float* d_stage = nullptr;          // host-I/O staging of x and y
+    size_t stage_cap = 0;
+    ~StepPlan() {
+        for (float* p : d_v) cudaFree(p);
+        cudaFree(d_z); cudaFree(d_c); cudaFree(d_stage);
+    }
+};
+static std::mutex g_step_mu;
+static std::list<std::unique_ptr<StepPlan>> g_step_plans;
+
+void drop_step_plans(const csb_matrix* A) {
+    std::lock_guard<std::mutex> lk(g_step_mu);
+    int prev = 0;
+    cudaGetDevice(&prev);
+    for (auto it = g_step_plans.begin(); it != g_step_plans.end();) {
+        if (std::find((*it)->uids.begin(), (*it)->uids.end(), A->uid) != (*it)->uids.end()) {
+            cudaSetDevice((*it)->device);
+            it = g_step_plans.erase(it);
+        } else ++it;
+    }
+    cudaSetDevice(prev);
+}
+
+__device__ __forceinline__ float logistic(float a) { return 1.f / (1.f + expf(-a)); }
+
+// Gate arithmetic of one LSTM layer and step for the whole batch (Section 2.1):
+//   c_t = s(z_f) c_{t-1} + s(z_i) tanh(z_g),  h_t = s(z_o) tanh(c_t),  rows of z stacked i, f, g, o.
+// h_t goes to v_self[b, off_self + j] (this layer's next product), to v_next[b, j] (the layer
+// above) when there is one, and to y_t[b, j] when asked.  With x_next the kernel also copies the
+// next step's input rows into v0[b, 0 .. I).
+__global__ void csb_lstm_gates_kernel(const float* __restrict__ Z, const float* __restrict__ bias, float* __restrict__ c,
+                                      float* __restrict__ v_self, int ld_self, int off_self, float* __restrict__ v_next,
+                                      int ld_next, float* __restrict__ y_t, const float* __restrict__ x_next, int I,
+                                      float* __restrict__ v0, int ld0, int B, int H) {
+    const int n = B * H;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
+        const int b = e / H, j = e - b * H;
+        const float* z = Z + (size_t)b * 4 * H;
+        float zi = z[j], zf = z[H + j], zg = z[2 * H + j], zo = z[3 * H + j];
+        if (bias) { zi += bias[j]; zf += bias[H + j]; zg += bias[2 * H + j]; zo += bias[3 * H + j]; }
+        const float cn = logistic(zf) * c[e] + logistic(zi) * tanhf(zg);
+        const float h = logistic(zo) * tanhf(cn);
+        c[e] = cn;
+        v_self[(size_t)b * ld_self + off_self + j] = h;
+        if (v_next) v_next[(size_t)b * ld_next + j] = h;
+        if (y_t) y_t[e] = h;
+    }
+    if (x_next) {
+        const int nx = B * I;
+        for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < nx; e += gridDim.x * blockDim.x) {
+            const int b = e / I, i = e - b * I;
+            v0[(size_t)b * ld0 + i] = x_next[e];
+        }
+    }
+}
+
+static int env_flag(const char* name) {
+    const char* v = getenv(name);
+    return v && *v ? atoi(v) : 0;
+}
+
+bool rnn_stepwise_wanted(int gates, int L, const csb_matrix* const* W, int B) {
+    if (gates != 4 || B < 16 || env_flag("CSB_RNN_NO_STEPWISE")) return false;
+    for (int l = 0; l < L; ++l)
+        if (!spmm_mma_applicable(W[l], B)) return false;
+    return true;
+}
+
+// Returns CSB_OK, an error, or 1 when the tensor-core plan of a layer does not fit (nothing the
+// caller can see has been written then; the caller runs the persistent kernel instead).
+int rnn_forward_stepwise(int L, const csb_matrix* const* W, const float* const* bias, const float* x, int64_t T, int B, int H,
+                         const int* in_size, const float* h0, const float* c0, float* y, float* hT, float* cT, unsigned flags,
+                         void* stream) {
+    StepPlan* P = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(g_step_mu);
+        for (auto& p : g_step_plans) {
+            if (p->L != L || p->B != B) continue;
+            bool same = true;
+            for (int l = 0; l < L; ++l) same = same && p->uids[l] == W[l]->uid;
+            if (same) { P = p.get(); break; }
+        }
+        if (!P) {
+            std::unique_ptr<StepPlan> np(new StepPlan());
+            np->L = L; np->B = B; np->H = H; np->device = W[0]->device;
+            for (int l = 0; l < L; ++l) {
+                np->uids.push_back(W[l]->uid);
+                np->in_size[l] = in_size[l];
+                CSB_CUDA(cudaMalloc((void**)&np->d_v[l], (size_t)B * (in_size[l] + H) * 4));
+            }
+            CSB_CUDA(cudaMalloc((void**)&np->d_z, (size_t)B * 4 * H * 4));
+            CSB_CUDA(cudaMalloc((void**)&np->d_c, (size_t)L * B * H * 4));
+            P = np.get();
+            g_step_plans.push_back(std::move(np));
+        }
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool host_io = (flags & CSB_FLAG_HOST_IO) != 0;
+    const int I0 = in_size[0];
+    const size_t nx = (size_t)T * B * I0, ny = (size_t)T * B * H, ns = (size_t)L * B * H;
+    const float* dx = x;
+    float* dy = y;
+    if (host_io) {
+        const size_t need = nx + (y ? ny : 0);
+        if (need > P->stage_cap) {
+            CSB_CUDA(cudaStreamSynchronize(st));
+            cudaFree(P->d_stage); P->d_stage = nullptr; P->stage_cap = 0;
+            CSB_CUDA(cudaMalloc((void**)&P->d_stage, need * 4));
+            P->stage_cap = need;
+        }
+        CSB_CUDA(cudaMemcpyAsync(P->d_stage, x, nx * 4, cudaMemcpyHostToDevice, st));
+        dx = P->d_stage;
+        dy = y ? P->d_stage + nx : nullptr;
+    }
+    const cudaMemcpyKind in_kind = host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
+    const cudaMemcpyKind out_kind = host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice;
+    const size_t hrow = (size_t)H * 4;
+    // V_l = [u_0 ; h_{-1}]: h0 (or zeros) on the right, x_0 on the left of layer 0
+    for (int l = 0; l < L; ++l) {
+        const int ld = in_size[l] + H;
+        if (h0) CSB_CUDA(cudaMemcpy2DAsync(P->d_v[l] + in_size[l], (size_t)ld * 4, h0 + (size_t)l * B * H, hrow, hrow, B, in_kind, st));
+        else CSB_CUDA(cudaMemset2DAsync(P->d_v[l] + in_size[l], (size_t)ld * 4, 0, hrow, B, st));
+    }
+    CSB_CUDA(cudaMemcpy2DAsync(P->d_v[0], (size_t)(I0 + H) * 4, dx, (size_t)I0 * 4, (size_t)I0 * 4, B, cudaMemcpyDeviceToDevice, st));
+    if (c0) CSB_CUDA(cudaMemcpyAsync(P->d_c, c0, ns * 4, in_kind, st));
+    else CSB_CUDA(cudaMemsetAsync(P->d_c, 0, ns * 4, st));
+
+    const int threads = 256;
+    const int blocks = std::max(1, std::min(1024, (B * std::max(H, I0) + threads - 1) / threads));
+    for (int64_t t = 0; t < T; ++t) {
+        for (int l = 0; l < L; ++l) {
+            const int ld = in_size[l] + H;
+            const int rc = launch_spmm_mma(W[l], P->d_v[l], ld, B, P->d_z, 4 * (int64_t)H, stream);
+            if (rc != CSB_OK) {
+                // in step 0 only scratch has been written so far (y is written behind the top layer's product)
+                if (rc == 1 && t > 0) { set_error("the tensor-core plan of layer %d became unusable in mid-sequence", l); return CSB_ERR_CUDA; }
+                return rc;
+            }
+            const bool top = l == L - 1;
+            const float* x_next = (l == 0 && t + 1 < T) ? dx + (size_t)(t + 1) * B * I0 : nullptr;
+            csb_lstm_gates_kernel<<<blocks, threads, 0, st>>>(P->d_z, bias ? bias[l] : nullptr, P->d_c + (size_t)l * B * H, P->d_v[l], ld,
+                                                             in_size[l], top ? nullptr : P->d_v[l + 1], top ? 0 : in_size[l + 1] + H,
+                                                             (top && dy) ? dy + (size_t)t * B * H : nullptr, x_next, I0, P->d_v[0],
+                                                             I0 + H, B, H);
+            CSB_CUDA(cudaGetLastError());
+        }
+    }
+    if (hT)
+        for (int l = 0; l < L; ++l)
+            CSB_CUDA(cudaMemcpy2DAsync(hT + (size_t)l * B * H, hrow, P->d_v[l] + in_size[l], (size_t)(in_size[l] + H) * 4, hrow, B, out_kind, st));
+    if (cT) CSB_CUDA(cudaMemcpyAsync(cT, P->d_c, ns * 4, out_kind, st));
+    if (host_io && y) CSB_CUDA(cudaMemcpyAsync(y, dy, ny * 4, cudaMemcpyDeviceToHost, st));
+    if (host_io || !(flags & CSB_FLAG_ASYNC)) {
+        CSB_CUDA(cudaStreamSynchronize(st));
+        for (int l = 0; l < L; ++l)
+            if (W[l]->product.h_status && *W[l]->product.h_status != 0) {
+                set_error("a product kernel of layer %d gave up a bounded wait (code %u)", l, *W[l]->product.h_status);
+                return CSB_ERR_TIMEOUT;
+            }
+    }
+    return CSB_OK;
+}
+
+}  // namespace csb

@@ -121,6 +121,32 @@ def test_resume_equals_one_call_bitwise_and_host_io():
     assert np.array_equal(y1, y3) and np.array_equal(h1, h3) and np.array_equal(c1, c3)
 
 
+@pytest.mark.parametrize("B,I,H,L,br,bc", [(16, 40, 48, 2, 16, 16), (32, 153, 160, 1, 32, 32), (40, 70, 192, 2, 64, 32)])
+def test_lstm_large_batch_runs_step_by_step_on_tensor_cores(B, I, H, L, br, bc):
+    # batches of 16 and more take the path of one product (tensor cores) + one gate kernel per layer
+    # and step; bias, initial states, resumption and host I/O as for the persistent kernel
+    w = workloads.make_rnn_workload(31, "lstm", I, H, L, br, bc, "lognormal", rate=4.0, T=6, B=B, w_std=0.15,
+                                    bias_std=0.2, state_std=0.4)
+    y1, h1, c1 = check(w)
+    y2, h2, c2 = run(w, chunks=[(0, 2), (2, 6)])
+    assert np.array_equal(y1, y2) and np.array_equal(h1, h2) and np.array_equal(c1, c2)
+    y3, h3, c3 = run(w, host_io=True)
+    assert np.array_equal(y1, y3) and np.array_equal(h1, h3) and np.array_equal(c1, c3)
+
+
+def test_lstm_large_batch_both_paths_agree(monkeypatch):
+    w = workloads.make_rnn_workload(32, "lstm", 64, 128, 2, 32, 32, "uniform", lo=0.3, hi=0.7, T=5, B=24, w_std=0.1,
+                                    bias_std=0.1, state_std=0.2)
+    ya, ha, ca = check(w)
+    monkeypatch.setenv("CSB_RNN_NO_STEPWISE", "1")       # the persistent kernel, CUDA cores
+    yb, hb, cb = check(w)
+    assert np.max(np.abs(ya - yb)) < 1e-4
+
+
+def test_cfg5_batch32_reduced_length():
+    check(workloads.CONFIGS["cfg5"](T=3, B=32))
+
+
 def test_zero_weight_closed_forms():
     w = workloads.make_rnn_workload(2, "gru", 16, 32, 1, 8, 8, "uniform", lo=0.5, hi=0.5, T=6, B=2, w_std=0.1, state_std=1.0)
     w.layers[0].dense[:] = 0
