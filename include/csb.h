@@ -223,10 +223,11 @@ int csb_gru_forward(int n_layers, const csb_matrix_t* const* W, const float* con
                     unsigned flags, void* stream);
 
 /*
- * csb_test_barrier_hook -- testing aid for the give-up path of the time loop's grid barrier
- * (the paper has no counterpart).  Makes every later recurrent call expect `extra_arrivals`
- * arrivals that never come and bounds each barrier wait to `limit_ns` nanoseconds, so the
- * kernel returns with CSB_ERR_TIMEOUT instead of completing; (0, 0) restores normal operation
+ * csb_test_barrier_hook -- testing aid for the give-up path of the time loop's waits on other
+ * CTAs (the paper has no counterpart).  Makes every later recurrent call expect `extra_arrivals`
+ * arrivals at its grid barrier that never come (at batch 1, where CTAs exchange h as flagged
+ * values instead: wait for a step number that never comes) and bounds each such wait to
+ * `limit_ns` nanoseconds, so the kernel returns with CSB_ERR_TIMEOUT instead of completing; (0, 0) restores normal operation
  * (no extra arrivals, 2 s bound).  Process-wide; not for production use.
  */
 void csb_test_barrier_hook(unsigned int extra_arrivals, unsigned long long limit_ns);

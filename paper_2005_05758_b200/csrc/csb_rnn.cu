@@ -36,6 +36,10 @@ struct RnnArgs {
     int T, B, H, L, gates, stage_bytes, stages, resident, max_warp_bytes, max_U, max_C;
     int v_tile;                // batched: [u_t ; h_{t-1}] of the current batch tile is staged in shared memory, [bt][column]
     int v_bulk;                // batch 1: [u_t ; h_{t-1}] may come in by bulk copy (16-byte aligned pieces)
+    // batch 1, flagged exchange of h (below): every h value travels with the number of its step
+    uint2* hll;                // [L][4][H] pairs (bits of h, step + 2), zero at launch; null = grid-barrier time loop
+    unsigned int* progress;    // [L] CTAs-times-steps whose input has been read, zero at launch
+    int layer_ctas[kMaxLayers];
 #ifdef CSB_PHASE_CLOCKS
     long long* clocks;         // [n_ctas][5] cycles summed over ticks: stage, walk, reduce, gates, barrier
 #endif
@@ -104,6 +108,23 @@ __device__ __forceinline__ bool grid_wait(const RnnArgs& a, unsigned int target,
 }
 
 __device__ __forceinline__ float sigmoidf_acc(float a) { return 1.f / (1.f + expf(-a)); }
+
+// Flagged exchange of h at batch 1.  A value and the number of the step it belongs to are written
+// with ONE aligned 8-byte store and read with one 8-byte load, so a reader that sees the step
+// number it is waiting for also holds the value: no fence, no counter, no second trip to memory.
+__device__ __forceinline__ void st_flagged(uint2* p, float v, uint32_t tag) {
+    asm volatile("st.volatile.global.v2.u32 [%0], {%1, %2};" ::"l"(p), "r"(__float_as_uint(v)), "r"(tag) : "memory");
+}
+__device__ __forceinline__ uint2 ld_flagged(const uint2* p) {
+    uint2 v;
+    asm volatile("ld.volatile.global.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned int ld_relaxed_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
 
 // Time loop.  Tick k: layer l works on step t = k - lag*l (lag = 2 above the first layer).  Inside
 // a tick a CTA
@@ -301,6 +322,154 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
         __syncwarp();
     };
 
+
+    // ------------------------------------------------------------------------------------------
+    // Batch 1 with the flagged exchange: no grid barrier.  Every CTA runs through its own steps;
+    // what it needs from others (h_{t-1} of its layer, h_t of the layer below) it reads as
+    // (value, step) pairs and spins on the step number, what it produces it publishes the same
+    // way.  h of step s sits in slot s & 3; before a CTA overwrites a slot it makes sure the layer
+    // above has read the step that is four back (a per-layer count of "CTA has read its input of
+    // step s", looked at one tick late, so it is off the critical path).  Every spin is bounded.
+    if (BT == 1 && a.hll != nullptr) {
+        uint2* ll_self = a.hll + (size_t)layer * 4 * H;
+        const uint2* ll_below = layer > 0 ? a.hll + (size_t)(layer - 1) * 4 * H : nullptr;
+        const uint32_t never = a.barrier_extra ? 0x40000000u : 0u;     // test hook: wait for a step that never comes
+        // read n flagged values of step `step` into shared memory; false = gave up (CTA-uniform after the barrier)
+        auto stage_flagged = [&](float* dst, const uint2* src, int n, int step) {
+            const uint32_t want = (uint32_t)(step + 2) + never;
+            for (int i0 = threadIdx.x; i0 < n; i0 += 4 * blockDim.x) {
+                uint2 v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { const int i = i0 + j * blockDim.x; v[j] = i < n ? ld_flagged(src + i) : make_uint2(0u, want); }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int i = i0 + j * blockDim.x;
+                    if (i >= n) continue;
+                    unsigned long long t0 = 0;
+                    unsigned int spins = 0;
+                    while (v[j].y != want) {
+                        if (*s_flag == 0) break;
+                        if ((++spins & 63u) == 0) {
+                            const unsigned long long now = global_ns();
+                            if (t0 == 0) t0 = now;
+                            else if (now - t0 > a.barrier_ns) { *(volatile uint32_t*)a.status = (uint32_t)kDevBarrierTimeout; *s_flag = 0; break; }
+                        }
+                        v[j] = ld_flagged(src + i);
+                    }
+                    dst[i] = __uint_as_float(v[j].x);
+                }
+            }
+        };
+        // h0 of this tile becomes "step -1" of the exchange
+        for (int u = threadIdx.x; u < U; u += blockDim.x)
+            st_flagged(ll_self + (size_t)3 * H + u0 + u, __ldcg(h_slot(layer, -1) + u0 + u), 1u);
+        unsigned int above_seen = 0;
+        for (int t = 0; t < a.T; ++t) {
+            // ---- input half: x_t, or h_t of the layer below
+            if (layer == 0) {
+                if (t == 0) stage_issue(0, vs, a.x, I);                // later steps: issued a step ahead, below
+                stage_wait(0, vs, a.x + (size_t)t * I, I);
+                if (a.v_bulk) __syncthreads();
+            } else { stage_flagged(vs, ll_below + (size_t)(t & 3) * H, I, t); __syncthreads(); }
+            RNN_LAP(0);
+            if (*s_flag == 0 || !__syncthreads_and(alive)) break;
+            if (layer > 0 && threadIdx.x == 0) atomicAdd(a.progress + layer, 1u);      // this CTA has read its input of step t
+            // the count of the layer above is asked for now and used at the end of the step
+            unsigned int above_now = above_seen;
+            const bool need_above = layer + 1 < a.L && t >= 4;
+            if (need_above && threadIdx.x == 0) above_now = ld_relaxed_u32(a.progress + layer + 1);
+            zero_zs();
+            walk_part(0, nullptr, nullptr, 0, 1);
+            // ---- recurrent half: h_{t-1} of this layer from every CTA of the layer
+            RNN_LAP(1);
+            stage_flagged(vs + I, ll_self + (size_t)((t - 1) & 3) * H, H, t - 1);
+            __syncthreads();
+            if (*s_flag == 0) break;
+            RNN_LAP(4);
+            // every warp is past the input half of vs: the next step's x may come in (bulk copy only;
+            // without it stage_wait loads at the top of the step)
+            if (layer == 0 && t + 1 < a.T) stage_issue(0, vs, a.x + (size_t)(t + 1) * I, I);
+            walk_part(1, nullptr, nullptr, 0, 1);
+            __syncthreads();
+            RNN_LAP(1);
+            // ---- add the accumulator copies, bias and activations (as in the barrier loop below)
+            {
+                const int NZ = 4 * U, NC = W * G;
+                int parts = 1;
+                while (parts < 32 && parts * 2 * NZ <= (int)blockDim.x) parts *= 2;
+                const int span = (NZ * parts + 31) & ~31;
+                for (int idx = threadIdx.x; idx < span; idx += blockDim.x) {
+                    const int e = idx / parts, pt = idx % parts;
+                    float sum = 0.f;
+                    if (e < NZ) {
+                        const float* src = zs_all + e;
+                        for (int c = pt; c < NC; c += 8 * parts) {
+                            float v[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) v[j] = (c + j * parts < NC) ? src[(c + j * parts) * S.zs_stride] : 0.f;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) sum += v[j];
+                        }
+                    }
+                    for (int off = parts >> 1; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+                    if (e < NZ && pt == 0) {
+                        const int g = e / U, u = e % U;
+                        float z = sum + (bias ? __ldg(bias + g * H + u0 + u) : 0.f);
+                        if (a.gates == 4) z = g == 2 ? tanhf(z) : sigmoidf_acc(z);
+                        else if (g < 2) z = sigmoidf_acc(z);
+                        zsum[e] = z;
+                    }
+                }
+            }
+            // slot t & 3 still holds step t - 4: the layer above must have read it
+            if (need_above && threadIdx.x == 0) {
+                const unsigned int need = (unsigned int)(t - 3) * (unsigned int)a.layer_ctas[layer + 1];
+                unsigned long long t0 = 0;
+                unsigned int spins = 0;
+                while (above_now < need) {
+                    if ((++spins & 63u) == 0) {
+                        const unsigned long long now = global_ns();
+                        if (t0 == 0) t0 = now;
+                        else if (now - t0 > a.barrier_ns) { *(volatile uint32_t*)a.status = (uint32_t)kDevBarrierTimeout; *s_flag = 0; break; }
+                    }
+                    above_now = ld_relaxed_u32(a.progress + layer + 1);
+                }
+                above_seen = above_now;
+            }
+            __syncthreads();
+            if (*s_flag == 0) break;
+            RNN_LAP(2);
+            // ---- gates, state, publish
+            float* h_dst = h_slot(layer, t);
+            for (int u = threadIdx.x; u < U; u += blockDim.x) {
+                float z[4];
+#pragma unroll
+                for (int g = 0; g < 4; ++g) z[g] = zsum[g * U + u];
+                float h;
+                if (a.gates == 4) {
+                    const float c = z[1] * cs[u] + z[0] * z[2];
+                    cs[u] = c;
+                    h = z[3] * tanhf(c);
+                    if (t == a.T - 1) a.cstate[(size_t)layer * H + u0 + u] = c;
+                } else {
+                    const float n = tanhf(z[2] + z[0] * z[3]);
+                    const float hp = vs[I + u0 + u];                   // h_{t-1}, staged above
+                    h = (1.f - z[1]) * n + z[1] * hp;
+                }
+                st_flagged(ll_self + (size_t)(t & 3) * H + u0 + u, h, (uint32_t)(t + 2));
+                h_dst[u0 + u] = h;
+                if (layer == a.L - 1 && a.y) a.y[(size_t)t * H + u0 + u] = h;
+            }
+            __syncthreads();
+            RNN_LAP(3);
+        }
+#ifdef CSB_PHASE_CLOCKS
+        if (threadIdx.x == 0) for (int i = 0; i < 5; ++i) a.clocks[(size_t)blockIdx.x * 5 + i] = rprof[i];
+#endif
+        if (!alive && lane == 0) *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout;
+        return;
+    }
+
     bool pre_done = false;        // the input half of the coming step is already in the accumulators
     bool in_flight = false;       // the copy of the coming step's input half has been issued
     for (int tick = 0; tick < n_ticks; ++tick) {
@@ -442,11 +611,13 @@ struct RnnPlan {
     int64_t stream_bytes = 0;
     uint8_t* d_stream = nullptr; Chunk* d_chunks = nullptr; uint32_t* d_wcb = nullptr; uint32_t* d_win = nullptr; RnnCtaDesc* d_ctas = nullptr;
     float* d_hbuf = nullptr; float* d_cstate = nullptr; unsigned int* d_barrier = nullptr;
+    uint2* d_hll = nullptr; unsigned int* d_progress = nullptr;      // flagged exchange of h (batch 1)
+    int layer_ctas[kMaxLayers] = {};
     uint32_t* h_status = nullptr; uint32_t* d_status = nullptr;
     float* d_stage = nullptr; size_t stage_cap = 0;      // host-I/O staging: x, y, states
     ~RnnPlan() {
         cudaFree(d_stream); cudaFree(d_chunks); cudaFree(d_wcb); cudaFree(d_win); cudaFree(d_ctas); cudaFree(d_hbuf);
-        cudaFree(d_cstate); cudaFree(d_barrier); cudaFree(d_stage);
+        cudaFree(d_cstate); cudaFree(d_barrier); cudaFree(d_stage); cudaFree(d_hll); cudaFree(d_progress);
         if (h_status) cudaFreeHost(h_status);
     }
 };
@@ -538,6 +709,11 @@ static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, i
     CSB_CUDA(cudaMalloc((void**)&P->d_hbuf, (size_t)L * 4 * B * H * 4));
     CSB_CUDA(cudaMalloc((void**)&P->d_cstate, (size_t)L * B * H * 4));
     CSB_CUDA(cudaMalloc((void**)&P->d_barrier, 4));
+    for (const RnnCtaDesc& cd : Hp.ctas) ++P->layer_ctas[cd.layer];
+    if (P->BT == 1) {
+        CSB_CUDA(cudaMalloc((void**)&P->d_hll, (size_t)L * 4 * H * sizeof(uint2)));
+        CSB_CUDA(cudaMalloc((void**)&P->d_progress, (size_t)kMaxLayers * 4));
+    }
     CSB_CUDA(cudaHostAlloc((void**)&P->h_status, 4, cudaHostAllocMapped));
     *P->h_status = 0;
     CSB_CUDA(cudaHostGetDevicePointer((void**)&P->d_status, P->h_status, 0));
@@ -680,6 +856,14 @@ static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const flo
         for (int l = 0; l < L; ++l) if (in_size[l] % 4) a.v_bulk = 0;
     }
     if (env_int("CSB_RNN_NO_VBULK", 0)) a.v_bulk = 0;
+    a.hll = nullptr; a.progress = P->d_progress;
+    for (int l = 0; l < L; ++l) a.layer_ctas[l] = P->layer_ctas[l];
+    if (P->BT == 1 && P->d_hll && !env_int("CSB_RNN_NO_FLAGGED", 0)) {
+        // every pair starts as "no step" and the read counts at zero
+        CSB_CUDA(cudaMemsetAsync(P->d_hll, 0, (size_t)L * 4 * H * sizeof(uint2), st));
+        CSB_CUDA(cudaMemsetAsync(P->d_progress, 0, (size_t)kMaxLayers * 4, st));
+        a.hll = P->d_hll;
+    }
     a.resident = P->resident; a.max_warp_bytes = P->max_warp_bytes; a.max_U = P->max_U; a.max_C = P->max_C;
 #ifdef CSB_PHASE_CLOCKS
     static long long* d_rclocks = nullptr;
