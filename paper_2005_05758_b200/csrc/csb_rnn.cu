@@ -41,7 +41,7 @@ struct RnnArgs {
     unsigned int* progress;    // [L] CTAs-times-steps whose input has been read, zero at launch
     int layer_ctas[kMaxLayers];
 #ifdef CSB_PHASE_CLOCKS
-    long long* clocks;         // [n_ctas][5] cycles summed over ticks: stage, walk, reduce, gates, barrier
+    long long* clocks;         // [n_ctas][8] cycles summed over ticks: stage, walk, reduce, gates, barrier / wait for h, sums only, slot guard
 #endif
 };
 
@@ -220,7 +220,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     auto input_of = [&](int step) -> const float* { return layer == 0 ? a.x + (size_t)step * B * I : h_slot(layer - 1, step); };
     const int in_ld = layer == 0 ? I : H;
 #ifdef CSB_PHASE_CLOCKS
-    long long rprof[5] = {0, 0, 0, 0, 0};
+    long long rprof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     long long rt = clock64();
 #endif
 
@@ -421,6 +421,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                     }
                 }
             }
+            RNN_LAP(5);
             // slot t & 3 still holds step t - 4: the layer above must have read it
             if (need_above && threadIdx.x == 0) {
                 const unsigned int need = (unsigned int)(t - 3) * (unsigned int)a.layer_ctas[layer + 1];
@@ -436,6 +437,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                 }
                 above_seen = above_now;
             }
+            RNN_LAP(6);
             __syncthreads();
             if (*s_flag == 0) break;
             RNN_LAP(2);
@@ -464,7 +466,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
             RNN_LAP(3);
         }
 #ifdef CSB_PHASE_CLOCKS
-        if (threadIdx.x == 0) for (int i = 0; i < 5; ++i) a.clocks[(size_t)blockIdx.x * 5 + i] = rprof[i];
+        if (threadIdx.x == 0) for (int i = 0; i < 8; ++i) a.clocks[(size_t)blockIdx.x * 8 + i] = rprof[i];
 #endif
         if (!alive && lane == 0) *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout;
         return;
@@ -585,7 +587,7 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
     }
     if (!alive && lane == 0) *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout;
 #ifdef CSB_PHASE_CLOCKS
-    if (threadIdx.x == 0) for (int i = 0; i < 5; ++i) a.clocks[(size_t)blockIdx.x * 5 + i] = rprof[i];
+    if (threadIdx.x == 0) for (int i = 0; i < 8; ++i) a.clocks[(size_t)blockIdx.x * 8 + i] = rprof[i];
 #endif
 }
 
@@ -755,7 +757,7 @@ static int dispatch_rnn_gw(const RnnPlan* P, RnnArgs& a, cudaStream_t st) {
 static long long* g_rnn_clocks = nullptr;
 static int g_rnn_clock_ctas = 0;
 extern "C" int csb_debug_rnn_clocks(long long* host_out, int max_ctas) {
-    cudaMemcpy(host_out, g_rnn_clocks, (size_t)std::min(max_ctas, g_rnn_clock_ctas) * 5 * 8, cudaMemcpyDeviceToHost);
+    cudaMemcpy(host_out, g_rnn_clocks, (size_t)std::min(max_ctas, g_rnn_clock_ctas) * 8 * 8, cudaMemcpyDeviceToHost);
     return g_rnn_clock_ctas;
 }
 #endif
