@@ -191,15 +191,25 @@ __global__ void __launch_bounds__(1024, 1) csb_panel_kernel(const __grid_constan
     const PanelHeader* H = reinterpret_cast<const PanelHeader*>(meta);
     PANEL_STAMP(2);
     if (!gave_up) {
-        // ---- gather the kept inputs of every block of the panel, once: a warp per block
+        // ---- gather the kept inputs of every block of the panel, once: four blocks per warp and
+        // round, eight lanes per block, a lane resolves four column indices at a time (indices and
+        // gathered inputs of a block are padded to four; padding indices are zero, i.e. the block's
+        // first column, which exists)
         {
             const uint2* gath = reinterpret_cast<const uint2*>(meta + H->gather_off);
             const uint8_t* cidx = meta + H->cidx_off;
             const int n_gather = (int)H->n_gather;
-            for (int g = warp; g < n_gather; g += W) {
-                const uint2 gd = gath[g];
+            for (int g0 = warp * 4; g0 < n_gather; g0 += W * 4) {
+                const int g = g0 + (lane >> 3);
+                const uint2 gd = g < n_gather ? gath[g] : make_uint2(0u, 0u);
                 const uint32_t xbase = gd.x & 0xffffu, n = gd.x >> 16, xoff = gd.y;
-                for (uint32_t k = lane; k < n; k += 32) xg[xoff + k] = xs[xbase + cidx[xoff + k]];
+                for (uint32_t k = (uint32_t)(lane & 7) * 4u; k < n; k += 32u) {
+                    const uint32_t c4 = *reinterpret_cast<const uint32_t*>(cidx + xoff + k);
+                    float4 v;
+                    v.x = xs[xbase + (c4 & 0xffu)]; v.y = xs[xbase + ((c4 >> 8) & 0xffu)];
+                    v.z = xs[xbase + ((c4 >> 16) & 0xffu)]; v.w = xs[xbase + (c4 >> 24)];
+                    *reinterpret_cast<float4*>(xg + xoff + k) = v;
+                }
             }
         }
         __syncthreads();

@@ -364,6 +364,18 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
         for (int u = threadIdx.x; u < U; u += blockDim.x)
             st_flagged(ll_self + (size_t)3 * H + u0 + u, __ldcg(h_slot(layer, -1) + u0 + u), 1u);
         unsigned int above_seen = 0;
+        // the sums after the walk: `parts` adjacent lanes share one accumulator entry, each adds every
+        // parts-th copy in order, a fixed xor-tree joins them; the lane that holds the total applies
+        // bias and the gate's activation.  One entry per thread, the same in every step.
+        const int NZ = 4 * U, NC = W * G;
+        int lp = 0;
+        while (lp < 5 && (2 << lp) * NZ <= (int)blockDim.x) ++lp;
+        const int parts = 1 << lp;
+        const int my_e = (int)threadIdx.x >> lp, my_pt = (int)threadIdx.x & (parts - 1);
+        const bool one_entry = NZ * parts <= (int)blockDim.x;
+        const bool sum_active = (int)threadIdx.x < ((NZ * parts + 31) & ~31);
+        const int my_g = my_e / U, my_u = my_e % U;
+        const float my_bias = (bias && my_e < NZ) ? __ldg(bias + my_g * H + u0 + my_u) : 0.f;
         for (int t = 0; t < a.T; ++t) {
             // ---- input half: x_t, or h_t of the layer below
             if (layer == 0) {
@@ -392,33 +404,38 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
             walk_part(1, nullptr, nullptr, 0, 1);
             __syncthreads();
             RNN_LAP(1);
-            // ---- add the accumulator copies, bias and activations (as in the barrier loop below)
-            {
-                const int NZ = 4 * U, NC = W * G;
-                int parts = 1;
-                while (parts < 32 && parts * 2 * NZ <= (int)blockDim.x) parts *= 2;
-                const int span = (NZ * parts + 31) & ~31;
-                for (int idx = threadIdx.x; idx < span; idx += blockDim.x) {
-                    const int e = idx / parts, pt = idx % parts;
+            // ---- add the accumulator copies, bias and activations (the thread's entry, its share of
+            // the copies and its bias were worked out before the loop)
+            if (!one_entry) {
+                // more entries than threads (few warps, wide tile): every thread takes several
+                for (int e = threadIdx.x; e < NZ; e += blockDim.x) {
                     float sum = 0.f;
-                    if (e < NZ) {
-                        const float* src = zs_all + e;
-                        for (int c = pt; c < NC; c += 8 * parts) {
-                            float v[8];
+                    for (int c = 0; c < NC; ++c) sum += zs_all[e + c * S.zs_stride];
+                    const int g = e / U, u = e % U;
+                    float z = sum + (bias ? __ldg(bias + g * H + u0 + u) : 0.f);
+                    if (a.gates == 4) z = g == 2 ? tanhf(z) : sigmoidf_acc(z);
+                    else if (g < 2) z = sigmoidf_acc(z);
+                    zsum[e] = z;
+                }
+            } else if (sum_active) {
+                float sum = 0.f;
+                if (my_e < NZ) {
+                    const float* src = zs_all + my_e;
+                    for (int c = my_pt; c < NC; c += 8 * parts) {       // eight loads in flight, added in order
+                        float v[8];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) v[j] = (c + j * parts < NC) ? src[(c + j * parts) * S.zs_stride] : 0.f;
+                        for (int j = 0; j < 8; ++j) v[j] = (c + j * parts < NC) ? src[(c + j * parts) * S.zs_stride] : 0.f;
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) sum += v[j];
-                        }
+                        for (int j = 0; j < 8; ++j) sum += v[j];
                     }
-                    for (int off = parts >> 1; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-                    if (e < NZ && pt == 0) {
-                        const int g = e / U, u = e % U;
-                        float z = sum + (bias ? __ldg(bias + g * H + u0 + u) : 0.f);
-                        if (a.gates == 4) z = g == 2 ? tanhf(z) : sigmoidf_acc(z);
-                        else if (g < 2) z = sigmoidf_acc(z);
-                        zsum[e] = z;
-                    }
+                }
+                for (int off = parts >> 1; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+                RNN_LAP(7);
+                if (my_e < NZ && my_pt == 0) {
+                    float z = sum + my_bias;
+                    if (a.gates == 4) z = my_g == 2 ? tanhf(z) : sigmoidf_acc(z);
+                    else if (my_g < 2) z = sigmoidf_acc(z);
+                    zsum[my_e] = z;
                 }
             }
             RNN_LAP(5);
