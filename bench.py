@@ -327,6 +327,33 @@ def spmv_sweep(binding, torch, dev, rates, batch, reps=10, with_cpu=False):
     return out
 
 
+def project_bench(binding, torch, reps=20):
+    """Projection onto the CSB pattern (RowPrune / ColumnPrune of Algorithm 1) of an 8192x8192 dense
+    weight, 64x64 blocks, 4x: two passes over the matrix plus two selections, device-resident input.
+    Launches rotate over two matrices (2 x 268 MB > L2)."""
+    hbm, _ = peaks()
+    R = C = 8192
+    g = torch.Generator(device="cuda").manual_seed(0)
+    Ws = [torch.randn((R, C), device="cuda", generator=g) * 0.05 for _ in range(2)]
+    rk, ck, ws = binding.csb_project(Ws[0], 64, 64, 0.75)
+    for i in range(3):
+        binding.csb_project(Ws[i % 2], 64, 64, 0.75, rk, ck, ws)
+    torch.cuda.synchronize()
+    ts = []
+    for i in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); binding.csb_project(Ws[i % 2], 64, 64, 0.75, rk, ck, ws); b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b) * 1e3)
+    us = float(np.median(ts))
+    nbr = nbc = 128
+    alg = 2 * R * C * 4 + 2 * (nbc * R + nbr * C) * 8 + 2 * nbr * nbc * 64     # two reads of W, norms written and read, masks
+    kept = float(rk.float().mean() * ck.float().mean())
+    return {"workload": "8192x8192 fp32, 64x64 blocks, prune_fraction 0.75", "us": round(us, 1), "algorithmic_bytes": alg,
+            "GBps": round(alg / us / 1e3, 1), "frac_hbm_measured": round(alg / us / 1e3 / hbm, 4), "kept_rows_x_cols": round(kept, 4),
+            "launches_per_call": 4}
+
+
 def slowest_rank_ms(local_ms, dist=None, device="cpu"):
     """Replicas only: every rank runs its own sequences with no data-path collective; the job's
     time for a step is the slowest rank's (max over ranks of the device-timed mean)."""
@@ -370,7 +397,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="rnn,e2e,spmv,spmm,configs,cpu",
+    ap.add_argument("--sections", default="rnn,e2e,spmv,spmm,project,configs,cpu",
                     help="comma list of: rnn (always), e2e, spmv, spmm, configs, cpu")
     ap.add_argument("--seq-len", type=int, default=512)
     ap.add_argument("--spmv-rates", default="4,8,16,25", help="pruning rates of the bare SpMV sweep")
@@ -474,6 +501,8 @@ def main():
         for bsz in [int(b) for b in args.spmm_batches.split(",")]:
             line["spmm"] += spmv_sweep(binding, torch, local, [float(r) for r in args.spmv_rates.split(",")], bsz,
                                        reps=args.spmv_reps)
+    if rank == 0 and "project" in sections:
+        line["project"] = project_bench(binding, torch)
     if rank == 0 and "configs" in sections:
         line["configs"] = other_configs(binding, torch, local, flush, quick=False)
     if rank == 0 and "cpu" in sections:

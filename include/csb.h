@@ -112,6 +112,29 @@ int csb_encode(const float* dense, int64_t rows, int64_t cols, int64_t ld, int b
                const uint8_t* row_keep, const uint8_t* col_keep, int val_dtype, int device,
                const csb_plan_opts* opts, csb_matrix_t** out);
 
+/*
+ * csb_project -- project a dense weight onto the CSB pattern: the RowPrune / ColumnPrune step of
+ * Algorithm 1 (Section 3.2), which gives the keep masks csb_encode takes.  RowPrune: in every
+ * block-column on its own, the squared l2-norm of each row segment (the part of a matrix row inside
+ * the block-column) is taken and the weakest segments are pruned; ColumnPrune: the same with the
+ * column segments of every block-row of the result (pruned row segments count as zeros).  Each
+ * prunes the fraction p = 1 - sqrt(1 - prune_fraction), so about prune_fraction of the weights are
+ * gone after both (prune_fraction = 0.75 is the paper's "4x").  Where the paper is silent: the
+ * number pruned per block-column is floor(p * rows + 0.5) (per block-row floor(p * cols + 0.5));
+ * among equal norms the higher index is pruned first; norms are summed in fp64.
+ *   dense       device, float32, rows x cols, row stride ld (>= cols) elements; not modified.
+ *   row_keep    device, [nblk * block_r] bytes, written: 1 = kept, in csb_encode's layout (flags of
+ *               in-block lines beyond the matrix edge are 0).  col_keep likewise, [nblk * block_c].
+ *   workspace   device, csb_project_workspace_bytes(...) bytes of scratch, caller-owned.
+ * Asynchronous on `stream`; all pointers on the current device.  The pruned matrix itself is
+ * dense with the masked entries zeroed; csb_encode applies the masks.
+ * Errors: INVALID_ARG (null, sizes, blocks outside 1..256, fraction outside [0, 1], workspace
+ * too small), UNSUPPORTED (rows or cols above 20480), CUDA.
+ */
+int64_t csb_project_workspace_bytes(int64_t rows, int64_t cols, int block_r, int block_c);
+int csb_project(const float* dense, int64_t rows, int64_t cols, int64_t ld, int block_r, int block_c, double prune_fraction,
+                uint8_t* row_keep, uint8_t* col_keep, void* workspace, int64_t workspace_bytes, void* stream);
+
 /* Borrow the canonical arrays (host memory, valid until csb_free). */
 int csb_view(const csb_matrix_t* A, csb_view_t* out);
 

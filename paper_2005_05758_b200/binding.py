@@ -189,6 +189,29 @@ def csb_panel_dump(A: CsbMatrix, ctas: int, warps_per_cta: int, stage_bytes: int
             "panels": panels[: int(info[1])], "cta": cta[: int(info[0])]}
 
 
+def csb_project(W, block_r: int, block_c: int, prune_fraction: float, row_keep=None, col_keep=None, workspace=None,
+                stream=None):
+    """Keep masks of the projection of the device matrix W (torch, float32, 2-D) onto the CSB pattern;
+    returns (row_keep, col_keep, workspace) as torch uint8 tensors on W's device (allocated when not given)."""
+    import torch
+    lib.csb_project_workspace_bytes.argtypes = [C.c_int64, C.c_int64, C.c_int, C.c_int]
+    lib.csb_project_workspace_bytes.restype = C.c_int64
+    lib.csb_project.argtypes = [_P, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_double, _P, _P, _P, C.c_int64, _P]
+    lib.csb_project.restype = C.c_int
+    rows, cols = W.shape
+    nblk = -(-rows // block_r) * -(-cols // block_c) if block_r > 0 and block_c > 0 else 0
+    if row_keep is None:
+        row_keep = torch.empty(max(nblk * block_r, 1), dtype=torch.uint8, device=W.device)
+    if col_keep is None:
+        col_keep = torch.empty(max(nblk * block_c, 1), dtype=torch.uint8, device=W.device)
+    if workspace is None:
+        workspace = torch.empty(max(int(lib.csb_project_workspace_bytes(rows, cols, block_r, block_c)), 16), dtype=torch.uint8,
+                                device=W.device)
+    _check(lib.csb_project(_ptr(W), rows, cols, W.stride(0), block_r, block_c, float(prune_fraction), _ptr(row_keep),
+                           _ptr(col_keep), _ptr(workspace), workspace.numel(), _stream(stream)))
+    return row_keep, col_keep, workspace
+
+
 def csb_spmv(A: CsbMatrix, x, y, stream=None) -> None:
     _check(lib.csb_spmv(A.handle, _ptr(x), _ptr(y), _stream(stream)))
 
