@@ -218,10 +218,13 @@ int project_device(const float* W, int64_t R, int64_t C, int64_t ld, int BR, int
     double* rn = reinterpret_cast<double*>(workspace);
     double* cn = rn + nbc * R;
     const double p = 1.0 - std::sqrt(1.0 - PR);
-    static bool configured = false;
-    if (!configured) {
+    // the selection kernel's shared memory is opted in per device (setting it twice is harmless)
+    int dev = 0;
+    CSB_CUDA(cudaGetDevice(&dev));
+    static bool configured[64] = {};
+    if (dev >= 64 || !configured[dev]) {
         CSB_CUDA(cudaFuncSetAttribute(csb_select_prune_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kMaxSelect * 8 + 2048)));
-        configured = true;
+        if (dev < 64) configured[dev] = true;
     }
     // flags of in-block lines beyond the matrix edge stay zero
     CSB_CUDA(cudaMemsetAsync(row_keep, 0, (size_t)(nbr * nbc * BR), st));
