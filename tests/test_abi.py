@@ -24,3 +24,26 @@ def test_oracle_and_library_do_not_import_each_other():
                     src = open(os.path.join(dirpath, f)).read()
                     assert not re.search(r"^\s*(from|import)\s+" + banned, src, flags=re.M), (d, f)
                     assert ("#include \"../" + banned) not in src
+
+
+def test_project_argument_checks_need_no_gpu():
+    # csb_project validates sizes, fraction, workspace and the selection kernel's limit before it
+    # touches the device, so the refusals can be checked with made-up (never dereferenced) pointers
+    lib = ctypes.CDLL(os.path.join(ROOT, "paper_2005_05758_b200", "libcsb.so"))
+    lib.csb_project_workspace_bytes.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int]
+    lib.csb_project_workspace_bytes.restype = ctypes.c_int64
+    lib.csb_project.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                ctypes.c_double, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]
+    lib.csb_last_error.restype = ctypes.c_char_p
+    # 8 bytes per row segment and per column segment: (nbc * rows + nbr * cols) * 8
+    assert lib.csb_project_workspace_bytes(300, 1177, 32, 32) == (37 * 300 + 10 * 1177) * 8
+    assert lib.csb_project_workspace_bytes(0, 5, 2, 2) == 0
+    fake = ctypes.c_void_p(4096)
+    big = 1 << 40
+    assert lib.csb_project(None, 8, 8, 8, 4, 4, 0.5, fake, fake, fake, big, None) == -1
+    assert lib.csb_project(fake, 8, 8, 4, 4, 4, 0.5, fake, fake, fake, big, None) == -1          # ld < cols
+    assert lib.csb_project(fake, 8, 8, 8, 4, 300, 0.5, fake, fake, fake, big, None) == -1        # block size
+    assert lib.csb_project(fake, 8, 8, 8, 4, 4, 1.5, fake, fake, fake, big, None) == -1          # fraction
+    assert lib.csb_project(fake, 8, 8, 8, 4, 4, float("nan"), fake, fake, fake, big, None) == -1
+    assert lib.csb_project(fake, 8, 8, 8, 4, 4, 0.5, fake, fake, fake, 16, None) == -1 and b"workspace" in lib.csb_last_error()
+    assert lib.csb_project(fake, 30000, 64, 64, 32, 32, 0.5, fake, fake, fake, big, None) == -8 and b"20480" in lib.csb_last_error()
