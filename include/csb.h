@@ -240,6 +240,9 @@ int csb_lstm_forward(int n_layers, const csb_matrix_t* const* W, const float* co
  *   r = s(zx_r + zh_r + b_r);  z = s(zx_z + zh_z + b_z);
  *   n = tanh(zx_n + b_in + r * (zh_n + b_hn));  h_t = (1 - z) * n + z * h_{t-1},
  * where zx / zh are the parts of the product over the input / hidden columns.
+ * With B >= 8, fp16 values and block_r <= 64 the sequence runs step by step like the LSTM at
+ * B >= 16: one tensor-core product per layer and step over 2B rows (row b holds [u_t ; 0], row
+ * B + b holds [0 ; h_{t-1}], which keeps zx and zh apart) and one gate kernel.
  */
 int csb_gru_forward(int n_layers, const csb_matrix_t* const* W, const float* const* bias,
                     const float* x, int64_t T, int B, const float* h0, float* y, float* hT,

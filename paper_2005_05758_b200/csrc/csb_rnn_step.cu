@@ -1,4 +1,4 @@
-// LSTM layers at larger batch, one timestep at a time on tensor cores.
+// LSTM and GRU layers at larger batch, one timestep at a time on tensor cores.
 //
 // With a batch of 16 or more the per-step product of Section 2.1, W . [u_t ; h_{t-1}] for all
 // batch columns at once, is a dense contraction per block (kernel matrix times gathered inputs),
@@ -9,6 +9,10 @@
 // layer read one buffer V_l = [u_t ; h_{t-1}] of shape [B, I_l + H]; the gate kernel of layer l
 // writes h_t into the right part of V_l (for step t + 1) and into the left part of V_{l+1} (the
 // layer above, same step) or into y, and the gate kernel of layer 0 also moves x_{t+1} in.
+//
+// GRU (reset gate applied after the recurrent product) needs the input part and the recurrent part
+// of the candidate's pre-activation apart.  One product still does: V_l has 2B rows, row b holds
+// [u_t ; 0] and row B + b holds [0 ; h_{t-1}], so row b of the product is W_x u and row B + b is W_h h.
 #include <algorithm>
 #include <list>
 #include <memory>
@@ -29,10 +33,10 @@ namespace csb {
 
 struct StepPlan {
     std::vector<uint64_t> uids;
-    int L = 0, B = 0, H = 0, device = -1;
+    int L = 0, B = 0, H = 0, gates = 0, device = -1;
     int in_size[kMaxLayers] = {};
-    float* d_v[kMaxLayers] = {};       // [B, in_size[l] + H] per layer
-    float* d_z = nullptr;              // [B, 4H] pre-activations of the layer being worked on
+    float* d_v[kMaxLayers] = {};       // [B, in_size[l] + H] per layer (GRU: [2B, ...], input rows then recurrent rows)
+    float* d_z = nullptr;              // [B, 4H] (GRU: [2B, 3H]) pre-activations of the layer being worked on
     float* d_c = nullptr;              // [L, B, H] cell state
     float* d_stage = nullptr;          // host-I/O staging of x and y
     size_t stage_cap = 0;
@@ -90,42 +94,75 @@ __global__ void csb_lstm_gates_kernel(const float* __restrict__ Z, const float* 
     }
 }
 
+// Gate arithmetic of one GRU layer and step (reset after the recurrent product):
+//   r = s(zx_r + zh_r + b_r),  u = s(zx_z + zh_z + b_z),  n = tanh(zx_n + b_in + r (zh_n + b_hn)),
+//   h_t = (1 - u) n + u h_{t-1};  zx = row b, zh = row B + b of Z [2B, 3H]; bias = b_r, b_z, b_in, b_hn.
+// h_t goes to the recurrent rows of v_self (row B + b, columns off_self ..), to the input rows of
+// v_next (row b) when there is a layer above, and to y_t; x_next as for the LSTM kernel.
+__global__ void csb_gru_gates_kernel(const float* __restrict__ Z, const float* __restrict__ bias, float* __restrict__ v_self,
+                                     int ld_self, int off_self, float* __restrict__ v_next, int ld_next, float* __restrict__ y_t,
+                                     const float* __restrict__ x_next, int I, float* __restrict__ v0, int ld0, int B, int H) {
+    const int n = B * H;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
+        const int b = e / H, j = e - b * H;
+        const float* zx = Z + (size_t)b * 3 * H;
+        const float* zh = Z + (size_t)(B + b) * 3 * H;
+        float ar = zx[j] + zh[j], au = zx[H + j] + zh[H + j], nx = zx[2 * H + j], nh = zh[2 * H + j];
+        if (bias) { ar += bias[j]; au += bias[H + j]; nx += bias[2 * H + j]; nh += bias[3 * H + j]; }
+        const float r = logistic(ar), u = logistic(au);
+        const float cand = tanhf(nx + r * nh);
+        float* hp = v_self + (size_t)(B + b) * ld_self + off_self + j;
+        const float h = (1.f - u) * cand + u * *hp;
+        *hp = h;
+        if (v_next) v_next[(size_t)b * ld_next + j] = h;
+        if (y_t) y_t[e] = h;
+    }
+    if (x_next) {
+        const int nx = B * I;
+        for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < nx; e += gridDim.x * blockDim.x) {
+            const int b = e / I, i = e - b * I;
+            v0[(size_t)b * ld0 + i] = x_next[e];
+        }
+    }
+}
+
 static int env_flag(const char* name) {
     const char* v = getenv(name);
     return v && *v ? atoi(v) : 0;
 }
 
 bool rnn_stepwise_wanted(int gates, int L, const csb_matrix* const* W, int B) {
-    if (gates != 4 || B < 16 || env_flag("CSB_RNN_NO_STEPWISE")) return false;
+    if (env_flag("CSB_RNN_NO_STEPWISE")) return false;
+    if (!(gates == 4 && B >= 16) && !(gates == 3 && B >= 8)) return false;
     for (int l = 0; l < L; ++l)
-        if (!spmm_mma_applicable(W[l], B)) return false;
+        if (!spmm_mma_applicable(W[l], gates == 3 ? 2 * B : B)) return false;
     return true;
 }
 
 // Returns CSB_OK, an error, or 1 when the tensor-core plan of a layer does not fit (nothing the
 // caller can see has been written then; the caller runs the persistent kernel instead).
-int rnn_forward_stepwise(int L, const csb_matrix* const* W, const float* const* bias, const float* x, int64_t T, int B, int H,
+int rnn_forward_stepwise(int gates, int L, const csb_matrix* const* W, const float* const* bias, const float* x, int64_t T, int B, int H,
                          const int* in_size, const float* h0, const float* c0, float* y, float* hT, float* cT, unsigned flags,
                          void* stream) {
     StepPlan* P = nullptr;
     {
         std::lock_guard<std::mutex> lk(g_step_mu);
         for (auto& p : g_step_plans) {
-            if (p->L != L || p->B != B) continue;
+            if (p->L != L || p->B != B || p->gates != gates) continue;
             bool same = true;
             for (int l = 0; l < L; ++l) same = same && p->uids[l] == W[l]->uid;
             if (same) { P = p.get(); break; }
         }
         if (!P) {
             std::unique_ptr<StepPlan> np(new StepPlan());
-            np->L = L; np->B = B; np->H = H; np->device = W[0]->device;
+            np->L = L; np->B = B; np->H = H; np->gates = gates; np->device = W[0]->device;
             for (int l = 0; l < L; ++l) {
                 np->uids.push_back(W[l]->uid);
                 np->in_size[l] = in_size[l];
-                CSB_CUDA(cudaMalloc((void**)&np->d_v[l], (size_t)B * (in_size[l] + H) * 4));
+                CSB_CUDA(cudaMalloc((void**)&np->d_v[l], (size_t)(gates == 3 ? 2 : 1) * B * (in_size[l] + H) * 4));
             }
-            CSB_CUDA(cudaMalloc((void**)&np->d_z, (size_t)B * 4 * H * 4));
-            CSB_CUDA(cudaMalloc((void**)&np->d_c, (size_t)L * B * H * 4));
+            CSB_CUDA(cudaMalloc((void**)&np->d_z, (size_t)(gates == 3 ? 2 : 1) * B * gates * H * 4));
+            if (gates == 4) CSB_CUDA(cudaMalloc((void**)&np->d_c, (size_t)L * B * H * 4));
             P = np.get();
             g_step_plans.push_back(std::move(np));
         }
@@ -151,22 +188,29 @@ int rnn_forward_stepwise(int L, const csb_matrix* const* W, const float* const* 
     const cudaMemcpyKind in_kind = host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
     const cudaMemcpyKind out_kind = host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice;
     const size_t hrow = (size_t)H * 4;
-    // V_l = [u_0 ; h_{-1}]: h0 (or zeros) on the right, x_0 on the left of layer 0
+    const bool gru = gates == 3;
+    const int vrows = gru ? 2 * B : B;                  // rows of V_l and of the product
+    // V_l = [u_0 ; h_{-1}]: h0 (or zeros) on the right, x_0 on the left of layer 0.  GRU: the
+    // recurrent rows (B ..) carry h and zeros on the left, the input rows zeros on the right.
     for (int l = 0; l < L; ++l) {
         const int ld = in_size[l] + H;
-        if (h0) CSB_CUDA(cudaMemcpy2DAsync(P->d_v[l] + in_size[l], (size_t)ld * 4, h0 + (size_t)l * B * H, hrow, hrow, B, in_kind, st));
-        else CSB_CUDA(cudaMemset2DAsync(P->d_v[l] + in_size[l], (size_t)ld * 4, 0, hrow, B, st));
+        float* hpart = P->d_v[l] + (gru ? (size_t)B * ld : 0) + in_size[l];
+        if (gru) CSB_CUDA(cudaMemsetAsync(P->d_v[l], 0, (size_t)vrows * ld * 4, st));
+        if (h0) CSB_CUDA(cudaMemcpy2DAsync(hpart, (size_t)ld * 4, h0 + (size_t)l * B * H, hrow, hrow, B, in_kind, st));
+        else if (!gru) CSB_CUDA(cudaMemset2DAsync(hpart, (size_t)ld * 4, 0, hrow, B, st));
     }
     CSB_CUDA(cudaMemcpy2DAsync(P->d_v[0], (size_t)(I0 + H) * 4, dx, (size_t)I0 * 4, (size_t)I0 * 4, B, cudaMemcpyDeviceToDevice, st));
-    if (c0) CSB_CUDA(cudaMemcpyAsync(P->d_c, c0, ns * 4, in_kind, st));
-    else CSB_CUDA(cudaMemsetAsync(P->d_c, 0, ns * 4, st));
+    if (!gru) {
+        if (c0) CSB_CUDA(cudaMemcpyAsync(P->d_c, c0, ns * 4, in_kind, st));
+        else CSB_CUDA(cudaMemsetAsync(P->d_c, 0, ns * 4, st));
+    }
 
     const int threads = 256;
     const int blocks = std::max(1, std::min(1024, (B * std::max(H, I0) + threads - 1) / threads));
     for (int64_t t = 0; t < T; ++t) {
         for (int l = 0; l < L; ++l) {
             const int ld = in_size[l] + H;
-            const int rc = launch_spmm_mma(W[l], P->d_v[l], ld, B, P->d_z, 4 * (int64_t)H, stream);
+            const int rc = launch_spmm_mma(W[l], P->d_v[l], ld, vrows, P->d_z, (int64_t)gates * H, stream);
             if (rc != CSB_OK) {
                 // in step 0 only scratch has been written so far (y is written behind the top layer's product)
                 if (rc == 1 && t > 0) { set_error("the tensor-core plan of layer %d became unusable in mid-sequence", l); return CSB_ERR_CUDA; }
@@ -174,17 +218,24 @@ int rnn_forward_stepwise(int L, const csb_matrix* const* W, const float* const* 
             }
             const bool top = l == L - 1;
             const float* x_next = (l == 0 && t + 1 < T) ? dx + (size_t)(t + 1) * B * I0 : nullptr;
-            csb_lstm_gates_kernel<<<blocks, threads, 0, st>>>(P->d_z, bias ? bias[l] : nullptr, P->d_c + (size_t)l * B * H, P->d_v[l], ld,
-                                                             in_size[l], top ? nullptr : P->d_v[l + 1], top ? 0 : in_size[l + 1] + H,
-                                                             (top && dy) ? dy + (size_t)t * B * H : nullptr, x_next, I0, P->d_v[0],
-                                                             I0 + H, B, H);
+            if (gru)
+                csb_gru_gates_kernel<<<blocks, threads, 0, st>>>(P->d_z, bias ? bias[l] : nullptr, P->d_v[l], ld, in_size[l],
+                                                                top ? nullptr : P->d_v[l + 1], top ? 0 : in_size[l + 1] + H,
+                                                                (top && dy) ? dy + (size_t)t * B * H : nullptr, x_next, I0, P->d_v[0],
+                                                                I0 + H, B, H);
+            else
+                csb_lstm_gates_kernel<<<blocks, threads, 0, st>>>(P->d_z, bias ? bias[l] : nullptr, P->d_c + (size_t)l * B * H, P->d_v[l], ld,
+                                                                 in_size[l], top ? nullptr : P->d_v[l + 1], top ? 0 : in_size[l + 1] + H,
+                                                                 (top && dy) ? dy + (size_t)t * B * H : nullptr, x_next, I0, P->d_v[0],
+                                                                 I0 + H, B, H);
             CSB_CUDA(cudaGetLastError());
         }
     }
     if (hT)
         for (int l = 0; l < L; ++l)
-            CSB_CUDA(cudaMemcpy2DAsync(hT + (size_t)l * B * H, hrow, P->d_v[l] + in_size[l], (size_t)(in_size[l] + H) * 4, hrow, B, out_kind, st));
-    if (cT) CSB_CUDA(cudaMemcpyAsync(cT, P->d_c, ns * 4, out_kind, st));
+            CSB_CUDA(cudaMemcpy2DAsync(hT + (size_t)l * B * H, hrow, P->d_v[l] + (gru ? (size_t)B * (in_size[l] + H) : 0) + in_size[l],
+                                       (size_t)(in_size[l] + H) * 4, hrow, B, out_kind, st));
+    if (cT && !gru) CSB_CUDA(cudaMemcpyAsync(cT, P->d_c, ns * 4, out_kind, st));
     if (host_io && y) CSB_CUDA(cudaMemcpyAsync(y, dy, ny * 4, cudaMemcpyDeviceToHost, st));
     if (host_io || !(flags & CSB_FLAG_ASYNC)) {
         CSB_CUDA(cudaStreamSynchronize(st));

@@ -143,6 +143,26 @@ def test_lstm_large_batch_both_paths_agree(monkeypatch):
     assert np.max(np.abs(ya - yb)) < 1e-4
 
 
+@pytest.mark.parametrize("B,I,H,L,br,bc", [(8, 40, 48, 2, 16, 16), (20, 39, 100, 1, 32, 32), (33, 70, 192, 2, 64, 32)])
+def test_gru_batch_runs_step_by_step_on_tensor_cores(B, I, H, L, br, bc):
+    # GRU from batch 8: one product over 2B rows ([u ; 0] and [0 ; h]) keeps the candidate's two parts apart
+    w = workloads.make_rnn_workload(41, "gru", I, H, L, br, bc, "lognormal", rate=4.0, T=6, B=B, w_std=0.15,
+                                    bias_std=0.2, state_std=0.4)
+    y1, h1, _ = check(w)
+    y2, h2, _ = run(w, chunks=[(0, 2), (2, 6)])
+    assert np.array_equal(y1, y2) and np.array_equal(h1, h2)
+    y3, h3, _ = run(w, host_io=True)
+    assert np.array_equal(y1, y3) and np.array_equal(h1, h3)
+
+
+@pytest.mark.parametrize("cell,B", [("gru", 8), ("lstm", 16)])
+def test_persistent_kernel_still_serves_these_batches(monkeypatch, cell, B):
+    monkeypatch.setenv("CSB_RNN_NO_STEPWISE", "1")
+    w = workloads.make_rnn_workload(42, cell, 40, 48, 2, 16, 16, "uniform", lo=0.2, hi=0.9, T=7, B=B, w_std=0.2,
+                                    bias_std=0.1, state_std=0.5)
+    check(w)
+
+
 def test_cfg5_batch32_reduced_length():
     check(workloads.CONFIGS["cfg5"](T=3, B=32))
 
