@@ -386,7 +386,7 @@ def other_configs(binding, torch, dev, flush, quick):
         out["%s_B%d" % (name, w.B)] = {"us_per_timestep": round(us, 3), "T": w.T, "B": w.B,
                                        "algorithmic_bytes_per_step": rnn_alg_bytes_per_step(w, infos),
                                        "GFLOPs": round(2 * sum(i["nnz"] for i in infos) * w.B / us / 1e3, 1),
-                                       "path": "per-step launches, products on tensor cores" if ((w.cell == "lstm" and w.B >= 16) or (w.cell == "gru" and w.B >= 8))
+                                       "path": "per-step launches, products on tensor cores" if (w.B >= 16 or (w.B >= 8 and sum(i["nnz"] for i in infos) >= 100000))
                                                else "persistent time-loop kernel"}
         for m in mats:
             m.free()

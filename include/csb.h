@@ -222,7 +222,8 @@ int csb_spmv_static_scratch(const csb_matrix_t* A, const float* x, float* y, voi
  *            through device staging buffers on `stream` and waits for the result.
  * The first call for a given (W..., B) builds and caches the time-loop schedule and its
  * device state (allocates, synchronises); later calls reuse it.  T = 0 or B = 0 is a no-op.
- * With B >= 16, fp16 values and block_r <= 64 the sequence is not run by the persistent kernel
+ * With B >= 16 (B >= 8 when the layers hold 100000 weights or more), fp16 values and block_r <= 64
+ * the sequence is not run by the persistent kernel
  * but step by step: per layer and step the batched product on tensor cores (as csb_spmm, same
  * input-range rule) and one kernel with the gate arithmetic; same results within rounding, same
  * arguments and flags (CSB_RNN_NO_STEPWISE=1 in the environment keeps the persistent kernel).
@@ -240,8 +241,7 @@ int csb_lstm_forward(int n_layers, const csb_matrix_t* const* W, const float* co
  *   r = s(zx_r + zh_r + b_r);  z = s(zx_z + zh_z + b_z);
  *   n = tanh(zx_n + b_in + r * (zh_n + b_hn));  h_t = (1 - z) * n + z * h_{t-1},
  * where zx / zh are the parts of the product over the input / hidden columns.
- * With B >= 8, fp16 values and block_r <= 64 the sequence runs step by step like the LSTM at
- * B >= 16: one tensor-core product per layer and step over 2B rows (row b holds [u_t ; 0], row
+ * At the same batch sizes as for the LSTM (fp16 values, block_r <= 64) the sequence runs step by step: one tensor-core product per layer and step over 2B rows (row b holds [u_t ; 0], row
  * B + b holds [0 ; h_{t-1}], which keeps zx and zh apart) and one gate kernel.
  */
 int csb_gru_forward(int n_layers, const csb_matrix_t* const* W, const float* const* bias,

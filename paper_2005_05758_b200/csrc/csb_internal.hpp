@@ -283,7 +283,7 @@ int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, 
 // csb_rnn.cu
 void drop_rnn_plans(const csb_matrix* A);  // forget cached time-loop plans that use A
 
-// csb_rnn_step.cu -- LSTM at batch >= 16, GRU at batch >= 8: one timestep at a time, products on tensor cores
+// csb_rnn_step.cu -- batch >= 16 (>= 8 for big layers): one timestep at a time, products on tensor cores
 bool rnn_stepwise_wanted(int gates, int L, const csb_matrix* const* W, int B);
 int rnn_forward_stepwise(int gates, int L, const csb_matrix* const* W, const float* const* bias, const float* x, int64_t T, int B, int H,
                          const int* in_size, const float* h0, const float* c0, float* y, float* hT, float* cT, unsigned flags,

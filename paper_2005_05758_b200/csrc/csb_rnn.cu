@@ -809,7 +809,7 @@ static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const flo
     CSB_CUDA(cudaSetDevice(W[0]->device));
     struct Restore { int d; ~Restore() { cudaSetDevice(d); } } restore{prev};
 
-    // LSTM at batch >= 16, GRU at batch >= 8, fp16 values: step by step, the products on tensor cores
+    // larger batches with fp16 values: step by step, the products on tensor cores
     if (rnn_stepwise_wanted(gates, L, W, B)) {
         const int rc = rnn_forward_stepwise(gates, L, W, bias, x, T, B, H, in_size, h0, c0, y, hT, cT, flags, stream);
         if (rc != 1) return rc;

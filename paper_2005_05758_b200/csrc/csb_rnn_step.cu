@@ -133,7 +133,11 @@ static int env_flag(const char* name) {
 
 bool rnn_stepwise_wanted(int gates, int L, const csb_matrix* const* W, int B) {
     if (env_flag("CSB_RNN_NO_STEPWISE")) return false;
-    if (!(gates == 4 && B >= 16) && !(gates == 3 && B >= 8)) return false;
+    // from batch 16 always; from batch 8 when the layers are big enough for three launches per layer
+    // and step to pay (measured: 591 k weights 24 -> 17 us per step, 25 k weights 9 -> 13)
+    int64_t nnz = 0;
+    for (int l = 0; l < L; ++l) nnz += W[l]->nnz;
+    if (!(B >= 16 || (B >= 8 && nnz >= 100000))) return false;
     for (int l = 0; l < L; ++l)
         if (!spmm_mma_applicable(W[l], gates == 3 ? 2 * B : B)) return false;
     return true;

@@ -121,7 +121,7 @@ def test_resume_equals_one_call_bitwise_and_host_io():
     assert np.array_equal(y1, y3) and np.array_equal(h1, h3) and np.array_equal(c1, c3)
 
 
-@pytest.mark.parametrize("B,I,H,L,br,bc", [(16, 40, 48, 2, 16, 16), (32, 153, 160, 1, 32, 32), (40, 70, 192, 2, 64, 32)])
+@pytest.mark.parametrize("B,I,H,L,br,bc", [(16, 40, 48, 2, 16, 16), (32, 153, 160, 1, 32, 32), (40, 70, 192, 2, 64, 32), (8, 200, 512, 1, 32, 32)])
 def test_lstm_large_batch_runs_step_by_step_on_tensor_cores(B, I, H, L, br, bc):
     # batches of 16 and more take the path of one product (tensor cores) + one gate kernel per layer
     # and step; bias, initial states, resumption and host I/O as for the persistent kernel
@@ -143,9 +143,9 @@ def test_lstm_large_batch_both_paths_agree(monkeypatch):
     assert np.max(np.abs(ya - yb)) < 1e-4
 
 
-@pytest.mark.parametrize("B,I,H,L,br,bc", [(8, 40, 48, 2, 16, 16), (20, 39, 100, 1, 32, 32), (33, 70, 192, 2, 64, 32)])
+@pytest.mark.parametrize("B,I,H,L,br,bc", [(16, 40, 48, 2, 16, 16), (20, 39, 100, 1, 32, 32), (33, 70, 192, 2, 64, 32), (8, 300, 512, 1, 32, 32)])
 def test_gru_batch_runs_step_by_step_on_tensor_cores(B, I, H, L, br, bc):
-    # GRU from batch 8: one product over 2B rows ([u ; 0] and [0 ; h]) keeps the candidate's two parts apart
+    # GRU from batch 16 (from batch 8 for layers of 100 k weights and more): one product over 2B rows ([u ; 0] and [0 ; h]) keeps the candidate's two parts apart
     w = workloads.make_rnn_workload(41, "gru", I, H, L, br, bc, "lognormal", rate=4.0, T=6, B=B, w_std=0.15,
                                     bias_std=0.2, state_std=0.4)
     y1, h1, _ = check(w)
