@@ -171,7 +171,9 @@ int csb_spmv(const csb_matrix_t* A, const float* x, float* y, void* stream);
  * columns are split into two binary16 halves (x = hi + lo, so no input precision is lost as long
  * as |x| < 65504) and multiplied with mma.sync, fp32 accumulation.  The first such call on a
  * handle builds a second device layout and a staging buffer for it (allocates and synchronises
- * the device once; make it outside of any stream capture).  Other cases use the CUDA-core kernel
+ * the device once; make it outside of any stream capture).  The two kernels of this path are
+ * launched with programmatic stream serialization and wait, first thing, for the work in front of
+ * them on `stream`.  Other cases use the CUDA-core kernel
  * in batch tiles of 8 / 4 / 1.
  */
 int csb_spmm(const csb_matrix_t* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy,

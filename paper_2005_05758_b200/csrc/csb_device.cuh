@@ -58,6 +58,13 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 // accesses it issues next.
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
+// Programmatic dependent launch.  A kernel launched with programmatic stream serialization may be
+// scheduled while the kernel in front of it on the stream is still draining; pdl_wait() blocks until
+// that kernel has completed and its writes are visible (at once for an ordinary launch), and
+// pdl_launch_dependents() tells the hardware that whatever comes next may be scheduled.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 template <typename T> struct WordTraits;
 template <> struct WordTraits<__half> {
     static constexpr int kRows = 2;

@@ -19,6 +19,7 @@
 #include <mutex>
 
 #include "csb_internal.hpp"
+#include "csb_device.cuh"
 
 namespace csb {
 
@@ -72,6 +73,8 @@ __global__ void csb_lstm_gates_kernel(const float* __restrict__ Z, const float* 
                                       float* __restrict__ v_self, int ld_self, int off_self, float* __restrict__ v_next,
                                       int ld_next, float* __restrict__ y_t, const float* __restrict__ x_next, int I,
                                       float* __restrict__ v0, int ld0, int B, int H) {
+    pdl_launch_dependents();
+    pdl_wait();                                    // Z comes from the product in front
     const int n = B * H;
     for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
         const int b = e / H, j = e - b * H;
@@ -102,6 +105,8 @@ __global__ void csb_lstm_gates_kernel(const float* __restrict__ Z, const float* 
 __global__ void csb_gru_gates_kernel(const float* __restrict__ Z, const float* __restrict__ bias, float* __restrict__ v_self,
                                      int ld_self, int off_self, float* __restrict__ v_next, int ld_next, float* __restrict__ y_t,
                                      const float* __restrict__ x_next, int I, float* __restrict__ v0, int ld0, int B, int H) {
+    pdl_launch_dependents();
+    pdl_wait();                                    // Z comes from the product in front
     const int n = B * H;
     for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
         const int b = e / H, j = e - b * H;
@@ -222,16 +227,22 @@ int rnn_forward_stepwise(int gates, int L, const csb_matrix* const* W, const flo
             }
             const bool top = l == L - 1;
             const float* x_next = (l == 0 && t + 1 < T) ? dx + (size_t)(t + 1) * B * I0 : nullptr;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3((unsigned)blocks); cfg.blockDim = dim3((unsigned)threads); cfg.dynamicSmemBytes = 0;
+            cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 1;
+            const float* bl = bias ? bias[l] : nullptr;
+            float* vn = top ? nullptr : P->d_v[l + 1];
+            const int ldn = top ? 0 : in_size[l + 1] + H;
+            float* yt = (top && dy) ? dy + (size_t)t * B * H : nullptr;
             if (gru)
-                csb_gru_gates_kernel<<<blocks, threads, 0, st>>>(P->d_z, bias ? bias[l] : nullptr, P->d_v[l], ld, in_size[l],
-                                                                top ? nullptr : P->d_v[l + 1], top ? 0 : in_size[l + 1] + H,
-                                                                (top && dy) ? dy + (size_t)t * B * H : nullptr, x_next, I0, P->d_v[0],
-                                                                I0 + H, B, H);
+                CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_gru_gates_kernel, (const float*)P->d_z, bl, P->d_v[l], ld, in_size[l], vn, ldn, yt,
+                                            x_next, I0, P->d_v[0], I0 + H, B, H));
             else
-                csb_lstm_gates_kernel<<<blocks, threads, 0, st>>>(P->d_z, bias ? bias[l] : nullptr, P->d_c + (size_t)l * B * H, P->d_v[l], ld,
-                                                                 in_size[l], top ? nullptr : P->d_v[l + 1], top ? 0 : in_size[l + 1] + H,
-                                                                 (top && dy) ? dy + (size_t)t * B * H : nullptr, x_next, I0, P->d_v[0],
-                                                                 I0 + H, B, H);
+                CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_lstm_gates_kernel, (const float*)P->d_z, bl, P->d_c + (size_t)l * B * H, P->d_v[l], ld,
+                                            in_size[l], vn, ldn, yt, x_next, I0, P->d_v[0], I0 + H, B, H));
             CSB_CUDA(cudaGetLastError());
         }
     }

@@ -50,6 +50,8 @@ struct MmaSmem {
 
 // Pack a slab of X: fp32 [batch][cols] -> fp16 hi / lo [cols][64] (batch columns past nb are zero).
 __global__ void csb_pack_x_kernel(const float* __restrict__ X, long long ldx, int nb, int cols, __half* __restrict__ xp) {
+    pdl_launch_dependents();
+    pdl_wait();                                    // X may come from the kernel in front; xp may still be read by it
     const int col = blockIdx.x * (blockDim.x / kSlab) + threadIdx.x / kSlab, b = threadIdx.x % kSlab;
     if (col >= cols) return;
     const float x = b < nb ? X[(long long)b * ldx + col] : 0.f;
@@ -70,6 +72,8 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
 
 template <int NT>
 __global__ void __launch_bounds__(256, 1) csb_spmm_mma_kernel(const MmaArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();                                    // the packed inputs come from the kernel in front
     extern __shared__ __align__(128) uint8_t smem[];
     const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const MmaSmem L(W, a.stages, a.stage_bytes, a.block_r);
@@ -326,10 +330,19 @@ int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch,
     for (int b0 = 0; b0 < batch; b0 += kSlab) {
         a.nb = std::min(kSlab, batch - b0);
         a.Y = Y + (int64_t)b0 * ldy;
-        csb_pack_x_kernel<<<(unsigned)((A->cols + 7) / 8), 256, 0, st>>>(X + (int64_t)b0 * ldx, ldx, a.nb, (int)A->cols, (__half*)P.d_xp);
-        if (a.nb <= 8) csb_spmm_mma_kernel<1><<<P.ctas, P.warps * 32, L.total, st>>>(a);
-        else if (a.nb <= 16) csb_spmm_mma_kernel<2><<<P.ctas, P.warps * 32, L.total, st>>>(a);
-        else csb_spmm_mma_kernel<4><<<P.ctas, P.warps * 32, L.total, st>>>(a);
+        // both kernels order themselves behind the work in front (pdl_wait at their top), so they may
+        // be launched with programmatic stream serialization: their scheduling overlaps its tail
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg{};
+        cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 1;
+        cfg.gridDim = dim3((unsigned)((A->cols + 7) / 8)); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0;
+        CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_pack_x_kernel, X + (int64_t)b0 * ldx, (long long)ldx, a.nb, (int)A->cols, (__half*)P.d_xp));
+        cfg.gridDim = dim3((unsigned)P.ctas); cfg.blockDim = dim3((unsigned)P.warps * 32u); cfg.dynamicSmemBytes = L.total;
+        if (a.nb <= 8) CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_spmm_mma_kernel<1>, a));
+        else if (a.nb <= 16) CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_spmm_mma_kernel<2>, a));
+        else CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_spmm_mma_kernel<4>, a));
         CSB_CUDA(cudaGetLastError());
     }
     return CSB_OK;
