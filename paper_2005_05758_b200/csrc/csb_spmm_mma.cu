@@ -73,7 +73,6 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
 template <int NT>
 __global__ void __launch_bounds__(256, 1) csb_spmm_mma_kernel(const MmaArgs a) {
     pdl_launch_dependents();
-    pdl_wait();                                    // the packed inputs come from the kernel in front
     extern __shared__ __align__(128) uint8_t smem[];
     const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const MmaSmem L(W, a.stages, a.stage_bytes, a.block_r);
@@ -103,6 +102,9 @@ __global__ void __launch_bounds__(256, 1) csb_spmm_mma_kernel(const MmaArgs a) {
     }
     for (int i = lane; i < a.block_r * kZStride; i += 32) zs[i] = 0.f;
     __syncwarp();
+    // everything so far touched only the planned stream (written once, at plan time) and shared
+    // memory; the packed inputs and Y belong to the work in front on the stream
+    pdl_wait();
 
     bool dead = false, reported = false;
     Chunk cur = Chunk{wd.z, wd.w};
