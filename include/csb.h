@@ -52,12 +52,16 @@ enum { CSB_FLAG_ASYNC = 1u,                 /* recurrent calls: do not wait for 
 
 typedef struct csb_matrix csb_matrix_t;     /* opaque: canonical arrays + device layout + schedule */
 
-/* Tuning knobs of the one-shot planning step; zero means "library default". */
+/* Tuning knobs of the one-shot planning step of the CUDA-core product kernel; zero means
+ * "library default".  Values outside the stated ranges make csb_encode fail with
+ * CSB_ERR_INVALID_ARG; so does a ring (warps x stages x stage_bytes) that cannot fit one CTA's
+ * shared memory even after the planner has reduced the warps per CTA. */
 typedef struct csb_plan_opts {
-    int ctas;            /* persistent grid size of the product kernels (default: SM count) */
-    int warps_per_cta;   /* warps per CTA (default 16)                                       */
-    int stage_bytes;     /* bytes per shared-memory ring stage of one warp (default 3072)    */
-    int stages;          /* ring depth per warp (default 3)                                  */
+    int ctas;            /* persistent grid size, >= 0 (default: SM count)                        */
+    int warps_per_cta;   /* warps per CTA, 0..16 (default 16)                                     */
+    int stage_bytes;     /* bytes per shared-memory ring stage of one warp, 1024..16384, rounded  */
+                         /* up to a multiple of 16 (default 4096)                                 */
+    int stages;          /* ring depth per warp, 1..8 (default 2)                                 */
 } csb_plan_opts;
 
 /* The canonical CSB arrays of Section 3.1.1 (n{}, m{}, RowIdx{}, ColIdx{}, Val{}) plus
@@ -162,7 +166,8 @@ void csb_free(csb_matrix_t* A);
 int csb_spmv(const csb_matrix_t* A, const float* x, float* y, void* stream);
 
 /*
- * csb_spmm -- Y[b, :] = A . X[b, :] for b < batch (the same product with a batch of vectors).
+ * csb_spmm -- Y[b, :] = A . X[b, :] for b < batch: the CSB matrix-vector product of Sections 4.2 and
+ * 4.3.1 (gather through ColIdx, kernel matrix, accumulate through RowIdx) with a batch of vectors.
  *   X  device, float32, batch rows of `cols` values, row stride ldx >= cols;
  *   Y  device, float32, batch rows of `rows` values, row stride ldy >= rows, overwritten.
  * batch = 0 is a no-op.  Same ordering / overlap rules as csb_spmv; results are bit-reproducible.
@@ -224,6 +229,11 @@ int csb_spmv_static_scratch(const csb_matrix_t* A, const float* x, float* y, voi
  *            through device staging buffers on `stream` and waits for the result.
  * The first call for a given (W..., B) builds and caches the time-loop schedule and its
  * device state (allocates, synchronises); later calls reuse it.  T = 0 or B = 0 is a no-op.
+ * That cached state (the ring of h slots, the barrier and status words, staging buffers) is one
+ * per (W..., B), not one per stream: two recurrent calls on the same matrices and batch size must
+ * not overlap on the GPU.  Calls queued on one stream are safe; calls on different streams need an
+ * event (or a synchronisation) between them, and then give identical bits.  The handles
+ * themselves are immutable and may be used from any stream.
  * With B >= 16 (B >= 8 when the layers hold 100000 weights or more), fp16 values and block_r <= 64
  * the sequence is not run by the persistent kernel
  * but step by step: per layer and step the batched product on tensor cores (as csb_spmm, same
@@ -238,12 +248,15 @@ int csb_lstm_forward(int n_layers, const csb_matrix_t* const* W, const float* co
                      float* y, float* hT, float* cT, unsigned flags, void* stream);
 
 /*
- * csb_gru_forward -- same for GRU layers.  W[l] is [3*H, I_l + H], rows r, z, n; bias[l] is
+ * csb_gru_forward -- a stack of GRU layers over a whole sequence (the GRU cell of Section 2.1: one
+ * CSB product per layer and step, gate arithmetic fused behind it); arguments, flags, caching and
+ * the no-overlap rule as for csb_lstm_forward.  W[l] is [3*H, I_l + H], rows r, z, n; bias[l] is
  * device float32 [4*H] = b_r, b_z, b_in, b_hn.  The reset gate acts after the recurrent product:
  *   r = s(zx_r + zh_r + b_r);  z = s(zx_z + zh_z + b_z);
  *   n = tanh(zx_n + b_in + r * (zh_n + b_hn));  h_t = (1 - z) * n + z * h_{t-1},
  * where zx / zh are the parts of the product over the input / hidden columns.
- * At the same batch sizes as for the LSTM (fp16 values, block_r <= 64) the sequence runs step by step: one tensor-core product per layer and step over 2B rows (row b holds [u_t ; 0], row
+ * At the same batch sizes as for the LSTM (fp16 values, block_r <= 64) the sequence runs step by
+ * step: one tensor-core product per layer and step over 2B rows (row b holds [u_t ; 0], row
  * B + b holds [0 ; h_{t-1}], which keeps zx and zh apart) and one gate kernel.
  */
 int csb_gru_forward(int n_layers, const csb_matrix_t* const* W, const float* const* bias,

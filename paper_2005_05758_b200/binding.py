@@ -12,7 +12,8 @@ from typing import Optional, Sequence
 
 import numpy as np
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcsb.so")
+# CSB_LIBRARY names another build of the same sources (an instrumented one, see build.py)
+_LIB_PATH = os.environ.get("CSB_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcsb.so")
 if not os.path.exists(_LIB_PATH):
     raise ImportError("libcsb.so is not built: run `python -m paper_2005_05758_b200.build` "
                       "(there is no CPU fallback)")

@@ -20,13 +20,24 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps if os.path.exists(d))
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the library if it is missing or older than its sources; return its path."""
-    if not force and not _stale():
+#: Instrumented variants (never the default build).  CSB_PHASE_CLOCKS makes the time-loop kernel sum
+#: clock64() cycles per phase and CTA (read back with csb_debug_rnn_clocks); CSB_PANEL_CLOCKS makes
+#: the SpMV panel kernel record wall-clock stamps per phase and CTA (csb_debug_panel_clocks).
+#: paper_2005_05758_b200/phase_clocks.py builds such a library beside the normal one and prints the figures.
+INSTRUMENT_DEFINES = ("CSB_PHASE_CLOCKS", "CSB_PANEL_CLOCKS")
+
+
+def build(force: bool = False, verbose: bool = False, defines=(), out: str = None) -> str:
+    """Compile the library if it is missing or older than its sources; return its path.
+    `defines` adds -D switches (see INSTRUMENT_DEFINES) and then needs `out`, the path of the
+    instrumented library, so that the normal libcsb.so is never replaced by one."""
+    if defines and not out:
+        raise ValueError("an instrumented build needs its own output path")
+    if not defines and not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-Xcompiler", "-fPIC", "-shared", "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
+           "-Xcompiler", "-fPIC", "-shared", "-o", out or LIB] + ["-D" + d for d in defines] + [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
@@ -35,7 +46,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
     if verbose:
         sys.stderr.write(res.stderr)
-    return LIB
+    return out or LIB
 
 
 if __name__ == "__main__":

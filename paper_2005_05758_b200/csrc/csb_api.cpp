@@ -55,6 +55,12 @@ int csb_encode(const float* dense, int64_t rows, int64_t cols, int64_t ld, int b
     if (block_r < 1 || block_r > 256 || block_c < 1 || block_c > 256) { set_error("block sizes must be 1..256, got %dx%d", block_r, block_c); return CSB_ERR_INVALID_ARG; }
     if (val_dtype != CSB_F32 && val_dtype != CSB_F16) { set_error("val_dtype %d", val_dtype); return CSB_ERR_DTYPE; }
     if (device < -1) { set_error("device %d", device); return CSB_ERR_INVALID_ARG; }
+    if (opts && (opts->ctas < 0 || opts->warps_per_cta < 0 || opts->warps_per_cta > 16 || opts->stages < 0 || opts->stages > 8 ||
+                 (opts->stage_bytes != 0 && (opts->stage_bytes < 1024 || opts->stage_bytes > 16384)))) {
+        set_error("csb_plan_opts out of range: ctas %d (>= 0), warps_per_cta %d (0..16), stage_bytes %d (0 or 1024..16384), stages %d (0..8)",
+                  opts->ctas, opts->warps_per_cta, opts->stage_bytes, opts->stages);
+        return CSB_ERR_INVALID_ARG;
+    }
     csb_matrix* A = new (std::nothrow) csb_matrix();
     if (!A) { set_error("out of host memory"); return CSB_ERR_ALLOC; }
     A->device = device;

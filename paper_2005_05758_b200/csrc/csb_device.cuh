@@ -83,11 +83,6 @@ template <> struct WordTraits<float> {
 __host__ __device__ constexpr int group_pad(int gw) { return gw == 32 ? 0 : gw; }
 __host__ __device__ constexpr int xg_stride(int gw, int bt) { return kMaxNk * bt + group_pad(gw); }
 
-#ifdef CSB_WALK_CLOCKS
-// instrumented build only: per-thread lap counters of walk_chunk (header, gather, multiply, fold, scatter, rounds)
-static __device__ long long csb_walk_prof_dummy;
-#define csb_walk_prof csb_walk_prof_local
-#endif
 
 template <int N> struct Log2;
 template <> struct Log2<8> { static constexpr int v = 3; };
@@ -117,11 +112,7 @@ __device__ __forceinline__ uint32_t chunk_bytes(const uint4& ch) {
 //   xg_w: per warp, G * xg_stride(GW, BT) floats;  zs_w: per warp, G * zs_stride floats.
 template <typename T, int BT, int GW, typename Gather>
 __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch, int lane, float* __restrict__ xg_w,
-                                           float* __restrict__ zs_w, int zs_stride, Gather gather4
-#ifdef CSB_WALK_CLOCKS
-                                           , long long* csb_walk_prof_local = &csb_walk_prof_dummy
-#endif
-                                           ) {
+                                           float* __restrict__ zs_w, int zs_stride, Gather gather4) {
     constexpr int R = WordTraits<T>::kRows;
     const int g = lane / GW, gl = lane % GW;
     const uint32_t sz[4] = {ch.x & 0xffffu, ch.x >> 16, ch.y & 0xffffu, ch.y >> 16};
@@ -135,12 +126,6 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
     const uint8_t* end = p + 16 * mine;
     float* xg = xg_w + g * xg_stride(GW, BT);
     float* zs = zs_w + g * zs_stride;
-#ifdef CSB_WALK_CLOCKS
-    long long tq = clock64();
-#define CSB_WALK_LAP(i) do { const long long n_ = clock64(); csb_walk_prof[i] += n_ - tq; tq = n_; } while (0)
-#else
-#define CSB_WALK_LAP(i) do { } while (0)
-#endif
     // The header and the column indices of an item are fetched one item ahead: both sit at fixed
     // places, so the loads go out together with the rest of the previous item's loads.  A lane
     // whose four indices lie past nk reads whatever follows (still inside the CTA's shared
@@ -171,7 +156,6 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
         }
         uint32_t rr = 0u;                                                 // this lane's R row indices, one byte each
         if (gl < RL) rr = (R == 2) ? (uint32_t)*reinterpret_cast<const uint16_t*>(ridx + 2 * gl) : (uint32_t)ridx[gl];
-        CSB_WALK_LAP(0);
 
         // ---- gather: each lane resolves four column indices at a time; indices past nk are
         // padding zeros, gather4 decides whether they may be dereferenced
@@ -180,7 +164,6 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
             for (int k4 = (gl + GW) * 4; k4 < nk; k4 += 4 * GW)
                 gather4(xbase, *reinterpret_cast<const uint32_t*>(item + 16 + k4), flags, nk - k4, xg + k4 * BT);
         __syncwarp();
-        CSB_WALK_LAP(1);
 
         // ---- multiply: lane gl reads words gl, gl + A, ... and walks columns kg, kg + S, ...
         const int kg = (int)(((uint32_t)gl * magic) >> 10);
@@ -236,7 +219,6 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
                 }
             }
         }
-        CSB_WALK_LAP(2);
 
         // ---- fold the sub-groups onto sub-group 0: a tree over kg (S need not be a power of
         // two); the number of rounds is the same for the whole warp
@@ -252,7 +234,6 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
                     if (take) acc[q][bt] += o;
                 }
         }
-        CSB_WALK_LAP(3);
 
         // ---- scatter-add through the row indices (distinct within an item: loads first, stores last)
         if (gl < RL) {
@@ -276,10 +257,6 @@ __device__ __forceinline__ void walk_chunk(const uint8_t* chunk, const uint4& ch
         h = hn;
         c4 = c4n;
         __syncwarp();
-        CSB_WALK_LAP(4);
-#ifdef CSB_WALK_CLOCKS
-        csb_walk_prof[5] += 1;
-#endif
     }
 }
 

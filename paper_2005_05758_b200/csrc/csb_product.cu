@@ -28,18 +28,8 @@ struct ProductArgs {
     long long ldx, ldy;
     uint32_t* status;
     int n_warps, nb, rows, cols, block_r, stage_bytes, stages, x_in_smem;
-#ifdef CSB_PHASE_CLOCKS
-    long long* clocks;         // [n_warps][6] cycle stamps: start, staged, first chunk, walked, flushed, end
-#endif
 };
 
-#ifdef CSB_PHASE_CLOCKS
-#define CSB_STAMP(i) do { if (lane == 0 && gw < a.n_warps) a.clocks[(size_t)gw * 6 + (i)] = clock64(); } while (0)
-#define CSB_ADD(i, v) do { if (lane == 0 && gw < a.n_warps) a.clocks[(size_t)gw * 6 + (i)] += (v); } while (0)
-#else
-#define CSB_STAMP(i) do { } while (0)
-#define CSB_ADD(i, v) do { } while (0)
-#endif
 
 constexpr uint32_t kOffMask = 0x3fffffffu;   // Chunk::off16 without the flush kind in its top two bits
 
@@ -183,10 +173,6 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
     const float* xs = reinterpret_cast<const float*>(smem + L.xs);
 
     const int gw = blockIdx.x * W + warp;
-    CSB_STAMP(0);
-#ifdef CSB_PHASE_CLOCKS
-    if (lane == 0 && gw < a.n_warps) { a.clocks[(size_t)gw * 6 + 2] = 0; a.clocks[(size_t)gw * 6 + 3] = 0; a.clocks[(size_t)gw * 6 + 4] = 0; }
-#endif
     // One 16-byte descriptor per warp (first chunk index, end chunk index, first chunk's place
     // and size) starts the pipeline with a single round trip; the loads of x are issued before
     // anything waits on it.
@@ -229,17 +215,10 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
         __syncwarp();
     }
 
-    CSB_STAMP(1);
-#if defined(CSB_PHASE_CLOCKS) || defined(CSB_WALK_CLOCKS)
-    long long wprof[6] = {0, 0, 0, 0, 0, 0};
-#endif
     bool dead = x_dead;
     bool reported = false;
     Chunk cur = Chunk{wd.z, wd.w};
     for (uint32_t c = c0; c < c1; ++c) {
-#ifdef CSB_PHASE_CLOCKS
-        const long long tc0 = clock64();
-#endif
         const int s = (int)((c - c0) % (uint32_t)a.stages);
         const uint32_t parity = ((c - c0) / (uint32_t)a.stages) & 1u;
         const uint32_t flush = cur.off16 >> 30;                       // known without the chunk itself
@@ -262,10 +241,6 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
             cur = nxt;
             continue;
         }
-#ifdef CSB_PHASE_CLOCKS
-        const long long tc1 = clock64();
-        CSB_ADD(2, tc1 - tc0);
-#endif
         const uint8_t* p = ring + (size_t)s * a.stage_bytes;
         const uint4 ch = *reinterpret_cast<const uint4*>(p);
         walk_chunk<T, BT, GW>(p, ch, lane, xg, zs, L.zs_stride,
@@ -290,14 +265,7 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
                 }
             }
         }
-#ifdef CSB_WALK_CLOCKS
-        , wprof
-#endif
         );
-#ifdef CSB_PHASE_CLOCKS
-        const long long tc2 = clock64();
-        CSB_ADD(3, tc2 - tc1);
-#endif
         if (flush == kFlushCta) {
             // the CTA owns this block-row: every warp is here with its last chunk of it
             // (three barriers whether the block-row is whole or a piece, so that a warp that gave
@@ -324,19 +292,12 @@ __global__ void __launch_bounds__(512, 1) csb_product_kernel(const ProductArgs a
             flush_block_row<BT, G>(a, zs, L.zs_stride, ch.z, ch.w, lane);
             __syncwarp();
         }
-#ifdef CSB_PHASE_CLOCKS
-        CSB_ADD(4, clock64() - tc2);
-#endif
         if (lane == 0 && refill.bytes) {
             mbar_expect_tx(&bars[s], refill.bytes);
             bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)(refill.off16 & kOffMask) * 16, refill.bytes, &bars[s]);
         }
         cur = nxt;
     }
-    CSB_STAMP(5);
-#ifdef CSB_PHASE_CLOCKS
-    if (lane == 0 && gw < a.n_warps) for (int i = 0; i < 6; ++i) a.clocks[(size_t)(a.n_warps + gw) * 6 + i] = wprof[i];
-#endif
 }
 
 #define CSB_CUDA(call)                                                                     \
@@ -389,15 +350,29 @@ int plan_product(csb_matrix* A) {
     // small matrices: no more warps than there is work for (about 2 KB of stream each)
     const int64_t approx = A->nnz * val_size(A->val_dtype) + (int64_t)A->ridx_off[A->nblk] + A->cidx_off[A->nblk] + 16 * A->nblk;
     const int64_t useful = std::max<int64_t>(1, approx / 2048);
+    // A row-owned plan fixes the CTA shape (its warps meet at CTA barriers), so that shape must fit
+    // shared memory at the narrowest batch tile; if the rings asked for do not, plan for fewer warps.
     ProductHostPlan H;
-    int rc = plan_product_host(A, ctas, wpc, useful, P.stage_bytes, &H);
-    if (rc != CSB_OK) return rc;
+    int rc = CSB_OK;
+    for (int w_try = wpc;; w_try /= 2) {
+        H = ProductHostPlan();
+        rc = plan_product_host(A, ctas, w_try, useful, P.stage_bytes, &H);
+        if (rc != CSB_OK) return rc;
+        P.row_owned = H.row_owned;
+        P.group_width = H.stream.group_width;
+        P.warps = H.row_owned ? H.warps_per_cta : 1;
+        size_t smem = 0;
+        if (fit_warps(A, P.warps, 1, 0, &smem) == P.warps) break;
+        if (w_try <= 1 || !H.row_owned) {
+            set_error("a shared-memory ring of %d stages of %d bytes per warp does not fit one CTA (%zu bytes available)", P.stages,
+                      P.stage_bytes, A->smem_optin);
+            return CSB_ERR_INVALID_ARG;
+        }
+    }
     const int n_warps = H.stream.n_warps;
-    P.row_owned = H.row_owned;
     if (H.row_owned) { P.warps = H.warps_per_cta; P.ctas = H.ctas; }
     else { P.warps = std::max(1, (n_warps + ctas - 1) / ctas); P.ctas = (n_warps + P.warps - 1) / P.warps; }
     P.n_slots = H.n_slots;
-    P.group_width = H.stream.group_width;
     P.balance = H.balance;
     P.stream_bytes = (int64_t)H.stream.bytes.size();
     P.n_warps = n_warps;
@@ -475,12 +450,6 @@ static int dispatch_tile(const csb_matrix* A, const ProductArgs& a, cudaStream_t
     return h ? dispatch_gw<__half, 1>(A, a, st) : dispatch_gw<float, 1>(A, a, st);
 }
 
-#ifdef CSB_PHASE_CLOCKS
-long long* g_phase_clocks = nullptr;
-extern "C" int csb_debug_phase_clocks(long long* host_out, int n_warps) {
-    return (int)cudaMemcpy(host_out, g_phase_clocks, (size_t)n_warps * 6 * 8, cudaMemcpyDeviceToHost);
-}
-#endif
 
 int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream) {
     const ProductPlan& P = A->product;
@@ -493,12 +462,6 @@ int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, 
     a.part_base = P.d_part_base; a.part_count = P.d_part_count; a.arrivals = P.d_arrivals; a.partials = P.d_partials;
     a.ldx = ldx; a.ldy = ldy; a.status = P.d_status; a.n_warps = P.n_warps;
     a.rows = (int)A->rows; a.cols = (int)A->cols; a.block_r = A->block_r; a.stage_bytes = P.stage_bytes; a.stages = P.stages;
-#ifdef CSB_PHASE_CLOCKS
-    static long long* d_clocks = nullptr;
-    if (!d_clocks) cudaMalloc((void**)&d_clocks, (size_t)1 << 22);
-    a.clocks = d_clocks;
-    g_phase_clocks = d_clocks;
-#endif
     cudaStream_t st = (cudaStream_t)stream;
     int rc = CSB_OK;
     int widest = kMaxBatchTile;                        // narrowed when a tile's shared memory does not fit the planned CTA
@@ -508,7 +471,10 @@ int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, 
         if (batch - b0 > 1 && bt == 1 && widest >= 4) bt = 4;          // 2 or 3 left: one padded tile of 4
         a.X = X + (int64_t)b0 * ldx; a.Y = Y + (int64_t)b0 * ldy; a.nb = std::min(bt, batch - b0);
         rc = dispatch_tile(A, a, st, bt);
-        if (rc == kTileDoesNotFit) { widest = bt == 8 ? 4 : 1; rc = CSB_OK; continue; }
+        if (rc == kTileDoesNotFit) {
+            if (bt == 1) { set_error("the planned CTA of %d warps does not fit shared memory even for one batch column", P.warps); rc = CSB_ERR_LAUNCH; break; }
+            widest = bt == 8 ? 4 : 1; rc = CSB_OK; continue;
+        }
         b0 += a.nb;
     }
     if (prev != A->device) cudaSetDevice(prev);
@@ -573,11 +539,9 @@ int launch_spmv_static_scratch(const csb_matrix* A, const float* x, float* y, vo
     a.ldx = A->cols; a.ldy = A->rows; a.status = P.d_status; a.n_warps = P.n_warps;
     a.rows = (int)A->rows; a.cols = (int)A->cols; a.block_r = A->block_r; a.stage_bytes = P.stage_bytes; a.stages = P.stages;
     a.X = x; a.Y = y; a.nb = 1;
-#ifdef CSB_PHASE_CLOCKS
-    a.clocks = g_phase_clocks;
-    if (!a.clocks) { set_error("instrumented build: call csb_spmv once first"); return CSB_ERR_UNSUPPORTED; }
-#endif
-    return dispatch_tile(A, a, st, 1);
+    rc = dispatch_tile(A, a, st, 1);
+    if (rc == kTileDoesNotFit) { set_error("the planned CTA of %d warps does not fit shared memory", P.warps); rc = CSB_ERR_LAUNCH; }
+    return rc;
 }
 
 }  // namespace csb

@@ -5,8 +5,11 @@
 // "context link" feeding the next step).  A CTA owns a tile of hidden units with all gate
 // rows of those units; its compressed weights stay in shared memory for the whole sequence
 // when they fit (otherwise they are re-streamed from L2 through the same bulk-copy ring as
-// the bare product).  Only h_t crosses CTAs, through global memory and one bounded grid
-// barrier per step.  Stacked layers run as a wavefront: in tick k layer l does step k - 2 l.
+// the bare product).  Only h_t crosses CTAs, through global memory.  At batch 1 every h value
+// is published together with the number of its step in one 8-byte store and readers spin
+// (bounded) on the step number, so CTAs and stacked layers run as a dataflow pipeline without a
+// grid barrier.  At larger batches one bounded grid barrier per step orders the exchange and
+// stacked layers run as a wavefront: in tick k layer l does step k - 2 l.
 #include <algorithm>
 #include <list>
 #include <memory>
@@ -439,9 +442,15 @@ __global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
                 }
             }
             RNN_LAP(5);
-            // slot t & 3 still holds step t - 4: the layer above must have read it
+            // slot t & 3 still holds step t - 4: every CTA of the layer above must have read it, i.e.
+            // each of its n CTAs must have counted at least t - 3 reads.  Only the sum of the counts is
+            // kept.  CTAs of one layer are never more than two steps apart (a CTA cannot finish step
+            // s + 1 before all of them have published, hence read the input of, step s), so if one CTA
+            // stood at t - 4 the others would stand at t - 2 at most and the sum at n (t - 2) - 2 at
+            // most: a sum of n (t - 2) - 1 rules that out.  The layer above reaches n (t - 2) without
+            // anything newer than step t - 3 from this layer, so the wait ends.
             if (need_above && threadIdx.x == 0) {
-                const unsigned int need = (unsigned int)(t - 3) * (unsigned int)a.layer_ctas[layer + 1];
+                const unsigned int need = (unsigned int)(t - 2) * (unsigned int)a.layer_ctas[layer + 1] - 1u;
                 unsigned long long t0 = 0;
                 unsigned int spins = 0;
                 while (above_now < need) {

@@ -1,0 +1,104 @@
+"""In-kernel phase timing of the two batch-1 kernels, from an instrumented build of the library.
+
+    python -m paper_2005_05758_b200.phase_clocks rnn   [cfg1 cfg2 cfg3 cfg5]
+    python -m paper_2005_05758_b200.phase_clocks panel [4 8 16 25]
+
+Builds libcsb_clocks.so beside the normal library with -DCSB_PHASE_CLOCKS -DCSB_PANEL_CLOCKS (see
+build.py), loads it instead of libcsb.so and prints
+  rnn:   cycles per timestep and phase of csb_rnn_kernel, summed by thread 0 of every CTA
+         (mean / min / max over the CTAs);
+  panel: wall-clock stamps of csb_panel_kernel per CTA, in microseconds from the earliest CTA start.
+The instrumented kernels are slower than the product ones (thread 0 reads the clock between phases),
+so these figures say where the time goes, never how long a call takes.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import sys
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+ROOT = os.path.dirname(HERE)
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+RNN_PHASES = ["stage input half", "walk items (both halves)", "sync after accumulator sums", "gates + publish",
+              "wait for h of the other CTAs", "activations (thread 0)", "slot-reuse guard", "loads + adds + shuffles of the sums"]
+PANEL_STAMPS = ["CTA start", "barriers set, first copies out", "bookkeeping + x landed", "inputs gathered", "bundles done",
+                "y stored", "-", "-"]
+
+
+def _load():
+    from paper_2005_05758_b200 import build
+    lib = build.build(defines=build.INSTRUMENT_DEFINES, out=os.path.join(HERE, "libcsb_clocks.so"))
+    os.environ["CSB_LIBRARY"] = lib
+    import torch
+    from paper_2005_05758_b200 import binding
+    return torch, binding
+
+
+def rnn(names):
+    import workloads
+    torch, binding = _load()
+    for name in names:
+        w = workloads.CONFIGS[name](**({"T": 128} if name == "cfg5" else {}))
+        mats = [binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, 0) for m in w.layers]
+        L, B, H, T = len(w.layers), w.B, w.hidden_size, w.T
+        x = torch.from_numpy(w.x).cuda()
+        y = torch.empty((T, B, H), device="cuda")
+        hT = torch.empty((L, B, H), device="cuda")
+        cT = torch.empty((L, B, H), device="cuda")
+        for _ in range(3):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            if w.cell == "lstm":
+                binding.csb_lstm_forward(mats, None, x, None, None, y, hT, cT, 0)
+            else:
+                binding.csb_gru_forward(mats, None, x, None, y, hT, 0)
+            b.record()
+            torch.cuda.synchronize()
+        ck = np.zeros((256, 8), np.int64)
+        n = binding.lib.csb_debug_rnn_clocks(C.c_void_p(ck.ctypes.data), 256)
+        ck = ck[:n] / T
+        print("%s: T=%d, %d CTAs, %.2f us per step (instrumented)" % (name, T, n, a.elapsed_time(b) * 1e3 / T))
+        for i, nm in enumerate(RNN_PHASES):
+            print("   %-38s cycles/step mean %7.0f  min %7.0f  max %7.0f" % (nm, ck[:, i].mean(), ck[:, i].min(), ck[:, i].max()))
+        for m in mats:
+            m.free()
+
+
+def panel(rates):
+    import workloads
+    torch, binding = _load()
+    for rate in rates:
+        w = workloads.CONFIGS["cfg4"](rate=float(rate), B=1)
+        m = w.matrix
+        A = binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, 0)
+        n = A.info()["panel_ctas"]
+        x = torch.from_numpy(w.X).cuda()
+        y = torch.empty(m.rows, device="cuda")
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        for _ in range(3):
+            flush.zero_()
+            binding.csb_spmv(A, x[0], y)
+            torch.cuda.synchronize()
+        ck = np.zeros((n, 8), np.uint64)
+        binding.lib.csb_debug_panel_clocks(C.c_void_p(ck.ctypes.data), n)
+        t = (ck.astype(np.float64) - float(ck[:, 0].min())) / 1e3
+        print("cfg4 rate %sx: %d CTAs, stamps in us from the earliest CTA start (cold L2)" % (rate, n))
+        for i, nm in enumerate(PANEL_STAMPS[:6]):
+            print("   %-34s mean %6.2f  min %6.2f  max %6.2f" % (nm, t[:, i].mean(), t[:, i].min(), t[:, i].max()))
+        A.free()
+
+
+if __name__ == "__main__":
+    what = sys.argv[1] if len(sys.argv) > 1 else "rnn"
+    rest = sys.argv[2:]
+    if what == "rnn":
+        rnn(rest or ["cfg1", "cfg2", "cfg3", "cfg5"])
+    elif what == "panel":
+        panel(rest or ["4", "25"])
+    else:
+        raise SystemExit(__doc__)

@@ -47,3 +47,20 @@ def test_project_argument_checks_need_no_gpu():
     assert lib.csb_project(fake, 8, 8, 8, 4, 4, float("nan"), fake, fake, fake, big, None) == -1
     assert lib.csb_project(fake, 8, 8, 8, 4, 4, 0.5, fake, fake, fake, 16, None) == -1 and b"workspace" in lib.csb_last_error()
     assert lib.csb_project(fake, 30000, 64, 64, 32, 32, 0.5, fake, fake, fake, big, None) == -8 and b"20480" in lib.csb_last_error()
+
+
+def test_plan_opts_out_of_range_are_refused():
+    # checked before anything is planned, so a host-only handle (device = -1) shows it without a GPU
+    import numpy as np
+    import pytest
+    from paper_2005_05758_b200 import binding
+    W = np.ones((8, 8), np.float32)
+    rk = ck = np.ones(8 * 2, np.uint8)
+    ok = binding.csb_encode(W, 4, 4, rk, ck, "f16", -1, dict(ctas=3, warps_per_cta=16, stage_bytes=16384, stages=8))
+    ok.free()
+    for bad in (dict(stages=9), dict(stage_bytes=512), dict(stage_bytes=1 << 20), dict(warps_per_cta=17), dict(ctas=-1)):
+        opts = dict(ctas=0, warps_per_cta=0, stage_bytes=0, stages=0)
+        opts.update(bad)
+        with pytest.raises(binding.CsbError) as e:
+            binding.csb_encode(W, 4, 4, rk, ck, "f16", -1, opts)
+        assert e.value.status == -1 and "csb_plan_opts" in str(e.value)

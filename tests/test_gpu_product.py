@@ -115,6 +115,22 @@ def test_schedules_agree(opts):
     run_case(w.matrix, w.X, full)
 
 
+def test_ring_too_large_for_16_warps_is_planned_with_fewer(spmv_path):
+    # 128 block-rows make the plan row-owned (the CTA shape is then part of the plan); eight stages
+    # of 8 KB per warp do not fit 16 warps, so the planner has to settle for fewer warps per CTA
+    # instead of producing a plan that can never be launched
+    if spmv_path != "stream":
+        pytest.skip("csb_plan_opts belong to the stream kernel")
+    rng = np.random.default_rng(17)
+    R, C, br, bc = 8192, 512, 64, 64
+    nblk = (R // br) * (C // bc)
+    mat = workloads.MatrixSpec((rng.standard_normal((R, C)) * 0.1).astype(np.float32), br, bc,
+                               (rng.random(nblk * br) < 0.4).astype(np.uint8), (rng.random(nblk * bc) < 0.4).astype(np.uint8), "f32")
+    for B in (1, 5):
+        info = run_case(mat, rng.standard_normal((B, C)).astype(np.float32), dict(ctas=0, warps_per_cta=0, stage_bytes=8192, stages=8))
+        assert info["plan_warps"] < 16
+
+
 @pytest.mark.parametrize("ctas,stage,ring", [(4, 8192, 14), (16, 8192, 15), (148, 16384, 15)])
 def test_panel_ring_is_refilled_many_times(monkeypatch, spmv_path, ctas, stage, ring):
     # few CTAs and a ring of two or four small stages: every slot is refilled dozens of times and
@@ -127,8 +143,31 @@ def test_panel_ring_is_refilled_many_times(monkeypatch, spmv_path, ctas, stage, 
     run_case(w.matrix, w.X, dict(ctas=ctas, warps_per_cta=0, stage_bytes=0, stages=0), repeat=3)
 
 
-def test_cfg4_full_size_sampled():
-    # the benchmark's matrix: full parity on a sample of rows is implied by full comparison here
-    w = workloads.CONFIGS["cfg4"](rate=16.0, B=1)
-    info = run_case(w.matrix, w.X)
-    assert info["balance"] > 0.5
+@pytest.mark.parametrize("rate", [4.0, 8.0, 16.0, 25.0])
+def test_cfg4_full_size_every_rate_and_batch(rate, spmv_path):
+    # the benchmarked matrices themselves (8192 x 8192, 64 x 64 blocks), every output compared with
+    # the oracle at every benchmarked batch size; the batched cases do not depend on the SpMV kernel
+    # choice and run once
+    w = workloads.CONFIGS["cfg4"](rate=rate, B=64)
+    m = w.matrix
+    args = (m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype)
+    want, scale = O.spmm(*args, w.X), O.abs_scale(*args, w.X)
+    A = binding.csb_encode(*args[:5], m.val_dtype, 0)
+    Xd = torch.from_numpy(w.X).cuda()
+    for B in ((1,) if spmv_path == "stream" else (1, 8, 64)):
+        outs = []
+        for _ in range(2):
+            Y = torch.full((B, m.rows), float("nan"), device="cuda")
+            if B == 1:
+                binding.csb_spmv(A, Xd[0], Y[0])
+            else:
+                binding.csb_spmm(A, Xd[:B], Y)
+            torch.cuda.synchronize()
+            outs.append(Y.cpu().numpy())
+        assert np.array_equal(outs[0], outs[1]), "two runs differ bitwise at batch %d" % B
+        check_product(outs[0], want[:B], scale[:B], m.val_dtype)
+        big = np.abs(want[:B]) > 1e-2 * scale[:B]
+        print("cfg4 %gx batch %d: max relative error %.3g over %d outputs above the floor"
+              % (rate, B, float(np.max(np.abs(outs[0] - want[:B])[big] / np.abs(want[:B])[big])), int(big.sum())))
+    assert A.info()["balance"] > 0.5
+    A.free()

@@ -36,6 +36,33 @@ def test_hand_example_arrays(vd):
     assert O.spmv_from_encoding(enc, g["x"]).tolist() == g["y"]
 
 
+@pytest.mark.parametrize("vd", ["f32", "f16"])
+def test_hand_example_abs_scale(vd):
+    # abs_scale sets the floor of every product tolerance, so it gets its own hand-written pin:
+    # an input of mixed signs (y differs from the scale), the same scale for W and -W, and the
+    # brute-force sum of |w||x| over all mask settings of a small matrix below
+    g, W = _hand()
+    xs = np.array([g["x_signed"]], dtype=np.float32)
+    for sign in (1.0, -1.0):
+        args = (sign * W, 2, 3, g["row_keep"], g["col_keep"], vd)
+        assert (sign * O.spmm(*args, xs)[0]).tolist() == g["y_signed"]
+        assert O.abs_scale(*args, xs)[0].tolist() == g["abs_scale_signed"]
+    # two batch rows keep their own scales
+    both = np.array([g["x_signed"], g["x"]], dtype=np.float32)
+    assert O.abs_scale(W, 2, 3, g["row_keep"], g["col_keep"], vd, both).tolist() == [g["abs_scale_signed"], g["y"]]
+
+
+def test_abs_scale_brute_force_all_masks():
+    rng = np.random.default_rng(11)
+    W = rng.integers(-8, 9, (4, 4)).astype(np.float32)
+    x = rng.integers(-8, 9, 4).astype(np.float32)
+    for bits in range(256):
+        rk = [(bits >> k) & 1 for k in range(8)]
+        ck = [((bits * 37 + 5) >> k) & 1 for k in range(8)]
+        want = _brute_spmv(np.abs(W), 2, 2, rk, ck, np.abs(x))     # scalar loops over |w| * |x|
+        assert O.abs_scale(W, 2, 2, rk, ck, "f32", x[None, :])[0].tolist() == want
+
+
 def _brute_spmv(W, BR, BC, rk, ck, x):
     """Scalar triple loop straight from the definition of the block pattern."""
     R, C = W.shape
