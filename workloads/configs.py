@@ -127,15 +127,17 @@ def make_matrix(seed, rows, cols, br, bc, law, *, w_std, val_dtype="f16", **mask
 @dataclass
 class RnnWorkload:
     """One recurrent workload: stacked layers, an input sequence, initial state."""
-    cell: str                        # "lstm" | "gru"
+    cell: str                        # "lstm" | "gru" | "lstmp" | "ligru" | "gru_rb" (reset gate before the product)
     input_size: int
     hidden_size: int
-    layers: List[MatrixSpec]         # layer l: [G*H, I_l + H], gate order i,f,g,o / r,z,n
-    bias: List[Optional[np.ndarray]]  # per layer float32 [4*H] (GRU: b_r, b_z, b_in, b_hn) or None
+    layers: List[MatrixSpec]         # layer l: [G*H, I_l + S], S = size of the recurrent state (H, or the projection size)
+    bias: List[Optional[np.ndarray]]  # per layer float32 (lstm, lstmp, gru: [4*H]; gru_rb: [3*H]; ligru: [2*H]) or None
     x: np.ndarray                    # float32 [T, B, I]
-    h0: Optional[np.ndarray]         # float32 [L, B, H] or None (= zeros)
-    c0: Optional[np.ndarray]
+    h0: Optional[np.ndarray]         # float32 [L, B, S] or None (= zeros)
+    c0: Optional[np.ndarray]         # float32 [L, B, H] (lstm, lstmp)
     name: str = ""
+    proj: Optional[List[MatrixSpec]] = None   # lstmp: per layer the projection [P, H]
+    proj_size: int = 0
 
     @property
     def T(self) -> int:
@@ -153,26 +155,34 @@ class SpmvWorkload:
     name: str = ""
 
 
+GATES = {"lstm": 4, "lstmp": 4, "gru": 3, "gru_rb": 3, "ligru": 2}
+BIAS_ROWS = {"lstm": 4, "lstmp": 4, "gru": 4, "gru_rb": 3, "ligru": 2}
+
+
 def make_rnn_workload(seed, cell, I, H, n_layers, br, bc, law, *, T, B, w_std, x_law="normal",
-                      val_dtype="f16", bias_std=0.0, state_std=0.0, name="", **mask_kw) -> RnnWorkload:
-    G = 4 if cell == "lstm" else 3
-    layers, biases = [], []
+                      val_dtype="f16", bias_std=0.0, state_std=0.0, name="", proj_size=0, **mask_kw) -> RnnWorkload:
+    G = GATES[cell]
+    S = proj_size if cell == "lstmp" else H          # width of the recurrent state
+    layers, biases, proj = [], [], []
     _, _, rng_x = _streams(seed)
     for l in range(n_layers):
-        in_l = I if l == 0 else H
-        layers.append(make_matrix(seed + 1000 * l, G * H, in_l + H, br, bc, law,
+        in_l = I if l == 0 else S
+        layers.append(make_matrix(seed + 1000 * l, G * H, in_l + S, br, bc, law,
                                   w_std=w_std, val_dtype=val_dtype, **mask_kw))
+        if cell == "lstmp":
+            proj.append(make_matrix(seed + 1000 * l + 500, S, H, br, bc, law, w_std=w_std, val_dtype=val_dtype, **mask_kw))
     if x_law == "normal":
         x = rng_x.standard_normal((T, B, I), dtype=np.float32)
     else:
         x = rng_x.uniform(-1.0, 1.0, (T, B, I)).astype(np.float32)
     for l in range(n_layers):
-        biases.append((rng_x.standard_normal(4 * H) * bias_std).astype(np.float32) if bias_std > 0 else None)
+        biases.append((rng_x.standard_normal(BIAS_ROWS[cell] * H) * bias_std).astype(np.float32) if bias_std > 0 else None)
     h0 = c0 = None
     if state_std > 0:
-        h0 = (rng_x.standard_normal((n_layers, B, H)) * state_std).astype(np.float32)
+        h0 = (rng_x.standard_normal((n_layers, B, S)) * state_std).astype(np.float32)
         c0 = (rng_x.standard_normal((n_layers, B, H)) * state_std).astype(np.float32)
-    return RnnWorkload(cell, I, H, layers, biases, x, h0, c0 if cell == "lstm" else None, name)
+    return RnnWorkload(cell, I, H, layers, biases, x, h0, c0 if cell in ("lstm", "lstmp") else None, name,
+                       proj if cell == "lstmp" else None, S if cell == "lstmp" else 0)
 
 
 def make_spmv_workload(seed, rows, cols, br, bc, law, *, batch, w_std, val_dtype="f16", name="",
