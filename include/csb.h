@@ -160,8 +160,9 @@ void csb_free(csb_matrix_t* A);
  * Matrices with fp16 values (block_c <= 128, cols <= 16384) run the panel kernel: every CTA owns
  * a range of output rows, so it needs no scratch.  That kernel is launched with programmatic
  * stream serialization: its start-up overlaps the end of the work in front of it on `stream`,
- * and it waits for that work before it reads x or writes y (set CSB_PANEL_PDL=0 in the
- * environment for an ordinary launch, CSB_NO_PANEL=1 at encode time for the other kernel).
+ * and it waits for that work before it reads x or writes y (CSB_PANEL_PDL=0 in the environment,
+ * looked up at every call, asks for an ordinary launch; CSB_NO_PANEL=1 at encode time for the other
+ * kernel).
  */
 int csb_spmv(const csb_matrix_t* A, const float* x, float* y, void* stream);
 
@@ -172,14 +173,16 @@ int csb_spmv(const csb_matrix_t* A, const float* x, float* y, void* stream);
  *   Y  device, float32, batch rows of `rows` values, row stride ldy >= rows, overwritten.
  * batch = 0 is a no-op.  Same ordering / overlap rules as csb_spmv; results are bit-reproducible.
  * With batch >= 8, fp16 values and block_r <= 64 the product runs on tensor cores (the kernel
- * matrix times the gathered inputs is then a dense contraction): the inputs of a slab of 32 batch
- * columns are split into two binary16 halves (x = hi + lo, so no input precision is lost as long
- * as |x| < 65504) and multiplied with mma.sync, fp32 accumulation.  The first such call on a
- * handle builds a second device layout and a staging buffer for it (allocates and synchronises
- * the device once; make it outside of any stream capture).  The two kernels of this path are
- * launched with programmatic stream serialization and wait, first thing, for the work in front of
- * them on `stream`.  Other cases use the CUDA-core kernel
- * in batch tiles of 8 / 4 / 1.
+ * matrix times the gathered inputs is then a dense contraction), 32 batch columns per pass: the
+ * inputs are split into two binary16 halves (x = hi + lo, so no input precision is lost as long
+ * as |x| < 65504; larger or non-finite inputs give inf / NaN) and multiplied with
+ * mma.sync.m16n8k16, fp32 accumulation, a block-row's outputs staying in registers across its
+ * blocks.  The first such call on a handle for a batch size class (<= 8, <= 16, more)
+ * builds a device layout for that class, a staging buffer for the packed inputs and, where row
+ * groups are shared between CTAs, scratch for their partial sums (allocates and synchronises the
+ * device once; make it outside of any stream capture).  The two kernels of this path are launched
+ * with programmatic stream serialization and wait, first thing, for the work in front of them on
+ * `stream`.  Other cases use the CUDA-core kernel in batch tiles of 8 / 4 / 1.
  */
 int csb_spmm(const csb_matrix_t* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy,
              void* stream);
@@ -308,6 +311,34 @@ int csb_plan_dump(const csb_matrix_t* A, int ctas, int warps_per_cta, int stage_
  */
 int csb_panel_dump(const csb_matrix_t* A, int ctas, int warps_per_cta, int stage_bytes, int64_t* info_out,
                    uint8_t* panels_out, int64_t panels_cap, uint32_t* cta_out, int64_t cta_cap);
+
+/*
+ * csb_spmm_plan_dump -- inspection / testing aid (the paper has no counterpart): plan the
+ * tensor-core layout of the batched product for a pass of `batch` columns (the class of batch sizes
+ * <= 8, <= 16 or more) and `sm_count` SMs on the host only and copy it out, so that the layout and
+ * the block -> CTA -> warp schedule can be checked without a GPU.  A CTA covers RG consecutive
+ * block-rows times a range of block-columns and has W warps (32 for up to 8 batch columns, else
+ * 16), each working for one block-row of the group; S CTAs share a row group.  Weight stream
+ * cta * W + w belongs to warp w.
+ *   info_out          host, int64[8]: CTAs, chunks, stream bytes, RG, 8-column batch tiles per warp
+ *                     + 256 * W, S, and the warp-level and CTA-level balance (mean / max of the
+ *                     modelled cost) times 1e6.
+ *   stream_out        host, `stream_cap` bytes, or NULL;  chunks_out  host, uint32 pairs (offset in
+ *                     16-byte units, bytes), or NULL;  stream_begin_out  host, uint32 first chunk of
+ *                     every weight stream plus one end entry, or NULL;  cta_out  host, 48 bytes per
+ *                     CTA (int32 row group, range number, first block-column, block-columns, then
+ *                     32 bytes: the block-row of the group each warp works for), `cta_cap` CTAs, or NULL.
+ * A chunk is 16 bytes (first word: size of what follows in 16-byte units) followed by items; an
+ * item is 16 bytes (u16 block-column counted from the CTA's first, u8 kept columns nk, u8 words
+ * per stored row, u64 mask of the kept in-block rows, u16 size in 16-byte units), nk column indices
+ * padded to 4 bytes, and the kept rows of the column slice, row-major, each padded to an even
+ * number of halves.
+ * Errors: UNSUPPORTED when the layout does not apply (fp32 values, block_r > 64), INVALID_ARG for a
+ * buffer that is too small; call once with NULL buffers to learn the sizes.
+ */
+int csb_spmm_plan_dump(const csb_matrix_t* A, int batch, int sm_count, int64_t* info_out, uint8_t* stream_out, int64_t stream_cap,
+                       uint32_t* chunks_out, int64_t chunks_cap, uint32_t* stream_begin_out, int64_t begin_cap, int32_t* cta_out,
+                       int64_t cta_cap);
 
 /* Short text for a status code; never NULL. */
 const char* csb_strerror(int status);

@@ -175,6 +175,26 @@ def csb_plan_dump(A: CsbMatrix, ctas: int, warps_per_cta: int, stage_bytes: int)
     return out
 
 
+def csb_spmm_plan_dump(A: CsbMatrix, batch: int, sm_count: int) -> dict:
+    """Host-only plan of the tensor-core batched product, copied out for inspection (see csb.h)."""
+    lib.csb_spmm_plan_dump.argtypes = [_P, C.c_int, C.c_int, _P, _P, C.c_int64, _P, C.c_int64, _P, C.c_int64, _P, C.c_int64]
+    lib.csb_spmm_plan_dump.restype = C.c_int
+    info = np.zeros(8, np.int64)
+    _check(lib.csb_spmm_plan_dump(A.handle, batch, sm_count, info.ctypes.data, None, 0, None, 0, None, 0, None, 0))
+    n_ctas, n_chunks, n_bytes = (int(v) for v in info[:3])
+    NT, warps = int(info[4]) & 255, int(info[4]) >> 8
+    stream = np.zeros(max(n_bytes, 1), np.uint8)
+    chunks = np.zeros((max(n_chunks, 1), 2), np.uint32)
+    begin = np.zeros(n_ctas * warps + 1, np.uint32)
+    cta = np.zeros((max(n_ctas, 1), 48), np.uint8)
+    _check(lib.csb_spmm_plan_dump(A.handle, batch, sm_count, info.ctypes.data, stream.ctypes.data, stream.size, chunks.ctypes.data,
+                                  chunks.shape[0], begin.ctypes.data, begin.size, cta.ctypes.data, cta.shape[0]))
+    cta = cta[:n_ctas]
+    return {"ctas": n_ctas, "RG": int(info[3]), "NT": NT, "warps": warps, "S": int(info[5]), "warp_balance": info[6] / 1e6,
+            "balance": info[7] / 1e6, "stream": stream[:n_bytes], "chunk_table": chunks[:n_chunks], "stream_begin": begin,
+            "cta": cta[:, :16].copy().view(np.int32).reshape(n_ctas, 4), "warp_row": cta[:, 16:16 + warps].copy()}
+
+
 def csb_panel_dump(A: CsbMatrix, ctas: int, warps_per_cta: int, stage_bytes: int) -> dict:
     """Host-only plan of the batch-1 panel layout, copied out for inspection (see csb.h)."""
     lib.csb_panel_dump.argtypes = [_P, C.c_int, C.c_int, C.c_int, _P, _P, C.c_int64, _P, C.c_int64]

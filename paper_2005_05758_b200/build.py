@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcsb.so")
-SOURCES = ["csb_api.cpp", "csb_encode.cpp", "csb_plan.cpp", "csb_schedule.cpp", "csb_mma_plan.cpp", "csb_panel_plan.cpp", "csb_product.cu", "csb_panel.cu", "csb_spmm_mma.cu", "csb_rnn.cu", "csb_rnn_step.cu", "csb_project.cu"]
+SOURCES = ["csb_api.cpp", "csb_encode.cpp", "csb_plan.cpp", "csb_schedule.cpp", "csb_spmm_plan.cpp", "csb_panel_plan.cpp", "csb_product.cu", "csb_panel.cu", "csb_spmm_mma.cu", "csb_rnn.cu", "csb_rnn_step.cu", "csb_project.cu"]
 HEADERS = ["csb_internal.hpp", "csb_device.cuh", os.path.join("..", "..", "include", "csb.h")]
 
 
@@ -22,9 +22,10 @@ def _stale() -> bool:
 
 #: Instrumented variants (never the default build).  CSB_PHASE_CLOCKS makes the time-loop kernel sum
 #: clock64() cycles per phase and CTA (read back with csb_debug_rnn_clocks); CSB_PANEL_CLOCKS makes
-#: the SpMV panel kernel record wall-clock stamps per phase and CTA (csb_debug_panel_clocks).
+#: the SpMV panel kernel record wall-clock stamps per phase and CTA (csb_debug_panel_clocks);
+#: CSB_SPMM_CLOCKS makes the batched tensor-core kernel sum cycles per phase and warp (csb_debug_spmm_clocks).
 #: paper_2005_05758_b200/phase_clocks.py builds such a library beside the normal one and prints the figures.
-INSTRUMENT_DEFINES = ("CSB_PHASE_CLOCKS", "CSB_PANEL_CLOCKS")
+INSTRUMENT_DEFINES = ("CSB_PHASE_CLOCKS", "CSB_PANEL_CLOCKS", "CSB_SPMM_CLOCKS")
 
 
 def build(force: bool = False, verbose: bool = False, defines=(), out: str = None) -> str:

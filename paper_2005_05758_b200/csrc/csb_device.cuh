@@ -38,13 +38,31 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Wait for a phase with a wall-clock bound; false = gave up.
+// The same test, but a thread that finds the phase unfinished may be parked by the hardware for up
+// to `ns` nanoseconds (it wakes when the phase completes): waiting warps then leave the issue slots
+// to the warps that still have work.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(ns) : "memory");
+    return ok != 0;
+}
+// Wait for a phase with a wall-clock bound; false = gave up.  The clock (a slow read) is looked at
+// only every 256 failed polls, so a wait that ends within microseconds never touches it.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
+    unsigned long long t0 = 0;
+    unsigned int spins = 0;
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (global_ns() - t0 > kCopyWaitNs) return false;
+        if ((++spins & 255u) == 0) {
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kCopyWaitNs) return false;
+        }
     }
 }
 // One bulk asynchronous copy global -> shared; completion is counted in bytes on `bar`.

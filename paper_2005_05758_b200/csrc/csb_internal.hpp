@@ -64,7 +64,7 @@ static_assert(sizeof(ChunkHeader) == 16, "header is one 16-byte word");
 
 enum : uint32_t { kFlushNone = 0, kFlushDirect = 1, kFlushPartial = 2, kFlushCta = 3, kFlushCtaPartial = 4, kSlotShift = 3 };
 enum : uint16_t { kItemRecurrent = 1 };
-enum { kMaxNk = 64, kItemAlign = 16, kMmaMaxNk = 32 };
+enum { kMaxNk = 64, kItemAlign = 16 };
 
 struct Chunk {
     uint32_t off16;    // offset of the chunk in the stream, in 16-byte units; top two bits: flush kind
@@ -196,29 +196,64 @@ struct RnnHostPlan {
 int plan_rnn_host(int gates, int n_layers, const csb_matrix* const* Wm, const int* in_size, int H, int n_ctas,
                   int warps, int stage_bytes, RnnHostPlan* out);
 
-// ---- tensor-core SpMM path (csb_mma_plan.cpp, csb_spmm_mma.cu) ----
-struct MmaItemHeader {
-    uint8_t nk, mr, RT, KT;   // kept columns / rows of the item, its 16-row and 8-column tile counts
-    uint32_t xbase;           // first column of the block
-    uint32_t pad[2];
+// ---- tensor-core SpMM path (csb_spmm_plan.cpp, csb_spmm_mma.cu) ----
+// The matrix is cut into CTA tiles: a group of RG consecutive block-rows times a contiguous range of
+// block-columns.  The warps of a CTA (16, or 32 for batches of up to 8) are dealt to the block-rows of its group in proportion to
+// their work; a warp keeps the block_r x batch outputs of its block-row in registers for the whole
+// range, and the blocks of a block-row go, in block-column order, to whichever of its warps has the
+// least work so far.  A warp's weights come through its own ring of bulk copies as items; the batch
+// of inputs comes through one ring of block-column tiles shared by the CTA.  An item is a column
+// slice (<= 64 kept columns) of one block:
+//   SpmmItemHeader (16 B), col_idx[nk] (in-block column indices, padded to 4 B), then the kernel
+//   matrix rows of the slice, row-major, each padded to an even number of halves (np2 words).
+// Items travel in chunks of at most kSpmmStageBytes; the chunks of a warp lie back to back, and a
+// chunk's 16-byte header holds the size of its items (16-byte units) and the byte sizes of the next
+// three chunks of the warp, so that a warp refills its ring without looking anything up in global memory.
+struct SpmmItemHeader {
+    uint16_t tile;            // block-column, counted from the CTA's first one
+    uint8_t nk;               // kept columns in this item, 1..64
+    uint8_t np2;              // 32-bit words per stored row, ceil(nk / 2)
+    uint32_t mask_lo, mask_hi;   // bit r: in-block row r is kept in this block
+    uint16_t size16;          // size of the item in 16-byte units
+    uint16_t pad;
 };
-static_assert(sizeof(MmaItemHeader) == 16, "header is one 16-byte word");
-struct MmaHostPlan {
-    std::vector<uint8_t> bytes;
+static_assert(sizeof(SpmmItemHeader) == 16, "header is one 16-byte word");
+enum { kSpmmStageBytes = 2304, kSpmmMaxWarps = 32 };
+struct SpmmCta {
+    int32_t group, split, tile0, ntiles;     // row group, which column range of it, the range in block-columns
+    uint8_t warp_row[kSpmmMaxWarps];         // which block-row of the group each warp works for (ascending)
+};
+static_assert(sizeof(SpmmCta) == 48, "three 16-byte words");
+// Warps per CTA: the 16 accumulator registers of one 8-column batch tile leave room for 32 warps per
+// SM, which halves the chain of dependent work a warp has to get through; wider tiles allow 16.
+inline int spmm_warps(int NT) { return NT == 1 ? 32 : 16; }
+// Batch classes: how many 8-column batch tiles a warp carries.  A pass covers 8 * NT <= 32 batch columns.
+inline int spmm_nt(int batch) { return batch <= 8 ? 1 : batch <= 16 ? 2 : 4; }
+inline int spmm_class_index(int batch) { return batch <= 8 ? 0 : batch <= 16 ? 1 : 2; }
+inline int spmm_pitch(int NT) { return NT * 32 + 16; }   // bytes of one packed input column: hi parts, lo parts, 16 spare
+struct SpmmHostPlan {
+    std::vector<uint8_t> bytes;               // all chunks back to back
     std::vector<Chunk> chunks;
-    std::vector<uint32_t> warp_chunk_begin;
-    int ctas = 0, warps_per_cta = 0;
-    size_t max_chunk_bytes = 0;
-    double balance = 1.0;
+    std::vector<uint32_t> stream_begin;       // [n_ctas * warps + 1] first chunk of every warp's weight stream
+    std::vector<uint32_t> warp_desc;          // four words per warp: first chunk's offset (16-byte units), chunk count,
+                                              // bytes of chunks 0 and 1 (16 bits each), bytes of chunk 2
+    std::vector<SpmmCta> ctas;
+    int RG = 1, S = 1, n_groups = 0, max_tiles = 0;
+    double balance = 1.0, warp_balance = 1.0; // mean / max of the modelled cost over CTAs, and over warps
 };
-int plan_mma_host(const csb_matrix* A, int ctas, int warps_per_cta, int stage_bytes, MmaHostPlan* out);
-struct MmaPlan {                           // device side, built on the first batched product
-    int ctas = 0, warps = 0, stage_bytes = 0, stages = 0, n_warps = 0;
-    uint8_t* d_stream = nullptr; Chunk* d_chunks = nullptr; void* d_warp_desc = nullptr;
-    void* d_xp = nullptr; size_t xp_bytes = 0;   // packed fp16 hi/lo copy of a 32-column batch slab
-    int64_t stream_bytes = 0;
-    double balance = 1.0;
-    bool built = false, unusable = false;
+// Plans for `sm_count` SMs; returns CSB_OK, or 1 when the path does not suit the matrix.
+int plan_spmm_host(const csb_matrix* A, int NT, int sm_count, SpmmHostPlan* out);
+struct MmaPlan {                           // device side, one per batch class, built on first use
+    struct PerClass {
+        bool built = false, unusable = false;
+        int RG = 1, S = 1, n_ctas = 0, n_groups = 0, x_depth = 0, w_stages = 0;
+        size_t smem_bytes = 0;
+        uint8_t* d_stream = nullptr; uint32_t* d_warp_desc = nullptr; SpmmCta* d_ctas = nullptr;
+        float* d_partials = nullptr; uint32_t* d_arrivals = nullptr;
+        void* d_xp = nullptr;
+        int64_t stream_bytes = 0;
+        double balance = 1.0, warp_balance = 1.0;
+    } cls[3];
 };
 int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream);
 bool spmm_mma_applicable(const csb_matrix* A, int batch);

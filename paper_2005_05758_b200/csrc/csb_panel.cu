@@ -89,11 +89,16 @@ __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepco
 // has given up.
 __device__ __forceinline__ bool panel_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* dead) {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
+    unsigned long long t0 = 0;                     // the clock is a slow read: looked at every 256 failed polls only
+    unsigned int spins = 0;
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*dead) return false;
-        if (global_ns() - t0 > kCopyWaitNs) return false;
+        if ((++spins & 255u) == 0) {
+            if (*dead) return false;
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kCopyWaitNs) return false;
+        }
     }
 }
 
@@ -107,10 +112,15 @@ __device__ __forceinline__ bool panel_wait_stage(uint64_t* full, volatile uint32
                                                  volatile uint32_t* dead) {
     const uint32_t slot = st & ((1u << log2_slots) - 1u), use = st >> log2_slots;
     if (use > 0u && issued[slot] <= use) {
-        const unsigned long long t0 = global_ns();
+        unsigned long long t0 = 0;
+        unsigned int spins = 0;
         while (issued[slot] <= use) {
-            if (*dead) return false;
-            if (global_ns() - t0 > kCopyWaitNs) return false;
+            if ((++spins & 255u) == 0) {
+                if (*dead) return false;
+                const unsigned long long now = global_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > kCopyWaitNs) return false;
+            }
         }
     }
     return panel_wait(&full[slot], use & 1u, dead);
@@ -452,7 +462,7 @@ int launch_panels(const csb_matrix* A, const float* x, float* y, void* stream) {
     // Programmatic stream serialization lets this grid's start-up (barriers, first copies of the
     // panels) overlap the end of the kernel in front of it; the kernel orders itself behind that
     // kernel before it touches x or y.  CSB_PANEL_PDL=0 asks for an ordinary launch.
-    static const int use_pdl = env_int("CSB_PANEL_PDL", 1);
+    const int use_pdl = env_int("CSB_PANEL_PDL", 1);      // read at every launch, so a caller can compare both kinds
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)P.ctas); cfg.blockDim = dim3((unsigned)P.warps * 32u);
     cfg.dynamicSmemBytes = P.smem_bytes; cfg.stream = (cudaStream_t)stream;

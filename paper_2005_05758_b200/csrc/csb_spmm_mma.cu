@@ -1,16 +1,34 @@
 // Tensor-core CSB-SpMM (batch >= 8, fp16 values, fp32 accumulation).
 //
 // With a batch of vectors the product of a block's kernel matrix (m kept rows x n kept columns)
-// with the gathered inputs (n x batch) is a small dense contraction, the one place on this path
-// where tensor cores apply.  Every kernel matrix is stored as 16 x 8 tiles in the register order of
-// mma.sync.m16n8k8's A operand; the gathered inputs sit in shared memory as [column][batch] rows
-// of fp16 and reach the B operand through ldmatrix.trans.  fp32 inputs are split into two fp16
-// halves (x = hi + lo) and multiplied separately, so no input precision is lost; products are
-// accumulated in fp32.  One launch handles a slab of up to 32 batch columns.
+// with the gathered inputs (n x batch) of Section 4.3.1 is a small dense contraction, the one place
+// on this path where tensor cores apply.  How it is laid out here:
 //
-// The bulk-copy ring, the row-owned schedule (a CTA owns whole block-rows, a CTA barrier ends each
-// one, warps' private sums are added in a fixed order) and the bounded waits are those of the
-// CUDA-core product kernel.
+//   * A warp works for one block-row over a range of block-columns and keeps that block-row's
+//     outputs, all block_r rows x up to 32 batch columns, in the accumulator registers of
+//     mma.sync.m16n8k16 for the whole range (several warps share a block-row's blocks; their sums
+//     meet once, at the end).  The kernel matrix is the A operand with its kept rows put back at their
+//     RowIdx positions: a lane finds the stored row behind an output row with a population count
+//     on the block's 64-bit row mask and loads its fragment straight from the compact row-major
+//     values (rows that are not kept give zero registers).  So nothing is scattered and nothing is
+//     read-modify-written per block; the row indices never leave the registers.
+//   * The inputs are packed once per call into binary16 pairs x = hi + lo (no input precision is
+//     lost as long as |x| < 65504), one row of batch values per matrix column, and reach shared
+//     memory as whole block-column tiles through a ring that all warps of the CTA share, so a tile
+//     is fetched from L2 once per CTA and not once per block.  The tiles come in by cp.async (16-byte
+//     pieces through the load/store path, completion counted on an mbarrier), not by bulk copy: bulk
+//     copies of one SM complete in order, and a tile queued behind the weight copies, which wait for
+//     HBM, reached shared memory a microsecond late every time.  The gather through ColIdx is done by
+//     the operand load itself: every lane hands ldmatrix.trans the address of the tile row of one
+//     kept column.  hi and lo are multiplied separately into the same accumulators.
+//   * The weights of a warp come through its own ring of bulk copies, so warps with light and heavy
+//     blocks do not wait for each other; they only meet at the input tiles, which a warp releases
+//     in order whether it used them or not, the last warp to release a slot refilling it.
+//   * A CTA covers RG block-rows x a range of block-columns (the planner's cut).  When a row group
+//     is divided between S CTAs each writes its partial sums to scratch and the last one to arrive
+//     adds them in the order of the ranges, so results are bit-reproducible.
+//   * More than 32 batch columns are served in passes of 32 (the weights of the later passes come
+//     from L2).
 #include <algorithm>
 #include <cstdio>
 #include <mutex>
@@ -20,225 +38,396 @@
 
 namespace csb {
 
-constexpr int kSlab = 32;                    // batch columns per launch
-constexpr int kXRowBytes = 80;               // one gathered column: 32 halves + 16 bytes so ldmatrix rows miss each other's banks
-constexpr int kZStride = 34;                 // floats per output row in a warp's private sums (32 + 2: spreads banks)
 constexpr uint32_t kOffMaskM = 0x3fffffffu;
-constexpr int kXBuf = 2 * kMmaMaxNk * kXRowBytes;   // one gather buffer: hi rows, then lo rows
+constexpr uint32_t kNoRow = 0xffffffffu;
 
-struct MmaArgs {
+struct SpmmArgs {
     const uint8_t* stream;
-    const Chunk* chunks;
-    const uint4* warp_desc;
-    const __half* xp;          // [cols][64]: 32 hi halves, 32 lo halves of the slab
-    float* Y;                  // slab's first batch row
+    const uint4* warp_desc;    // per warp: first chunk's offset, chunk count, sizes of its first three chunks
+    const SpmmCta* ctas;
+    const uint8_t* xp;         // packed inputs: one row of `pitch` bytes per matrix column
+    float* Y;
     long long ldy;
+    float* partials;           // [group][range][8 * NT][RG * block_r], S > 1 only
+    uint32_t* arrivals;        // [group], zero between launches
     uint32_t* status;
-    int n_warps, nb, rows, block_r, stage_bytes, stages;
+    int nb, rows, cols, block_r, block_c, RG, S, x_depth, w_stages, pitch, tile_bytes;
+#ifdef CSB_SPMM_CLOCKS
+    long long* clocks;         // instrumented build only: [CTA][warp][8] cycles per phase
+#endif
 };
 
-struct MmaSmem {
-    size_t ring, bars, zs, xs, total;
-    __host__ __device__ MmaSmem(int W, int stages, int stage_bytes, int block_r) {
-        ring = 0;
-        bars = ring + (size_t)W * stages * stage_bytes;
-        zs = (bars + (size_t)W * stages * 8 + 15) & ~(size_t)15;
-        xs = (zs + (size_t)W * block_r * kZStride * 4 + 15) & ~(size_t)15;
-        total = xs + (size_t)W * 2 * 2 * kMmaMaxNk * kXRowBytes;       // two buffers x (hi, lo) x rows
+#ifdef CSB_SPMM_CLOCKS
+#define SPMM_LAP(i) do { const long long n_ = clock64(); sprof[i] += n_ - st_; st_ = n_; } while (0)
+#else
+#define SPMM_LAP(i) do { } while (0)
+#endif
+
+// Shared-memory carve-up, identical on host and device.  The small fixed part comes first; the two
+// rings follow and are reused for the warps' partial sums once the main loop is over.
+struct SpmmSmem {
+    size_t wfull, xfull, wcnt, xcnt, dead, zero, rings, wring, xring, total;
+    __host__ __device__ SpmmSmem(int n_warps, int w_stages, int x_depth, int tile_bytes, int pitch, int MT, int NT) {
+        const int n_streams = n_warps;
+        wfull = 0;
+        xfull = wfull + (size_t)n_streams * w_stages * 8;
+        wcnt = xfull + (size_t)x_depth * 8;
+        xcnt = wcnt + (size_t)n_streams * w_stages * 4;
+        dead = xcnt + (size_t)x_depth * 4;
+        zero = (dead + 4 + 127) & ~(size_t)127;
+        rings = (zero + (size_t)pitch + 127) & ~(size_t)127;
+        wring = rings;
+        xring = wring + (size_t)n_streams * w_stages * kSpmmStageBytes;
+        const size_t ring_end = xring + (size_t)x_depth * tile_bytes;
+        const size_t sums_end = rings + (size_t)n_warps * MT * 16 * (NT * 8 + 1) * 4;
+        total = ring_end > sums_end ? ring_end : sums_end;
     }
 };
 
-// Pack a slab of X: fp32 [batch][cols] -> fp16 hi / lo [cols][64] (batch columns past nb are zero).
-__global__ void csb_pack_x_kernel(const float* __restrict__ X, long long ldx, int nb, int cols, __half* __restrict__ xp) {
+// Pack X: fp32 [batch][cols] -> per column one row of binary16 values: the hi parts of the 8 * NT batch
+// columns, then the lo parts (x = hi + lo); batch columns past nb are zero.
+__global__ void csb_pack_x_kernel(const float* __restrict__ X, long long ldx, int nb, int cols, uint8_t* __restrict__ xp, int pitch, int NT) {
     pdl_launch_dependents();
     pdl_wait();                                    // X may come from the kernel in front; xp may still be read by it
-    const int col = blockIdx.x * (blockDim.x / kSlab) + threadIdx.x / kSlab, b = threadIdx.x % kSlab;
-    if (col >= cols) return;
-    const float x = b < nb ? X[(long long)b * ldx + col] : 0.f;
-    const __half hi = __float2half_rn(x);
-    const __half lo = __float2half_rn(x - __half2float(hi));
-    xp[(size_t)col * 64 + b] = hi;
-    xp[(size_t)col * 64 + kSlab + b] = lo;
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5, c0 = blockIdx.x * 32;
+    const int cap = 8 * NT;
+    for (int b = ty; b < cap; b += 8) tile[b][tx] = (b < nb && c0 + tx < cols) ? X[(long long)b * ldx + c0 + tx] : 0.f;
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < 32 * cap; idx += blockDim.x) {
+        const int c = idx / cap, b = idx % cap;
+        if (c0 + c >= cols) break;
+        const float x = tile[b][c];
+        const __half hi = __float2half_rn(x);
+        const __half lo = __float2half_rn(x - __half2float(hi));
+        __half* row = reinterpret_cast<__half*>(xp + (size_t)(c0 + c) * pitch);
+        row[b] = hi;
+        row[cap + b] = lo;
+    }
 }
 
-__device__ __forceinline__ void mma_m16n8k8(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(b0));
+__device__ __forceinline__ void mma_m16n8k16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* row_ptr) {
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(row_ptr)));
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t atom_add_acq_rel_shared(uint32_t* p, uint32_t v) {
+    uint32_t old;
+    asm volatile("atom.acq_rel.cta.shared.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(smem_u32(p)), "r"(v) : "memory");
+    return old;
 }
 
-template <int NT>
-__global__ void __launch_bounds__(256, 1) csb_spmm_mma_kernel(const MmaArgs a) {
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+template <int MT, int NT>
+__global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_kernel(const SpmmArgs a) {
+    constexpr int kSpmmWarps = NT == 1 ? 32 : 16;
     pdl_launch_dependents();
     extern __shared__ __align__(128) uint8_t smem[];
-    const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const MmaSmem L(W, a.stages, a.stage_bytes, a.block_r);
-    uint8_t* ring = smem + L.ring + (size_t)warp * a.stages * a.stage_bytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.bars) + warp * a.stages;
-    float* zs_all = reinterpret_cast<float*>(smem + L.zs);
-    float* zs = zs_all + (size_t)warp * a.block_r * kZStride;
-    uint8_t* xs_base = smem + L.xs + (size_t)warp * 2 * kXBuf;
-    const int g = lane >> 2, t = lane & 3;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const SpmmSmem L(kSpmmWarps, a.w_stages, a.x_depth, a.tile_bytes, a.pitch, MT, NT);
+    uint64_t* wfull = reinterpret_cast<uint64_t*>(smem + L.wfull) + warp * a.w_stages;
+    uint64_t* xfull = reinterpret_cast<uint64_t*>(smem + L.xfull);
+    uint32_t* xcnt = reinterpret_cast<uint32_t*>(smem + L.xcnt);
+    volatile uint32_t* s_dead = reinterpret_cast<volatile uint32_t*>(smem + L.dead);
+    uint8_t* wring = smem + L.wring + (size_t)warp * a.w_stages * kSpmmStageBytes;
+    uint8_t* xring = smem + L.xring;
+    const uint32_t zero_addr = smem_u32(smem + L.zero);
 
-    const int gw = blockIdx.x * W + warp;
-    uint4 wd = make_uint4(0u, 0u, 0u, 0u);
-    if (gw < a.n_warps) wd = __ldg(a.warp_desc + gw);
-    const uint32_t c0 = wd.x, c1 = wd.y;
-    if (lane == 0) {
-        for (int s = 0; s < a.stages; ++s) mbar_init(&bars[s], 1);
+#ifdef CSB_SPMM_CLOCKS
+    long long sprof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    long long st_ = clock64();
+#endif
+    // the CTA's descriptor goes to shared memory, one word per thread
+    __shared__ __align__(16) SpmmCta s_me;
+    __shared__ int s_first[5];                     // first warp of every block-row of the group (the warps of a row are neighbours)
+    if (threadIdx.x < sizeof(SpmmCta) / 4) reinterpret_cast<uint32_t*>(&s_me)[threadIdx.x] = reinterpret_cast<const uint32_t*>(a.ctas + blockIdx.x)[threadIdx.x];
+    const uint4 wd = __ldg(a.warp_desc + (size_t)blockIdx.x * kSpmmWarps + warp);
+    const uint32_t n_chunks = wd.y;
+    __syncthreads();
+    const SpmmCta* me = &s_me;
+    const int ntiles = me->ntiles, tile0 = me->tile0;
+    auto tile_bytes_of = [&](int tl) { return (uint32_t)min(a.block_c, a.cols - (tile0 + tl) * a.block_c) * (uint32_t)a.pitch; };
+    auto tile_src = [&](int tl) { return a.xp + (size_t)(tile0 + tl) * a.block_c * a.pitch; };
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kSpmmWarps * a.w_stages; ++i) mbar_init(reinterpret_cast<uint64_t*>(smem + L.wfull) + i, 1);
+        for (int i = 0; i < a.x_depth; ++i) { mbar_init(&xfull[i], 32); xcnt[i] = 0u; }    // one arrival per lane of the warp that fetches a tile
+        *s_dead = 0u;
         mbar_fence_init();
-        if (c0 < c1) {
-            mbar_expect_tx(&bars[0], wd.w);
-            bulk_g2s(ring, a.stream + (size_t)(wd.z & kOffMaskM) * 16, wd.w, &bars[0]);
-        }
-        for (int s = 1; s < a.stages && c0 + s < c1; ++s) {
-            const Chunk ch = a.chunks[c0 + s];
-            mbar_expect_tx(&bars[s], ch.bytes);
-            bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)(ch.off16 & kOffMaskM) * 16, ch.bytes, &bars[s]);
+    }
+    for (int i = threadIdx.x; i < (a.pitch + 16) / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem + L.zero)[i] = 0u;
+    __syncthreads();
+    // the weights were written at plan time: their first copies go out before the work in front is waited for
+    // (a warp's chunks lie back to back; issue_off is where the next one to be fetched starts)
+    uint32_t issue_off = wd.x;
+    {
+        const uint32_t first[3] = {wd.z & 0xffffu, wd.z >> 16, wd.w};
+        for (int s = 0; s < a.w_stages && s < (int)n_chunks; ++s) {
+            if (lane == 0) {
+                mbar_expect_tx(&wfull[s], first[s]);
+                bulk_g2s(wring + (size_t)s * kSpmmStageBytes, a.stream + (size_t)issue_off * 16, first[s], &wfull[s]);
+            }
+            issue_off += first[s] >> 4;
         }
     }
-    for (int i = lane; i < a.block_r * kZStride; i += 32) zs[i] = 0.f;
-    __syncwarp();
-    // everything so far touched only the planned stream (written once, at plan time) and shared
-    // memory; the packed inputs and Y belong to the work in front on the stream
-    pdl_wait();
-
-    bool dead = false, reported = false;
-    Chunk cur = Chunk{wd.z, wd.w};
-    for (uint32_t c = c0; c < c1; ++c) {
-        const int s = (int)((c - c0) % (uint32_t)a.stages);
-        const uint32_t parity = ((c - c0) / (uint32_t)a.stages) & 1u;
-        const uint32_t flush = cur.off16 >> 30;
-        const Chunk nxt = (c + 1 < c1) ? a.chunks[c + 1] : Chunk{0, 0};
-        const Chunk refill = (c + a.stages < c1) ? a.chunks[c + a.stages] : Chunk{0, 0};
-        if (!dead) dead = __any_sync(0xffffffffu, !mbar_wait_bounded(&bars[s], parity));
-        if (dead && !reported) {
-            reported = true;
-            if (lane == 0) {
-                *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout;
-                for (uint32_t j = c; j < c1 && j < c + (uint32_t)a.stages; ++j)
-                    mbar_wait_bounded(&bars[(j - c0) % (uint32_t)a.stages], ((j - c0) / (uint32_t)a.stages) & 1u);
-            }
-        }
-        if (dead) {                                   // keep the CTA's barriers company, touch no data
-            if (flush == kFlushCta) { __syncthreads(); __syncthreads(); }
-            cur = nxt;
-            continue;
-        }
-        const uint8_t* p = ring + (size_t)s * a.stage_bytes;
-        const uint4 chh = *reinterpret_cast<const uint4*>(p);
-        const uint8_t* end = p + 16 + 16 * (chh.x & 0xffffu);
-        p += 16;
-        // Gather of one item into buffer `buf`, asynchronously: each kept column is 128 contiguous
-        // bytes of the packed slab (64 hi, 64 lo); eight lanes move one column, four columns per pass;
-        // rows past nk up to the tile edge are zeroed.
-        auto gather_async = [&](const uint8_t* item, int buf) {
-            const uint4 hh = *reinterpret_cast<const uint4*>(item);
-            const int nk_ = (int)(hh.x & 0xffu), kpad_ = (int)(hh.x >> 24) * 8;
-            const uint8_t* cidx_ = item + 16;
-            uint8_t* hi = xs_base + buf * kXBuf;
-            const int piece = lane & 7;                           // 16-byte piece: 0..3 hi, 4..7 lo
-            for (int k = lane >> 3; k < kpad_; k += 4) {
-                uint8_t* dst = hi + (piece < 4 ? 0 : kMmaMaxNk * kXRowBytes) + k * kXRowBytes + (piece & 3) * 16;
-                if (k < nk_) {
-                    const void* src = reinterpret_cast<const uint4*>(a.xp + (size_t)(hh.y + cidx_[k]) * 64) + piece;
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
-                } else {
-                    *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+    if (threadIdx.x == 0) {
+        int rr = 0;
+        s_first[0] = 0;
+        for (int w = 0; w < kSpmmWarps; ++w)
+            while (rr < (int)me->warp_row[w]) s_first[++rr] = w;
+        while (rr < 4) s_first[++rr] = kSpmmWarps;
+    }
+    pdl_wait();                                    // the packed inputs and Y belong to the work in front on the stream
+    // One warp fetches a tile: every lane copies its 16-byte pieces and then arrives on the slot's
+    // barrier, the arrival taking effect when the lane's copies have landed.
+    auto fetch_tile = [&](int slot, int tl) {
+        const uint32_t bytes = tile_bytes_of(tl);
+        const uint8_t* src = tile_src(tl);
+        const uint32_t dst = smem_u32(xring + (size_t)slot * a.tile_bytes);
+        for (uint32_t off = (uint32_t)lane * 16u; off < bytes; off += 512u)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + off), "l"(src + off) : "memory");
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&xfull[slot])) : "memory");
+    };
+    if (warp == 0)
+        for (int tl = 0; tl < a.x_depth && tl < ntiles; ++tl) fetch_tile(tl, tl);
+    SPMM_LAP(0);                                   // set-up, first copies out, the work in front waited for
+    // A wait gives up after a second, or as soon as any warp of the CTA has given up.
+    auto wait_bar = [&](uint64_t* bar, uint32_t parity) -> bool {
+        bool ok = mbar_try_wait(bar, parity);
+        if (!ok) {
+            unsigned long long t0 = 0;                // the clock is a slow read: only every 256 failed polls
+            unsigned int spins = 0;
+            for (;;) {
+                if (mbar_try_wait_parked(bar, parity, 4000u)) { ok = true; break; }
+                if ((++spins & 255u) == 0) {
+                    if (*s_dead) break;
+                    const unsigned long long now = global_ns();
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > kCopyWaitNs) { *s_dead = 1u; *(volatile uint32_t*)a.status = (uint32_t)kDevCopyTimeout; break; }
                 }
             }
-            asm volatile("cp.async.commit_group;" ::: "memory");
-        };
-        auto item_size = [](const uint8_t* item) {
-            const uint4 hh = *reinterpret_cast<const uint4*>(item);
-            const int nk_ = (int)(hh.x & 0xffu), mr_ = (int)((hh.x >> 8) & 0xffu), RT_ = (int)((hh.x >> 16) & 0xffu), KT_ = (int)(hh.x >> 24);
-            return ((16 + ((nk_ + 3) & ~3) + ((mr_ + 3) & ~3) + 15) & ~15) + RT_ * KT_ * 256;
-        };
-        int buf = 0;
-        if (p < end) gather_async(p, 0);
+        }
+        return __all_sync(0xffffffffu, ok);          // the whole warp goes on, or none of it
+    };
+    // The tile this warp is at (tcur) sits in slot xs of the input ring, in the use of that slot with
+    // parity xpar; both move along with tcur, so nothing is divided.
+    int tcur = 0, xs = 0;
+    uint32_t xpar = 0u;
+    auto wait_x = [&]() -> bool { return wait_bar(&xfull[xs], xpar); };
+    // This warp is done with tile tcur; the last warp of the CTA to say so refills the slot.
+    auto release_x = [&]() {
+        __syncwarp();
+        uint32_t last = 0u;
+        // A plain (relaxed) add: the loads this warp made from the slot have all returned (the tensor
+        // instructions that used them have been issued), and a fence here would also wait for the
+        // weight copies this lane has in flight from HBM.
+        if (lane == 0) {
+            last = atomicAdd(&xcnt[xs], 1u) == (uint32_t)kSpmmWarps - 1u;
+            if (last) *reinterpret_cast<volatile uint32_t*>(&xcnt[xs]) = 0u;
+        }
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last && tcur + a.x_depth < ntiles) fetch_tile(xs, tcur + a.x_depth);
+        ++tcur;
+        if (++xs == a.x_depth) { xs = 0; xpar ^= 1u; }
+    };
+
+    float acc[MT][NT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0.f;
+
+    const uint32_t x_lane_off = (uint32_t)(lane >> 4) * 16u;                 // this lane's 16 bytes inside a tile row
+    const int kr_lane = ((lane >> 3) & 1) * 8 + (lane & 7);                  // its k row inside a 16-column slab
+    bool alive = true;
+    int s = 0;                                     // stage of this warp's weight ring, and the parity of its current use
+    uint32_t parity = 0u;
+    for (uint32_t c = 0; c < n_chunks && alive; ++c) {
+        SPMM_LAP(4);
+        if (!wait_bar(&wfull[s], parity)) { alive = false; break; }
+        SPMM_LAP(1);                               // waiting for weights
+        const uint8_t* p = wring + (size_t)s * kSpmmStageBytes;
+        const uint4 chh = *reinterpret_cast<const uint4*>(p);              // items' size, sizes of the next three chunks
+        const uint8_t* end = p + 16 + 16 * (size_t)chh.x;
+        const uint32_t refill_bytes = a.w_stages == 3 ? chh.w : chh.z;     // the chunk w_stages further on
+        p += 16;
         while (p < end) {
             const uint4 h = *reinterpret_cast<const uint4*>(p);
-            const int nk = (int)(h.x & 0xffu), mr = (int)((h.x >> 8) & 0xffu), RT = (int)((h.x >> 16) & 0xffu), KT = (int)(h.x >> 24);
+            const int tile = (int)(h.x & 0xffffu), nk = (int)((h.x >> 16) & 0xffu), np2 = (int)(h.x >> 24);
+            const uint32_t mask_lo = h.y, mask_hi = h.z;
             const uint8_t* cidx = p + 16;
-            const uint8_t* ridx = cidx + ((nk + 3) & ~3);
-            const uint8_t* tiles = p + ((16 + ((nk + 3) & ~3) + ((mr + 3) & ~3) + 15) & ~15);
-            p += item_size(p);
-            // the next item's inputs are fetched while this one is multiplied
-            if (p < end) {
-                gather_async(p, buf ^ 1);
-                asm volatile("cp.async.wait_group 1;" ::: "memory");
-            } else {
-                asm volatile("cp.async.wait_group 0;" ::: "memory");
+            const uint32_t vals = smem_u32(cidx + ((nk + 3) & ~3));
+            p += 16 * (size_t)(h.w & 0xffffu);
+            // tiles this warp has no block in are passed in order
+            SPMM_LAP(4);
+            while (tcur < tile && alive) {
+                if (!wait_x()) { alive = false; break; }
+                release_x();
             }
-            __syncwarp();
-            const uint8_t* xs_hi = xs_base + buf * kXBuf;
-            const uint8_t* xs_lo = xs_hi + kMmaMaxNk * kXRowBytes;
-            buf ^= 1;
-            // ---- multiply: D[16 kept rows x 8 batch] += A[16 x 8 kept columns] . B[8 x 8], four batch tiles
-            for (int rt = 0; rt < RT; ++rt) {
-                float acc[NT][4];
+            if (!alive || !wait_x()) { alive = false; break; }
+            SPMM_LAP(2);                           // passing tiles and waiting for this item's tile
+            const uint32_t xtile = smem_u32(xring + (size_t)xs * a.tile_bytes);
+            // address of this lane's words in the stored row behind each of its output rows (rows that are
+            // not kept have none).  Lane l works out where in-block rows l and l + 32 are stored (a
+            // population count on the row mask) and the lanes fetch what they need by shuffle.
+            uint32_t rowaddr[MT][2];
+            {
+                const uint32_t below = (1u << lane) - 1u;
+                const uint32_t e_lo = ((mask_lo >> lane) & 1u) ? (uint32_t)__popc(mask_lo & below) : 0xffffu;
+                const uint32_t e_hi = ((mask_hi >> lane) & 1u) ? (uint32_t)(__popc(mask_lo) + __popc(mask_hi & below)) : 0xffffu;
+                const uint32_t mine = e_lo | (e_hi << 16);
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt)
+                for (int q = 0; q < (MT < 2 ? MT : 2); ++q)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
-                const uint2* at = reinterpret_cast<const uint2*>(tiles + (size_t)rt * KT * 256) + lane;
-                for (int kt = 0; kt < KT; ++kt) {
-                    const uint2 af = at[kt * 32];
-                    // lane l hands ldmatrix the address of row (l % 8) of matrix (l / 8) = batch tile
-                    const int off = (kt * 8 + (lane & 7)) * kXRowBytes + (lane >> 3) * 16;
-                    uint32_t bh[4], bl[4];
-                    ldmatrix_x4_trans(bh, xs_hi + off);
-                    ldmatrix_x4_trans(bl, xs_lo + off);
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const uint32_t v = __shfl_sync(0xffffffffu, mine, 16 * q + g + 8 * hh);
+                        const uint32_t lo = v & 0xffffu, hi = v >> 16;
+                        rowaddr[q][hh] = lo != 0xffffu ? vals + (lo * (uint32_t)np2 + (uint32_t)t) * 4u : kNoRow;
+                        if (MT > 2) rowaddr[(q + 2) % MT][hh] = hi != 0xffffu ? vals + (hi * (uint32_t)np2 + (uint32_t)t) * 4u : kNoRow;
+                    }
+            }
+            for (int kb = 0; kb < nk; kb += 16) {
+                // ---- B operand: the gathered inputs, 16 kept columns x this warp's batch columns
+                const int kr = kb + kr_lane;
+                const uint32_t rowp = (kr < nk ? xtile + (uint32_t)cidx[kr] * (uint32_t)a.pitch : zero_addr) + x_lane_off;
+                uint32_t bh[NT][2], bl[NT][2];
+                if (NT == 1) {
+                    uint32_t r4[4];
+                    ldmatrix_x4_trans(r4, rowp);                       // (hi, k 0-7), (hi, k 8-15), (lo, k 0-7), (lo, k 8-15)
+                    bh[0][0] = r4[0]; bh[0][1] = r4[1]; bl[0][0] = r4[2]; bl[0][1] = r4[3];
+                } else {
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {          // batch tiles past NT hold zero columns: skipped
-                        mma_m16n8k8(acc[nt], af.x, af.y, bh[nt]);
-                        mma_m16n8k8(acc[nt], af.x, af.y, bl[nt]);
+                    for (int q = 0; q < NT / 2; ++q) {
+                        uint32_t r4[4];
+                        ldmatrix_x4_trans(r4, rowp + 32u * q);         // batch tiles 2q, 2q + 1 of the hi part
+                        bh[2 * q][0] = r4[0]; bh[2 * q][1] = r4[1]; bh[(2 * q + 1) % NT][0] = r4[2]; bh[(2 * q + 1) % NT][1] = r4[3];
+                        ldmatrix_x4_trans(r4, rowp + 16u * NT + 32u * q);   // the same of the lo part
+                        bl[2 * q][0] = r4[0]; bl[2 * q][1] = r4[1]; bl[(2 * q + 1) % NT][0] = r4[2]; bl[(2 * q + 1) % NT][1] = r4[3];
                     }
                 }
-                // ---- scatter-add through the row indices: this lane holds rows g, g + 8 of the tile,
-                // batch columns 2t, 2t + 1 of every batch tile
+                // ---- A operand: the kernel matrix with its rows at their RowIdx positions.  Words past the
+                // end of a stored row (last slab of a slice that is not a multiple of 16 wide) are zero.
+                const uint32_t koff = (uint32_t)kb * 2u;                             // bytes into a stored row
+                const bool v0 = (uint32_t)(kb >> 1) + (uint32_t)t < (uint32_t)np2, v1 = (uint32_t)(kb >> 1) + (uint32_t)t + 4u < (uint32_t)np2;
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const int r = rt * 16 + g + 8 * half;
-                    if (r < mr) {
-                        float* z = zs + (int)ridx[r] * kZStride + 2 * t;
+                for (int mt = 0; mt < MT; ++mt) {
+                    uint32_t af[4];
+                    af[0] = (rowaddr[mt][0] != kNoRow && v0) ? lds_u32(rowaddr[mt][0] + koff) : 0u;
+                    af[1] = (rowaddr[mt][1] != kNoRow && v0) ? lds_u32(rowaddr[mt][1] + koff) : 0u;
+                    af[2] = (rowaddr[mt][0] != kNoRow && v1) ? lds_u32(rowaddr[mt][0] + koff + 16u) : 0u;
+                    af[3] = (rowaddr[mt][1] != kNoRow && v1) ? lds_u32(rowaddr[mt][1] + koff + 16u) : 0u;
 #pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) {
-                            float2 cur2 = *reinterpret_cast<float2*>(z + nt * 8);
-                            cur2.x += acc[nt][2 * half]; cur2.y += acc[nt][2 * half + 1];
-                            *reinterpret_cast<float2*>(z + nt * 8) = cur2;
-                        }
+                    for (int nt = 0; nt < NT; ++nt) {
+                        mma_m16n8k16(acc[mt][nt], af, bh[nt][0], bh[nt][1]);
+                        mma_m16n8k16(acc[mt][nt], af, bl[nt][0], bl[nt][1]);
                     }
                 }
             }
-            __syncwarp();
         }
-        if (flush == kFlushCta) {
-            __syncthreads();
-            // the CTA owns this block-row: add the warps' private sums in warp order and store y
-            const int zbase = (int)chh.z;
-            const int nrows = min(a.block_r, a.rows - zbase);
-            for (int idx = threadIdx.x; idx < nrows * a.nb; idx += blockDim.x) {
-                const int b = idx / nrows, r = idx % nrows;
-                float sum = 0.f;
-                for (int w = 0; w < W; ++w) sum += zs_all[((size_t)w * a.block_r + r) * kZStride + b];
-                a.Y[(long long)b * a.ldy + zbase + r] = sum;
+        if (!alive) break;
+        SPMM_LAP(3);                               // row map, operand loads, tensor instructions
+        // this warp is done with the stage and refills it
+        __syncwarp();
+        if (refill_bytes) {
+            if (lane == 0) {
+                fence_proxy_async_all();
+                mbar_expect_tx(&wfull[s], refill_bytes);
+                bulk_g2s(wring + (size_t)s * kSpmmStageBytes, a.stream + (size_t)issue_off * 16, refill_bytes, &wfull[s]);
             }
-            __syncthreads();
-            for (int i = lane; i < a.block_r * kZStride; i += 32) zs[i] = 0.f;
-            __syncwarp();
+            issue_off += refill_bytes >> 4;
         }
-        if (lane == 0 && refill.bytes) {
-            mbar_expect_tx(&bars[s], refill.bytes);
-            bulk_g2s(ring + (size_t)s * a.stage_bytes, a.stream + (size_t)(refill.off16 & kOffMaskM) * 16, refill.bytes, &bars[s]);
-        }
-        cur = nxt;
+        if (++s == a.w_stages) { s = 0; parity ^= 1u; }
     }
-}
+    SPMM_LAP(4);                                   // ring bookkeeping
+    while (tcur < ntiles && alive) {
+        if (!wait_x()) { alive = false; break; }
+        release_x();
+    }
+    SPMM_LAP(5);                                   // the tiles behind this warp's last item
+    __syncthreads();
+    SPMM_LAP(6);                                   // waiting for the other warps of the CTA
+    if (*s_dead) {
+        // a wait gave up (the status word says so): give copies that may still be in flight a bounded
+        // time to land before the CTA's shared memory goes away, and write nothing
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+        return;
+    }
 
+    // ---- the warps' sums meet in shared memory (the rings are no longer in use)
+    constexpr int kP = NT * 8 + 1;                         // floats per row: odd, so that a column read is conflict-free
+    float* P = reinterpret_cast<float*>(smem + L.rings);
+    {
+        float* Pw = P + (size_t)warp * MT * 16 * kP;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                float* q = Pw + (16 * mt + g) * kP + 8 * nt + 2 * t;
+                q[0] = acc[mt][nt][0]; q[1] = acc[mt][nt][1];
+                q[8 * kP] = acc[mt][nt][2]; q[8 * kP + 1] = acc[mt][nt][3];
+            }
+    }
+    __syncthreads();
+    const int group_rows = a.RG * a.block_r, row0 = me->group * group_rows;
+    const int nrows = min(group_rows, a.rows - row0);
+    constexpr int cap = 8 * NT;
+    float* part = a.S > 1 ? a.partials + ((size_t)me->group * a.S + me->split) * cap * group_rows : nullptr;
+    {
+        // element idx = b * nrows + rloc, taken blockDim apart; (b, rloc, block-row, row in it) move along without a division
+        int b = 0, rloc = threadIdx.x;
+        while (rloc >= nrows) { rloc -= nrows; ++b; }
+        int rr = 0, r = rloc;
+        while (r >= a.block_r) { r -= a.block_r; ++rr; }
+        while (b < a.nb) {
+            float sum = 0.f;
+            for (int w = s_first[rr]; w < s_first[rr + 1]; ++w) sum += P[((size_t)w * MT * 16 + r) * kP + b];
+            if (part) part[(size_t)b * group_rows + rloc] = sum;
+            else a.Y[(long long)b * a.ldy + row0 + rloc] = sum;
+            rloc += blockDim.x;
+            while (rloc >= nrows) { rloc -= nrows; ++b; }
+            rr = 0; r = rloc;
+            while (r >= a.block_r) { r -= a.block_r; ++rr; }
+        }
+    }
+    if (part) {
+        // the last CTA of the row group to arrive adds the ranges' partial sums in range order
+        __shared__ uint32_t s_last;
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) s_last = atomicAdd(a.arrivals + me->group, 1u) == (uint32_t)a.S - 1u;
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            const float* base = a.partials + (size_t)me->group * a.S * cap * group_rows;
+            int b = 0, rloc = threadIdx.x;
+            while (rloc >= nrows) { rloc -= nrows; ++b; }
+            while (b < a.nb) {
+                float sum = 0.f;
+                for (int s2 = 0; s2 < a.S; ++s2) sum += __ldcg(base + ((size_t)s2 * cap + b) * group_rows + rloc);
+                a.Y[(long long)b * a.ldy + row0 + rloc] = sum;
+                rloc += blockDim.x;
+                while (rloc >= nrows) { rloc -= nrows; ++b; }
+            }
+            if (threadIdx.x == 0) a.arrivals[me->group] = 0u;
+        }
+    }
+    SPMM_LAP(7);                                   // sums of the warps, partial sums of the ranges, store
+#ifdef CSB_SPMM_CLOCKS
+    if (lane == 0) for (int i = 0; i < 8; ++i) a.clocks[((size_t)blockIdx.x * kSpmmWarps + warp) * 8 + i] = sprof[i];
+#endif
+}
 
 #define CSB_CUDA(call)                                                                     \
     do {                                                                                   \
@@ -251,7 +440,8 @@ __global__ void __launch_bounds__(256, 1) csb_spmm_mma_kernel(const MmaArgs a) {
 
 bool spmm_mma_applicable(const csb_matrix* A, int batch) {
     if (getenv("CSB_NO_MMA") && atoi(getenv("CSB_NO_MMA"))) return false;
-    return batch >= 8 && A->val_dtype == CSB_F16 && A->block_r <= 64 && A->device >= 0 && !(A->mma && A->mma->unusable);
+    if (!(batch >= 8 && A->val_dtype == CSB_F16 && A->block_r <= 64 && A->device >= 0)) return false;
+    return !(A->mma && A->mma->cls[spmm_class_index(batch)].unusable);
 }
 
 template <typename V>
@@ -262,30 +452,54 @@ static int upload_v(const std::vector<V>& h, V** d) {
     return CSB_OK;
 }
 
-static int build_mma_plan(const csb_matrix* A, MmaPlan* P) {
-    P->warps = 8; P->stage_bytes = 4096; P->stages = 2;
-    const int ctas = A->opts.ctas > 0 ? A->opts.ctas : A->sm_count;
-    const MmaSmem L(P->warps, P->stages, P->stage_bytes, A->block_r);
-    if (L.total > A->smem_optin) { P->unusable = true; return CSB_OK; }
-    MmaHostPlan H;
-    int rc = plan_mma_host(A, ctas, P->warps, P->stage_bytes, &H);
+static int mt_of(const csb_matrix* A) { return A->block_r <= 16 ? 1 : A->block_r <= 32 ? 2 : 4; }
+
+template <int MT, int NT>
+static cudaError_t set_smem_attr(size_t bytes) {
+    return cudaFuncSetAttribute(csb_spmm_tile_kernel<MT, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+template <int MT, int NT>
+static cudaError_t launch_tile_kernel(const cudaLaunchConfig_t* cfg, const SpmmArgs& a) {
+    return cudaLaunchKernelEx(cfg, csb_spmm_tile_kernel<MT, NT>, a);
+}
+#define CSB_SPMM_DISPATCH(fn, MT, NT, ...)                                                                        \
+    ((MT) == 1 ? ((NT) == 1 ? fn<1, 1>(__VA_ARGS__) : (NT) == 2 ? fn<1, 2>(__VA_ARGS__) : fn<1, 4>(__VA_ARGS__))  \
+     : (MT) == 2 ? ((NT) == 1 ? fn<2, 1>(__VA_ARGS__) : (NT) == 2 ? fn<2, 2>(__VA_ARGS__) : fn<2, 4>(__VA_ARGS__)) \
+                 : ((NT) == 1 ? fn<4, 1>(__VA_ARGS__) : (NT) == 2 ? fn<4, 2>(__VA_ARGS__) : fn<4, 4>(__VA_ARGS__)))
+
+static int build_spmm_plan(const csb_matrix* A, int ci, MmaPlan::PerClass* P) {
+    const int NT = 1 << ci;
+    SpmmHostPlan H;
+    const int sms = A->opts.ctas > 0 ? A->opts.ctas : A->sm_count;
+    int rc = plan_spmm_host(A, NT, sms, &H);
+    if (rc == 1) { P->unusable = true; return CSB_OK; }
     if (rc != CSB_OK) return rc;
-    if (H.max_chunk_bytes > (size_t)P->stage_bytes) { P->unusable = true; return CSB_OK; }
-    P->ctas = H.ctas; P->n_warps = H.ctas * H.warps_per_cta; P->balance = H.balance;
+    const int MT = mt_of(A), pitch = spmm_pitch(NT);
+    const int tile_bytes = (A->block_c * pitch + 127) & ~127;
+    // rings: as many weight stages (3, else 2) and input tiles (up to 8, at least 2) as shared memory holds
+    int w_stages = 0, x_depth = 0;
+    size_t smem = 0;
+    for (int ws = 3; ws >= 2 && !x_depth; --ws)
+        for (int xd = std::min(8, std::max(2, H.max_tiles)); xd >= 2; --xd) {
+            const SpmmSmem L(spmm_warps(NT), ws, xd, tile_bytes, pitch, MT, NT);
+            if (L.total <= A->smem_optin) { w_stages = ws; x_depth = xd; smem = L.total; break; }
+        }
+    if (!x_depth) { P->unusable = true; return CSB_OK; }
+    P->RG = H.RG; P->S = H.S; P->n_ctas = (int)H.ctas.size(); P->n_groups = H.n_groups;
+    P->w_stages = w_stages; P->x_depth = x_depth; P->smem_bytes = smem; P->balance = H.balance; P->warp_balance = H.warp_balance;
     P->stream_bytes = (int64_t)H.bytes.size();
-    std::vector<uint4> wdesc(P->n_warps);
-    for (int w = 0; w < P->n_warps; ++w) {
-        const uint32_t c0 = H.warp_chunk_begin[w], c1 = H.warp_chunk_begin[w + 1];
-        wdesc[w] = make_uint4(c0, c1, c0 < c1 ? H.chunks[c0].off16 : 0u, c0 < c1 ? H.chunks[c0].bytes : 0u);
-    }
     if ((rc = upload_v(H.bytes, &P->d_stream)) != CSB_OK) return rc;
-    if ((rc = upload_v(H.chunks, &P->d_chunks)) != CSB_OK) return rc;
-    if ((rc = upload_v(wdesc, (uint4**)&P->d_warp_desc)) != CSB_OK) return rc;
-    P->xp_bytes = (size_t)A->cols * 64 * sizeof(__half);
-    CSB_CUDA(cudaMalloc(&P->d_xp, P->xp_bytes));
-    CSB_CUDA(cudaFuncSetAttribute(csb_spmm_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
-    CSB_CUDA(cudaFuncSetAttribute(csb_spmm_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
-    CSB_CUDA(cudaFuncSetAttribute(csb_spmm_mma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
+    if ((rc = upload_v(H.warp_desc, &P->d_warp_desc)) != CSB_OK) return rc;
+    if ((rc = upload_v(H.ctas, &P->d_ctas)) != CSB_OK) return rc;
+    const size_t xp_bytes = (size_t)A->nbc * A->block_c * pitch;          // whole tiles, so that a tile copy never runs past the end
+    CSB_CUDA(cudaMalloc(&P->d_xp, xp_bytes));
+    CSB_CUDA(cudaMemset(P->d_xp, 0, xp_bytes));
+    if (H.S > 1) {
+        CSB_CUDA(cudaMalloc((void**)&P->d_partials, (size_t)H.n_groups * H.S * 8 * NT * H.RG * A->block_r * 4));
+        CSB_CUDA(cudaMalloc((void**)&P->d_arrivals, (size_t)H.n_groups * 4));
+        CSB_CUDA(cudaMemset(P->d_arrivals, 0, (size_t)H.n_groups * 4));
+    }
+    CSB_CUDA(CSB_SPMM_DISPATCH(set_smem_attr, MT, NT, smem));
     CSB_CUDA(cudaDeviceSynchronize());
     P->built = true;
     return CSB_OK;
@@ -296,13 +510,25 @@ void free_mma(csb_matrix* A) {
     int prev = 0;
     cudaGetDevice(&prev);
     cudaSetDevice(A->device);
-    cudaFree(A->mma->d_stream); cudaFree(A->mma->d_chunks); cudaFree(A->mma->d_warp_desc); cudaFree(A->mma->d_xp);
+    for (auto& c : A->mma->cls) {
+        cudaFree(c.d_stream); cudaFree(c.d_warp_desc); cudaFree(c.d_ctas);
+        cudaFree(c.d_partials); cudaFree(c.d_arrivals); cudaFree(c.d_xp);
+    }
     cudaSetDevice(prev);
     delete A->mma;
     A->mma = nullptr;
 }
 
-// Returns CSB_OK after launching, or kMmaNotUsed (1) when the caller should use the CUDA-core path.
+#ifdef CSB_SPMM_CLOCKS
+static long long* g_spmm_clocks = nullptr;
+static int g_spmm_clock_warps = 0;
+extern "C" int csb_debug_spmm_clocks(long long* host_out, int max_warps) {
+    cudaMemcpy(host_out, g_spmm_clocks, (size_t)std::min(max_warps, g_spmm_clock_warps) * 8 * 8, cudaMemcpyDeviceToHost);
+    return g_spmm_clock_warps;
+}
+#endif
+
+// Returns CSB_OK after launching, or 1 when the caller should use the CUDA-core path.
 int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream) {
     const ProductPlan& PP = A->product;
     if (PP.h_status && *PP.h_status != 0) { set_error("an earlier product on this handle gave up waiting on the device (code %u)", *PP.h_status); return CSB_ERR_TIMEOUT; }
@@ -310,44 +536,89 @@ int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch,
     CSB_CUDA(cudaGetDevice(&prev));
     if (prev != A->device) CSB_CUDA(cudaSetDevice(A->device));
     struct Restore { int prev, cur; ~Restore() { if (prev != cur) cudaSetDevice(prev); } } restore{prev, A->device};
+    const int ci = spmm_class_index(batch);
     {
         std::lock_guard<std::mutex> lk(A->mma_mu);
         if (!A->mma) {
             A->mma = new (std::nothrow) MmaPlan();
             if (!A->mma) { set_error("out of host memory"); return CSB_ERR_ALLOC; }
+        }
+        MmaPlan::PerClass& C = A->mma->cls[ci];
+        if (!C.built && !C.unusable) {
             int rc;
-            try { rc = build_mma_plan(A, A->mma); }
+            try { rc = build_spmm_plan(A, ci, &C); }
             catch (const std::bad_alloc&) { set_error("out of host memory while planning the batched product"); rc = CSB_ERR_ALLOC; }
-            if (rc != CSB_OK) { A->mma->unusable = true; return rc; }
+            if (rc != CSB_OK) { C.unusable = true; return rc; }
         }
     }
-    const MmaPlan& P = *A->mma;
+    const MmaPlan::PerClass& P = A->mma->cls[ci];
     if (P.unusable || !P.built) return 1;
+    const int NT = 1 << ci, MT = mt_of(A), cap = 8 * NT;
     cudaStream_t st = (cudaStream_t)stream;
-    const MmaSmem L(P.warps, P.stages, P.stage_bytes, A->block_r);
-    MmaArgs a{};
-    a.stream = P.d_stream; a.chunks = P.d_chunks; a.warp_desc = (const uint4*)P.d_warp_desc; a.xp = (const __half*)P.d_xp;
-    a.ldy = ldy; a.status = PP.d_status; a.n_warps = P.n_warps; a.rows = (int)A->rows; a.block_r = A->block_r;
-    a.stage_bytes = P.stage_bytes; a.stages = P.stages;
-    for (int b0 = 0; b0 < batch; b0 += kSlab) {
-        a.nb = std::min(kSlab, batch - b0);
+    SpmmArgs a{};
+    a.stream = P.d_stream; a.warp_desc = (const uint4*)P.d_warp_desc; a.ctas = P.d_ctas;
+    a.xp = (const uint8_t*)P.d_xp; a.ldy = ldy; a.partials = P.d_partials; a.arrivals = P.d_arrivals; a.status = PP.d_status;
+    a.rows = (int)A->rows; a.cols = (int)A->cols; a.block_r = A->block_r; a.block_c = A->block_c;
+    a.RG = P.RG; a.S = P.S; a.x_depth = P.x_depth; a.w_stages = P.w_stages;
+    a.pitch = spmm_pitch(NT); a.tile_bytes = (A->block_c * a.pitch + 127) & ~127;
+#ifdef CSB_SPMM_CLOCKS
+    if (!g_spmm_clocks) cudaMalloc((void**)&g_spmm_clocks, (size_t)1 << 24);
+    a.clocks = g_spmm_clocks;
+    g_spmm_clock_warps = P.n_ctas * spmm_warps(NT);
+#endif
+    for (int b0 = 0; b0 < batch; b0 += cap) {
+        a.nb = std::min(cap, batch - b0);
         a.Y = Y + (int64_t)b0 * ldy;
-        // both kernels order themselves behind the work in front (pdl_wait at their top), so they may
-        // be launched with programmatic stream serialization: their scheduling overlaps its tail
+        // both kernels order themselves behind the work in front (pdl_wait), so they may be launched
+        // with programmatic stream serialization: their scheduling overlaps its tail
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cudaLaunchConfig_t cfg{};
         cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 1;
-        cfg.gridDim = dim3((unsigned)((A->cols + 7) / 8)); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0;
-        CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_pack_x_kernel, X + (int64_t)b0 * ldx, (long long)ldx, a.nb, (int)A->cols, (__half*)P.d_xp));
-        cfg.gridDim = dim3((unsigned)P.ctas); cfg.blockDim = dim3((unsigned)P.warps * 32u); cfg.dynamicSmemBytes = L.total;
-        if (a.nb <= 8) CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_spmm_mma_kernel<1>, a));
-        else if (a.nb <= 16) CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_spmm_mma_kernel<2>, a));
-        else CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_spmm_mma_kernel<4>, a));
+        cfg.gridDim = dim3((unsigned)((A->cols + 31) / 32)); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0;
+        CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_pack_x_kernel, X + (int64_t)b0 * ldx, (long long)ldx, a.nb, (int)A->cols, (uint8_t*)P.d_xp,
+                                    a.pitch, NT));
+        cfg.gridDim = dim3((unsigned)P.n_ctas); cfg.blockDim = dim3((unsigned)spmm_warps(NT) * 32u); cfg.dynamicSmemBytes = P.smem_bytes;
+        CSB_CUDA(CSB_SPMM_DISPATCH(launch_tile_kernel, MT, NT, &cfg, a));
         CSB_CUDA(cudaGetLastError());
     }
     return CSB_OK;
 }
 
 }  // namespace csb
+
+// Inspection / testing aid: the plan of the batched product, made on the host only.
+extern "C" int csb_spmm_plan_dump(const csb_matrix_t* A, int batch, int sm_count, int64_t* info_out, uint8_t* stream_out, int64_t stream_cap,
+                                  uint32_t* chunks_out, int64_t chunks_cap, uint32_t* stream_begin_out, int64_t begin_cap, int32_t* cta_out,
+                                  int64_t cta_cap) {
+    using namespace csb;
+    clear_error();
+    if (!A || !info_out || batch < 1 || sm_count < 1) { set_error("csb_spmm_plan_dump: bad argument"); return CSB_ERR_INVALID_ARG; }
+    SpmmHostPlan H;
+    int rc;
+    try { rc = plan_spmm_host(A, spmm_nt(batch), sm_count, &H); }
+    catch (const std::bad_alloc&) { set_error("out of host memory while planning"); return CSB_ERR_ALLOC; }
+    if (rc == 1) { set_error("the tensor-core layout does not apply to this matrix (fp16 values, block_r <= 64)"); return CSB_ERR_UNSUPPORTED; }
+    if (rc != CSB_OK) return rc;
+    info_out[0] = (int64_t)H.ctas.size(); info_out[1] = (int64_t)H.chunks.size(); info_out[2] = (int64_t)H.bytes.size();
+    info_out[3] = H.RG; info_out[4] = spmm_nt(batch) | (spmm_warps(spmm_nt(batch)) << 8); info_out[5] = H.S; info_out[6] = (int64_t)(H.warp_balance * 1e6);
+    info_out[7] = (int64_t)(H.balance * 1e6);
+    if (stream_out) {
+        if (stream_cap < (int64_t)H.bytes.size()) { set_error("stream buffer too small"); return CSB_ERR_INVALID_ARG; }
+        std::memcpy(stream_out, H.bytes.data(), H.bytes.size());
+    }
+    if (chunks_out) {
+        if (chunks_cap < (int64_t)H.chunks.size()) { set_error("chunk buffer too small"); return CSB_ERR_INVALID_ARG; }
+        for (size_t i = 0; i < H.chunks.size(); ++i) { chunks_out[2 * i] = H.chunks[i].off16; chunks_out[2 * i + 1] = H.chunks[i].bytes; }
+    }
+    if (stream_begin_out) {
+        if (begin_cap < (int64_t)H.stream_begin.size()) { set_error("stream table too small"); return CSB_ERR_INVALID_ARG; }
+        for (size_t i = 0; i < H.stream_begin.size(); ++i) stream_begin_out[i] = H.stream_begin[i];
+    }
+    if (cta_out) {
+        if (cta_cap < (int64_t)H.ctas.size()) { set_error("CTA table too small"); return CSB_ERR_INVALID_ARG; }
+        std::memcpy(cta_out, H.ctas.data(), H.ctas.size() * sizeof(SpmmCta));
+    }
+    return CSB_OK;
+}

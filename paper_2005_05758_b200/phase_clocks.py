@@ -2,12 +2,15 @@
 
     python -m paper_2005_05758_b200.phase_clocks rnn   [cfg1 cfg2 cfg3 cfg5]
     python -m paper_2005_05758_b200.phase_clocks panel [4 8 16 25]
+    python -m paper_2005_05758_b200.phase_clocks spmm  [rate:batch ...]      (default 4:8 4:32 25:8)
 
 Builds libcsb_clocks.so beside the normal library with -DCSB_PHASE_CLOCKS -DCSB_PANEL_CLOCKS (see
 build.py), loads it instead of libcsb.so and prints
   rnn:   cycles per timestep and phase of csb_rnn_kernel, summed by thread 0 of every CTA
          (mean / min / max over the CTAs);
-  panel: wall-clock stamps of csb_panel_kernel per CTA, in microseconds from the earliest CTA start.
+  panel: wall-clock stamps of csb_panel_kernel per CTA, in microseconds from the earliest CTA start;
+  spmm:  cycles per phase of csb_spmm_tile_kernel, summed per warp (mean / max over the warps, and the
+         same for the slowest CTA).
 The instrumented kernels are slower than the product ones (thread 0 reads the clock between phases),
 so these figures say where the time goes, never how long a call takes.
 """
@@ -93,6 +96,38 @@ def panel(rates):
         A.free()
 
 
+SPMM_PHASES = ["set-up, first copies, wait for the work in front", "waiting for weights", "passing tiles, waiting for the item's tile",
+               "row map, operand loads, tensor instructions", "ring bookkeeping, item headers", "tiles behind the last item",
+               "waiting for the CTA's other warps", "warp sums, range sums, store"]
+
+
+def spmm(cases):
+    import workloads
+    torch, binding = _load()
+    for case in cases:
+        rate, B = case.split(":")
+        w = workloads.CONFIGS["cfg4"](rate=float(rate), B=int(B))
+        m = w.matrix
+        As = [binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, 0) for _ in range(3)]
+        X = torch.from_numpy(w.X).cuda()
+        Y = torch.empty((int(B), m.rows), device="cuda")
+        for i in range(6):
+            binding.csb_spmm(As[i % 3], X, Y)
+            torch.cuda.synchronize()
+        ck = np.zeros((1 << 16, 8), np.int64)
+        n = binding.lib.csb_debug_spmm_clocks(C.c_void_p(ck.ctypes.data), 1 << 16)
+        ck = ck[:n].astype(np.float64)
+        wpc = 32 if int(B) <= 8 else 16
+        per_cta = ck.reshape(-1, wpc, 8)
+        slow = per_cta[np.argmax(per_cta.sum(axis=2).max(axis=1))]
+        print("cfg4 rate %sx batch %s: %d warps (%d per CTA); cycles per phase, last pass of 32 batch columns" % (rate, B, n, wpc))
+        for i, nm in enumerate(SPMM_PHASES):
+            print("   %-52s mean %8.0f  max %8.0f   slowest CTA: mean %8.0f  max %8.0f" % (nm, ck[:, i].mean(), ck[:, i].max(), slow[:, i].mean(), slow[:, i].max()))
+        print("   %-52s mean %8.0f  max %8.0f" % ("all phases", ck.sum(axis=1).mean(), ck.sum(axis=1).max()))
+        for a in As:
+            a.free()
+
+
 if __name__ == "__main__":
     what = sys.argv[1] if len(sys.argv) > 1 else "rnn"
     rest = sys.argv[2:]
@@ -100,5 +135,7 @@ if __name__ == "__main__":
         rnn(rest or ["cfg1", "cfg2", "cfg3", "cfg5"])
     elif what == "panel":
         panel(rest or ["4", "25"])
+    elif what == "spmm":
+        spmm(rest or ["4:8", "4:32", "25:8"])
     else:
         raise SystemExit(__doc__)
