@@ -321,16 +321,17 @@ int csb_panel_dump(const csb_matrix_t* A, int ctas, int warps_per_cta, int stage
  * 16), each working for one block-row of the group; S CTAs share a row group.  Weight stream
  * cta * W + w belongs to warp w.
  *   info_out          host, int64[8]: CTAs, chunks, stream bytes, RG, 8-column batch tiles per warp
- *                     + 256 * W, S, and the warp-level and CTA-level balance (mean / max of the
- *                     modelled cost) times 1e6.
+ *                     + 256 * W + 65536 * G (an input tile spans G block-columns), S, and the
+ *                     warp-level and CTA-level balance (mean / max of the modelled cost) times 1e6.
  *   stream_out        host, `stream_cap` bytes, or NULL;  chunks_out  host, uint32 pairs (offset in
  *                     16-byte units, bytes), or NULL;  stream_begin_out  host, uint32 first chunk of
  *                     every weight stream plus one end entry, or NULL;  cta_out  host, 48 bytes per
- *                     CTA (int32 row group, range number, first block-column, block-columns, then
+ *                     CTA (int32 row group, range number, first block-column, input tiles, then
  *                     32 bytes: the block-row of the group each warp works for), `cta_cap` CTAs, or NULL.
  * A chunk is 16 bytes (first word: size of what follows in 16-byte units) followed by items; an
- * item is 16 bytes (u16 block-column counted from the CTA's first, u8 kept columns nk, u8 words
+ * item is 16 bytes (u16 input tile counted from the CTA's first, u8 kept columns nk, u8 words
  * per stored row, u64 mask of the kept in-block rows, u16 size in 16-byte units), nk column indices
+ * inside the input tile (block-column inside the tile times block_c plus the in-block index)
  * padded to 4 bytes, and the kept rows of the column slice, row-major, each padded to an even
  * number of halves.
  * Errors: UNSUPPORTED when the layout does not apply (fp32 values, block_r > 64), INVALID_ARG for a

@@ -182,7 +182,7 @@ def csb_spmm_plan_dump(A: CsbMatrix, batch: int, sm_count: int) -> dict:
     info = np.zeros(8, np.int64)
     _check(lib.csb_spmm_plan_dump(A.handle, batch, sm_count, info.ctypes.data, None, 0, None, 0, None, 0, None, 0))
     n_ctas, n_chunks, n_bytes = (int(v) for v in info[:3])
-    NT, warps = int(info[4]) & 255, int(info[4]) >> 8
+    NT, warps, tile_blocks = int(info[4]) & 255, (int(info[4]) >> 8) & 255, int(info[4]) >> 16
     stream = np.zeros(max(n_bytes, 1), np.uint8)
     chunks = np.zeros((max(n_chunks, 1), 2), np.uint32)
     begin = np.zeros(n_ctas * warps + 1, np.uint32)
@@ -190,7 +190,7 @@ def csb_spmm_plan_dump(A: CsbMatrix, batch: int, sm_count: int) -> dict:
     _check(lib.csb_spmm_plan_dump(A.handle, batch, sm_count, info.ctypes.data, stream.ctypes.data, stream.size, chunks.ctypes.data,
                                   chunks.shape[0], begin.ctypes.data, begin.size, cta.ctypes.data, cta.shape[0]))
     cta = cta[:n_ctas]
-    return {"ctas": n_ctas, "RG": int(info[3]), "NT": NT, "warps": warps, "S": int(info[5]), "warp_balance": info[6] / 1e6,
+    return {"ctas": n_ctas, "RG": int(info[3]), "NT": NT, "warps": warps, "tile_blocks": tile_blocks, "S": int(info[5]), "warp_balance": info[6] / 1e6,
             "balance": info[7] / 1e6, "stream": stream[:n_bytes], "chunk_table": chunks[:n_chunks], "stream_begin": begin,
             "cta": cta[:, :16].copy().view(np.int32).reshape(n_ctas, 4), "warp_row": cta[:, 16:16 + warps].copy()}
 

@@ -2,6 +2,7 @@
 // planner, launch glue).  Nothing here is part of the public C ABI.
 #pragma once
 
+#include <algorithm>
 #include <cstdint>
 #include <cstring>
 #include <mutex>
@@ -204,13 +205,13 @@ int plan_rnn_host(int gates, int n_layers, const csb_matrix* const* Wm, const in
 // least work so far.  A warp's weights come through its own ring of bulk copies as items; the batch
 // of inputs comes through one ring of block-column tiles shared by the CTA.  An item is a column
 // slice (<= 64 kept columns) of one block:
-//   SpmmItemHeader (16 B), col_idx[nk] (in-block column indices, padded to 4 B), then the kernel
+//   SpmmItemHeader (16 B), col_idx[nk] (column indices inside the input tile, padded to 4 B), then the kernel
 //   matrix rows of the slice, row-major, each padded to an even number of halves (np2 words).
 // Items travel in chunks of at most kSpmmStageBytes; the chunks of a warp lie back to back, and a
 // chunk's 16-byte header holds the size of its items (16-byte units) and the byte sizes of the next
 // three chunks of the warp, so that a warp refills its ring without looking anything up in global memory.
 struct SpmmItemHeader {
-    uint16_t tile;            // block-column, counted from the CTA's first one
+    uint16_t tile;            // input tile (spmm_tile_blocks block-columns), counted from the CTA's first one
     uint8_t nk;               // kept columns in this item, 1..64
     uint8_t np2;              // 32-bit words per stored row, ceil(nk / 2)
     uint32_t mask_lo, mask_hi;   // bit r: in-block row r is kept in this block
@@ -220,7 +221,7 @@ struct SpmmItemHeader {
 static_assert(sizeof(SpmmItemHeader) == 16, "header is one 16-byte word");
 enum { kSpmmStageBytes = 2304, kSpmmMaxWarps = 32 };
 struct SpmmCta {
-    int32_t group, split, tile0, ntiles;     // row group, which column range of it, the range in block-columns
+    int32_t group, split, tile0, ntiles;     // row group, which column range of it, its first block-column, its input tiles
     uint8_t warp_row[kSpmmMaxWarps];         // which block-row of the group each warp works for (ascending)
 };
 static_assert(sizeof(SpmmCta) == 48, "three 16-byte words");
@@ -231,6 +232,9 @@ inline int spmm_warps(int NT) { return NT == 1 ? 32 : 16; }
 inline int spmm_nt(int batch) { return batch <= 8 ? 1 : batch <= 16 ? 2 : 4; }
 inline int spmm_class_index(int batch) { return batch <= 8 ? 0 : batch <= 16 ? 1 : 2; }
 inline int spmm_pitch(int NT) { return NT * 32 + 16; }   // bytes of one packed input column: hi parts, lo parts, 16 spare
+// An input tile of the shared ring spans this many block-columns (at most 256 matrix columns, so that a
+// column index inside a tile is one byte): fewer, larger tiles mean fewer hand-overs between the warps.
+inline int spmm_tile_blocks(int block_c) { return block_c >= 256 ? 1 : std::min(4, 256 / block_c); }
 struct SpmmHostPlan {
     std::vector<uint8_t> bytes;               // all chunks back to back
     std::vector<Chunk> chunks;

@@ -15,10 +15,8 @@
 //   * The inputs are packed once per call into binary16 pairs x = hi + lo (no input precision is
 //     lost as long as |x| < 65504), one row of batch values per matrix column, and reach shared
 //     memory as whole block-column tiles through a ring that all warps of the CTA share, so a tile
-//     is fetched from L2 once per CTA and not once per block.  The tiles come in by cp.async (16-byte
-//     pieces through the load/store path, completion counted on an mbarrier), not by bulk copy: bulk
-//     copies of one SM complete in order, and a tile queued behind the weight copies, which wait for
-//     HBM, reached shared memory a microsecond late every time.  The gather through ColIdx is done by
+//     is fetched from L2 once per CTA and not once per block.  A tile spans up to four block-columns
+//     (256 matrix columns), so that the warps hand tiles over a few times per CTA only.  The gather through ColIdx is done by
 //     the operand load itself: every lane hands ldmatrix.trans the address of the tile row of one
 //     kept column.  hi and lo are multiplied separately into the same accumulators.
 //   * The weights of a warp come through its own ring of bulk copies, so warps with light and heavy
@@ -51,7 +49,7 @@ struct SpmmArgs {
     float* partials;           // [group][range][8 * NT][RG * block_r], S > 1 only
     uint32_t* arrivals;        // [group], zero between launches
     uint32_t* status;
-    int nb, rows, cols, block_r, block_c, RG, S, x_depth, w_stages, pitch, tile_bytes;
+    int nb, rows, cols, block_r, block_c, tile_cols, RG, S, x_depth, w_stages, pitch, tile_bytes;   // tile_cols: matrix columns per input tile
 #ifdef CSB_SPMM_CLOCKS
     long long* clocks;         // instrumented build only: [CTA][warp][8] cycles per phase
 #endif
@@ -152,20 +150,18 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     if (threadIdx.x < sizeof(SpmmCta) / 4) reinterpret_cast<uint32_t*>(&s_me)[threadIdx.x] = reinterpret_cast<const uint32_t*>(a.ctas + blockIdx.x)[threadIdx.x];
     const uint4 wd = __ldg(a.warp_desc + (size_t)blockIdx.x * kSpmmWarps + warp);
     const uint32_t n_chunks = wd.y;
-    __syncthreads();
-    const SpmmCta* me = &s_me;
-    const int ntiles = me->ntiles, tile0 = me->tile0;
-    auto tile_bytes_of = [&](int tl) { return (uint32_t)min(a.block_c, a.cols - (tile0 + tl) * a.block_c) * (uint32_t)a.pitch; };
-    auto tile_src = [&](int tl) { return a.xp + (size_t)(tile0 + tl) * a.block_c * a.pitch; };
-
     if (threadIdx.x == 0) {
         for (int i = 0; i < kSpmmWarps * a.w_stages; ++i) mbar_init(reinterpret_cast<uint64_t*>(smem + L.wfull) + i, 1);
-        for (int i = 0; i < a.x_depth; ++i) { mbar_init(&xfull[i], 32); xcnt[i] = 0u; }    // one arrival per lane of the warp that fetches a tile
+        for (int i = 0; i < a.x_depth; ++i) { mbar_init(&xfull[i], 1); xcnt[i] = 0u; }
         *s_dead = 0u;
         mbar_fence_init();
     }
     for (int i = threadIdx.x; i < (a.pitch + 16) / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem + L.zero)[i] = 0u;
     __syncthreads();
+    const SpmmCta* me = &s_me;
+    const int ntiles = me->ntiles, tile0 = me->tile0;
+    auto tile_bytes_of = [&](int tl) { return (uint32_t)min(a.tile_cols, a.cols - (tile0 * a.block_c + tl * a.tile_cols)) * (uint32_t)a.pitch; };
+    auto tile_src = [&](int tl) { return a.xp + (size_t)(tile0 * a.block_c + tl * a.tile_cols) * a.pitch; };
     // the weights were written at plan time: their first copies go out before the work in front is waited for
     // (a warp's chunks lie back to back; issue_off is where the next one to be fetched starts)
     uint32_t issue_off = wd.x;
@@ -187,18 +183,16 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
         while (rr < 4) s_first[++rr] = kSpmmWarps;
     }
     pdl_wait();                                    // the packed inputs and Y belong to the work in front on the stream
-    // One warp fetches a tile: every lane copies its 16-byte pieces and then arrives on the slot's
-    // barrier, the arrival taking effect when the lane's copies have landed.
+    // One lane fetches a tile with one bulk copy.  (No proxy fence in front of a refill: the slot's
+    // readers have their data in registers by the time they release it, and the release orders them
+    // before this copy is issued.)
     auto fetch_tile = [&](int slot, int tl) {
-        const uint32_t bytes = tile_bytes_of(tl);
-        const uint8_t* src = tile_src(tl);
-        const uint32_t dst = smem_u32(xring + (size_t)slot * a.tile_bytes);
-        for (uint32_t off = (uint32_t)lane * 16u; off < bytes; off += 512u)
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + off), "l"(src + off) : "memory");
-        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&xfull[slot])) : "memory");
+        if (lane == 0) {
+            mbar_expect_tx(&xfull[slot], tile_bytes_of(tl));
+            bulk_g2s(xring + (size_t)slot * a.tile_bytes, tile_src(tl), tile_bytes_of(tl), &xfull[slot]);
+        }
     };
-    if (warp == 0)
-        for (int tl = 0; tl < a.x_depth && tl < ntiles; ++tl) fetch_tile(tl, tl);
+    if (warp < a.x_depth && warp < ntiles) fetch_tile(warp, warp);          // the first tiles, one warp each
     SPMM_LAP(0);                                   // set-up, first copies out, the work in front waited for
     // A wait gives up after a second, or as soon as any warp of the CTA has given up.
     auto wait_bar = [&](uint64_t* bar, uint32_t parity) -> bool {
@@ -334,14 +328,13 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
                     }
                 }
             }
+            SPMM_LAP(3);                           // row map, operand loads, tensor instructions
         }
         if (!alive) break;
-        SPMM_LAP(3);                               // row map, operand loads, tensor instructions
         // this warp is done with the stage and refills it
         __syncwarp();
         if (refill_bytes) {
             if (lane == 0) {
-                fence_proxy_async_all();
                 mbar_expect_tx(&wfull[s], refill_bytes);
                 bulk_g2s(wring + (size_t)s * kSpmmStageBytes, a.stream + (size_t)issue_off * 16, refill_bytes, &wfull[s]);
             }
@@ -385,20 +378,35 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     constexpr int cap = 8 * NT;
     float* part = a.S > 1 ? a.partials + ((size_t)me->group * a.S + me->split) * cap * group_rows : nullptr;
     {
-        // element idx = b * nrows + rloc, taken blockDim apart; (b, rloc, block-row, row in it) move along without a division
-        int b = 0, rloc = threadIdx.x;
-        while (rloc >= nrows) { rloc -= nrows; ++b; }
-        int rr = 0, r = rloc;
-        while (r >= a.block_r) { r -= a.block_r; ++rr; }
-        while (b < a.nb) {
-            float sum = 0.f;
-            for (int w = s_first[rr]; w < s_first[rr + 1]; ++w) sum += P[((size_t)w * MT * 16 + r) * kP + b];
-            if (part) part[(size_t)b * group_rows + rloc] = sum;
-            else a.Y[(long long)b * a.ldy + row0 + rloc] = sum;
-            rloc += blockDim.x;
-            while (rloc >= nrows) { rloc -= nrows; ++b; }
-            rr = 0; r = rloc;
-            while (r >= a.block_r) { r -= a.block_r; ++rr; }
+        // four outputs per thread at a time; the warps of a block-row are added in warp order
+        const int total = nrows * a.nb;
+        for (int i0 = threadIdx.x; i0 < total; i0 += 4 * blockDim.x) {
+            int bb[4], rl[4], w0[4], w1[4], rin[4];
+            float sum[4];
+            int wmax = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int idx = min(i0 + j * (int)blockDim.x, total - 1);
+                bb[j] = idx / nrows; rl[j] = idx - bb[j] * nrows;
+                const int rr = rl[j] / a.block_r;
+                rin[j] = rl[j] - rr * a.block_r;
+                w0[j] = s_first[rr]; w1[j] = s_first[rr + 1];
+                wmax = max(wmax, w1[j] - w0[j]);
+                sum[j] = 0.f;
+            }
+            for (int k = 0; k < wmax; ++k) {
+                float v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[j] = w0[j] + k < w1[j] ? P[((size_t)(w0[j] + k) * MT * 16 + rin[j]) * kP + bb[j]] : 0.f;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) sum[j] += v[j];
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j * (int)blockDim.x < total) {
+                    if (part) part[(size_t)bb[j] * group_rows + rl[j]] = sum[j];
+                    else a.Y[(long long)bb[j] * a.ldy + row0 + rl[j]] = sum[j];
+                }
         }
     }
     if (part) {
@@ -411,14 +419,27 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
         if (s_last) {
             __threadfence();
             const float* base = a.partials + (size_t)me->group * a.S * cap * group_rows;
-            int b = 0, rloc = threadIdx.x;
-            while (rloc >= nrows) { rloc -= nrows; ++b; }
-            while (b < a.nb) {
-                float sum = 0.f;
-                for (int s2 = 0; s2 < a.S; ++s2) sum += __ldcg(base + ((size_t)s2 * cap + b) * group_rows + rloc);
-                a.Y[(long long)b * a.ldy + row0 + rloc] = sum;
-                rloc += blockDim.x;
-                while (rloc >= nrows) { rloc -= nrows; ++b; }
+            // four outputs per thread at a time, so that the loads of all ranges' partial sums are in flight together
+            const int total = nrows * a.nb;
+            for (int i0 = threadIdx.x; i0 < total; i0 += 4 * blockDim.x) {
+                int bb[4], rl[4];
+                float sum[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int idx = min(i0 + j * (int)blockDim.x, total - 1);
+                    bb[j] = idx / nrows; rl[j] = idx - bb[j] * nrows;
+                    sum[j] = 0.f;
+                }
+                for (int s2 = 0; s2 < a.S; ++s2) {
+                    float v[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) v[j] = __ldcg(base + ((size_t)s2 * cap + bb[j]) * group_rows + rl[j]);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) sum[j] += v[j];
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (i0 + j * (int)blockDim.x < total) a.Y[(long long)bb[j] * a.ldy + row0 + rl[j]] = sum[j];
             }
             if (threadIdx.x == 0) a.arrivals[me->group] = 0u;
         }
@@ -475,7 +496,7 @@ static int build_spmm_plan(const csb_matrix* A, int ci, MmaPlan::PerClass* P) {
     if (rc == 1) { P->unusable = true; return CSB_OK; }
     if (rc != CSB_OK) return rc;
     const int MT = mt_of(A), pitch = spmm_pitch(NT);
-    const int tile_bytes = (A->block_c * pitch + 127) & ~127;
+    const int tile_bytes = (spmm_tile_blocks(A->block_c) * A->block_c * pitch + 127) & ~127;
     // rings: as many weight stages (3, else 2) and input tiles (up to 8, at least 2) as shared memory holds
     int w_stages = 0, x_depth = 0;
     size_t smem = 0;
@@ -560,7 +581,8 @@ int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch,
     a.xp = (const uint8_t*)P.d_xp; a.ldy = ldy; a.partials = P.d_partials; a.arrivals = P.d_arrivals; a.status = PP.d_status;
     a.rows = (int)A->rows; a.cols = (int)A->cols; a.block_r = A->block_r; a.block_c = A->block_c;
     a.RG = P.RG; a.S = P.S; a.x_depth = P.x_depth; a.w_stages = P.w_stages;
-    a.pitch = spmm_pitch(NT); a.tile_bytes = (A->block_c * a.pitch + 127) & ~127;
+    a.tile_cols = spmm_tile_blocks(A->block_c) * A->block_c;
+    a.pitch = spmm_pitch(NT); a.tile_bytes = (a.tile_cols * a.pitch + 127) & ~127;
 #ifdef CSB_SPMM_CLOCKS
     if (!g_spmm_clocks) cudaMalloc((void**)&g_spmm_clocks, (size_t)1 << 24);
     a.clocks = g_spmm_clocks;
@@ -602,7 +624,7 @@ extern "C" int csb_spmm_plan_dump(const csb_matrix_t* A, int batch, int sm_count
     if (rc == 1) { set_error("the tensor-core layout does not apply to this matrix (fp16 values, block_r <= 64)"); return CSB_ERR_UNSUPPORTED; }
     if (rc != CSB_OK) return rc;
     info_out[0] = (int64_t)H.ctas.size(); info_out[1] = (int64_t)H.chunks.size(); info_out[2] = (int64_t)H.bytes.size();
-    info_out[3] = H.RG; info_out[4] = spmm_nt(batch) | (spmm_warps(spmm_nt(batch)) << 8); info_out[5] = H.S; info_out[6] = (int64_t)(H.warp_balance * 1e6);
+    info_out[3] = H.RG; info_out[4] = spmm_nt(batch) | (spmm_warps(spmm_nt(batch)) << 8) | (spmm_tile_blocks(A->block_c) << 16); info_out[5] = H.S; info_out[6] = (int64_t)(H.warp_balance * 1e6);
     info_out[7] = (int64_t)(H.balance * 1e6);
     if (stream_out) {
         if (stream_cap < (int64_t)H.bytes.size()) { set_error("stream buffer too small"); return CSB_ERR_INVALID_ARG; }

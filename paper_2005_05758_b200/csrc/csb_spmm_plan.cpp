@@ -35,7 +35,7 @@ static size_t spmm_item_bytes(int m, int nk) {
 // bookkeeping) and per 16-column slab the operand loads and the tensor instructions.
 static double item_cost(int nk, int MT, int NT) { return 110.0 + (double)((nk + 15) / 16) * (14.0 + MT * (6.0 + 2.0 * NT)); }
 
-static void emit_spmm_item(const csb_matrix* A, int64_t b, int k0, int k1, int tile, std::vector<uint8_t>& out) {
+static void emit_spmm_item(const csb_matrix* A, int64_t b, int k0, int k1, int tile, int col_base, std::vector<uint8_t>& out) {
     const int m = A->m[b], n = A->n[b], nk = k1 - k0, np2 = (nk + 1) / 2;
     const size_t base = out.size(), bytes = spmm_item_bytes(m, nk);
     out.resize(base + bytes, 0);
@@ -48,20 +48,20 @@ static void emit_spmm_item(const csb_matrix* A, int64_t b, int k0, int k1, int t
     h.mask_lo = (uint32_t)mask; h.mask_hi = (uint32_t)(mask >> 32);
     std::memcpy(p, &h, sizeof h);
     const uint8_t* ci = A->col_idx.data() + A->cidx_off[b];
-    for (int k = 0; k < nk; ++k) p[sizeof h + k] = ci[k0 + k];
+    for (int k = 0; k < nk; ++k) p[sizeof h + k] = (uint8_t)(col_base + ci[k0 + k]);
     uint8_t* v = p + sizeof h + pad_to((size_t)nk, 4);
     const uint8_t* src = A->val.data() + A->val_off[b] * 2;
     for (int r = 0; r < m; ++r)
         std::memcpy(v + (size_t)r * np2 * 4, src + ((size_t)r * n + k0) * 2, (size_t)nk * 2);
 }
 
-struct PlannedItem { int64_t block; int k0, k1, tile; };
+struct PlannedItem { int64_t block; int k0, k1, tile, col_base; };
 
 int plan_spmm_host(const csb_matrix* A, int NT, int sm_count, SpmmHostPlan* out) {
     if (A->val_dtype != CSB_F16 || A->block_r > 64 || A->nbc > 60000) return 1;
     const int64_t nbr = A->nbr, nbc = A->nbc;
     const int MT = A->block_r <= 16 ? 1 : A->block_r <= 32 ? 2 : 4;
-    const int nb_max = 8 * NT, n_warps = spmm_warps(NT);
+    const int nb_max = 8 * NT, n_warps = spmm_warps(NT), G = spmm_tile_blocks(A->block_c);
     const double x_bytes = (double)A->cols * spmm_pitch(NT), w_bytes = (double)A->nnz * 2.0 + 24.0 * (double)A->nblk;
     // ---- shape of the CTA tile: at most four block-rows, so that a block-row has several warps to
     // share its blocks between
@@ -96,7 +96,7 @@ int plan_spmm_host(const csb_matrix* A, int NT, int sm_count, SpmmHostPlan* out)
         // ---- column ranges of equal modelled work
         std::vector<double> prefix(nbc + 1, 0.0);
         for (int64_t j = 0; j < nbc; ++j) {
-            double c = 16.0;                                  // every tile is waited for and released by every warp
+            double c = 16.0 / G;                              // every tile is waited for and released by every warp
             for (int64_t bi = br0; bi < br1; ++bi) c += cost_of_block(bi * nbc + j);
             prefix[j + 1] = prefix[j] + c;
         }
@@ -113,8 +113,8 @@ int plan_spmm_host(const csb_matrix* A, int NT, int sm_count, SpmmHostPlan* out)
         for (int s = 0; s < S; ++s) {
             const int64_t j0 = cut[s], j1 = cut[s + 1];
             SpmmCta cta{};
-            cta.group = (int32_t)g; cta.split = s; cta.tile0 = (int32_t)j0; cta.ntiles = (int32_t)(j1 - j0);
-            out->max_tiles = std::max<int>(out->max_tiles, (int)(j1 - j0));
+            cta.group = (int32_t)g; cta.split = s; cta.tile0 = (int32_t)j0; cta.ntiles = (int32_t)((j1 - j0 + G - 1) / G);
+            out->max_tiles = std::max<int>(out->max_tiles, cta.ntiles);
             cta_cost.push_back(prefix[j1] - prefix[j0]);
             // ---- warps per block-row in proportion to the rows' work (largest remainders; at least one each)
             std::vector<double> row_work(nrows, 0.0);
@@ -149,7 +149,7 @@ int plan_spmm_host(const csb_matrix* A, int NT, int sm_count, SpmmHostPlan* out)
                     for (int k0 = 0; k0 < n; k0 += ksl) {
                         const int k1 = std::min(n, k0 + ksl);
                         const int w = (int)(std::min_element(load.begin(), load.end()) - load.begin());
-                        per_warp[w].push_back(PlannedItem{b, k0, k1, (int)(j - j0)});
+                        per_warp[w].push_back(PlannedItem{b, k0, k1, (int)((j - j0) / G), (int)((j - j0) % G) * A->block_c});
                         load[w] += item_cost(k1 - k0, MT, NT);
                     }
                 }
@@ -174,7 +174,7 @@ int plan_spmm_host(const csb_matrix* A, int NT, int sm_count, SpmmHostPlan* out)
                             used = 16;
                             open = true;
                         }
-                        emit_spmm_item(A, it.block, it.k0, it.k1, it.tile, out->bytes);
+                        emit_spmm_item(A, it.block, it.k0, it.k1, it.tile, it.col_base, out->bytes);
                         used += ib;
                     }
                     close();

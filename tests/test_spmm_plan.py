@@ -42,10 +42,12 @@ def decode(plan, rows, cols, br, bc):
                     kept_rows = [r for r in range(64) if (mask >> r) & 1]
                     need = len(kept_rows) * np2 * 4 + 16 + ((nk + 3) & ~3)
                     assert need <= size < need + 16
-                    bi, bj = group * RG + rr, tile0 + tile
+                    G = plan["tile_blocks"]
+                    assert np.all(cidx // bc == cidx[0] // bc) and cidx[0] // bc < G   # one block per item
+                    bi, bj = group * RG + rr, tile0 + tile * G + int(cidx[0]) // bc
                     for i, r in enumerate(kept_rows):
                         for k in range(nk):
-                            R, Cc = bi * br + r, bj * bc + int(cidx[k])
+                            R, Cc = bi * br + r, bj * bc + int(cidx[k]) % bc
                             W[R, Cc] = float(vals[i * np2 * 2 + k])
                             seen[R, Cc] += 1
                         if nk % 2:
@@ -72,8 +74,8 @@ def test_every_weight_once_in_the_right_stream(shape, batch, sms):
     for g in range(groups):
         mine = [c for c in plan["cta"] if c[0] == g]
         assert [c[1] for c in mine] == list(range(plan["S"]))
-        assert mine[0][2] == 0 and all(mine[i][2] + mine[i][3] == mine[i + 1][2] for i in range(len(mine) - 1))
-        assert mine[-1][2] + mine[-1][3] == nbc
+        assert mine[0][2] == 0 and all(mine[i][2] < mine[i + 1][2] <= mine[i][2] + mine[i][3] * plan["tile_blocks"] for i in range(len(mine) - 1))
+        assert mine[-1][2] + mine[-1][3] * plan["tile_blocks"] >= nbc
     W, seen = decode(plan, nbr * br, nbc * bc, br, bc)
     want = O.masked_dense(m.dense, br, bc, m.row_keep, m.col_keep, "f16")
     mask = O.block_mask(R, C, br, bc, m.row_keep, m.col_keep)
