@@ -178,9 +178,8 @@ int csb_spmv(const csb_matrix_t* A, const float* x, float* y, void* stream);
  * as |x| < 65504; larger or non-finite inputs give inf / NaN) and multiplied with
  * mma.sync.m16n8k16, fp32 accumulation, a block-row's outputs staying in registers across its
  * blocks.  The first such call on a handle for a batch size class (<= 8, <= 16, more)
- * builds a device layout for that class, a staging buffer for the packed inputs and, where row
- * groups are shared between CTAs, scratch for their partial sums (allocates and synchronises the
- * device once; make it outside of any stream capture).  The two kernels of this path are launched
+ * builds a device layout for that class and a staging buffer for the packed inputs (allocates and
+ * synchronises the device once; make it outside of any stream capture).  The two kernels of this path are launched
  * with programmatic stream serialization and wait, first thing, for the work in front of them on
  * `stream`.  Other cases use the CUDA-core kernel in batch tiles of 8 / 4 / 1.
  */

@@ -253,7 +253,6 @@ struct MmaPlan {                           // device side, one per batch class, 
         int RG = 1, S = 1, n_ctas = 0, n_groups = 0, x_depth = 0, w_stages = 0;
         size_t smem_bytes = 0;
         uint8_t* d_stream = nullptr; uint32_t* d_warp_desc = nullptr; SpmmCta* d_ctas = nullptr;
-        float* d_partials = nullptr; uint32_t* d_arrivals = nullptr;
         void* d_xp = nullptr;
         int64_t stream_bytes = 0;
         double balance = 1.0, warp_balance = 1.0;

@@ -23,8 +23,9 @@
 //     blocks do not wait for each other; they only meet at the input tiles, which a warp releases
 //     in order whether it used them or not, the last warp to release a slot refilling it.
 //   * A CTA covers RG block-rows x a range of block-columns (the planner's cut).  When a row group
-//     is divided between S CTAs each writes its partial sums to scratch and the last one to arrive
-//     adds them in the order of the ranges, so results are bit-reproducible.
+//     is divided between S CTAs these are launched as one thread-block cluster and add their sums
+//     through distributed shared memory, every CTA for a share of the rows and in the order of the
+//     ranges, so results are bit-reproducible and no scratch in global memory is needed.
 //   * More than 32 batch columns are served in passes of 32 (the weights of the later passes come
 //     from L2).
 #include <algorithm>
@@ -46,8 +47,6 @@ struct SpmmArgs {
     const uint8_t* xp;         // packed inputs: one row of `pitch` bytes per matrix column
     float* Y;
     long long ldy;
-    float* partials;           // [group][range][8 * NT][RG * block_r], S > 1 only
-    uint32_t* arrivals;        // [group], zero between launches
     uint32_t* status;
     int nb, rows, cols, block_r, block_c, tile_cols, RG, S, x_depth, w_stages, pitch, tile_bytes;   // tile_cols: matrix columns per input tile
 #ifdef CSB_SPMM_CLOCKS
@@ -64,8 +63,9 @@ struct SpmmArgs {
 // Shared-memory carve-up, identical on host and device.  The small fixed part comes first; the two
 // rings follow and are reused for the warps' partial sums once the main loop is over.
 struct SpmmSmem {
-    size_t wfull, xfull, wcnt, xcnt, dead, zero, rings, wring, xring, total;
-    __host__ __device__ SpmmSmem(int n_warps, int w_stages, int x_depth, int tile_bytes, int pitch, int MT, int NT) {
+    size_t wfull, xfull, wcnt, xcnt, dead, zero, rings, wring, xring, qsums, total;
+    // q_bytes: room for the CTA's own sums of its row group when a cluster shares the group (else 0)
+    __host__ __device__ SpmmSmem(int n_warps, int w_stages, int x_depth, int tile_bytes, int pitch, int MT, int NT, size_t q_bytes) {
         const int n_streams = n_warps;
         wfull = 0;
         xfull = wfull + (size_t)n_streams * w_stages * 8;
@@ -77,7 +77,8 @@ struct SpmmSmem {
         wring = rings;
         xring = wring + (size_t)n_streams * w_stages * kSpmmStageBytes;
         const size_t ring_end = xring + (size_t)x_depth * tile_bytes;
-        const size_t sums_end = rings + (size_t)n_warps * MT * 16 * (NT * 8 + 1) * 4;
+        qsums = (rings + (size_t)n_warps * MT * 16 * (NT * 8 + 1) * 4 + 127) & ~(size_t)127;
+        const size_t sums_end = qsums + q_bytes;
         total = ring_end > sums_end ? ring_end : sums_end;
     }
 };
@@ -119,6 +120,26 @@ __device__ __forceinline__ uint32_t atom_add_acq_rel_shared(uint32_t* p, uint32_
     return old;
 }
 
+// Thread-block cluster: barrier over all threads of all CTAs of the cluster (release / acquire), this
+// CTA's rank, the address of a shared-memory location in another CTA of the cluster, and a load from it.
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cluster_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
@@ -131,7 +152,7 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     pdl_launch_dependents();
     extern __shared__ __align__(128) uint8_t smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const SpmmSmem L(kSpmmWarps, a.w_stages, a.x_depth, a.tile_bytes, a.pitch, MT, NT);
+    const SpmmSmem L(kSpmmWarps, a.w_stages, a.x_depth, a.tile_bytes, a.pitch, MT, NT, a.S > 1 ? (size_t)8 * NT * a.RG * a.block_r * 4 : 0);
     uint64_t* wfull = reinterpret_cast<uint64_t*>(smem + L.wfull) + warp * a.w_stages;
     uint64_t* xfull = reinterpret_cast<uint64_t*>(smem + L.xfull);
     uint32_t* xcnt = reinterpret_cast<uint32_t*>(smem + L.xcnt);
@@ -350,12 +371,13 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     SPMM_LAP(5);                                   // the tiles behind this warp's last item
     __syncthreads();
     SPMM_LAP(6);                                   // waiting for the other warps of the CTA
-    if (*s_dead) {
+    const bool dead = *s_dead != 0u;
+    if (dead) {
         // a wait gave up (the status word says so): give copies that may still be in flight a bounded
         // time to land before the CTA's shared memory goes away, and write nothing
         const unsigned long long t0 = global_ns();
         while (global_ns() - t0 < 200000ull) __nanosleep(1000);
-        return;
+        if (a.S == 1) return;                      // (a CTA of a cluster still has to keep the cluster's barriers company)
     }
 
     // ---- the warps' sums meet in shared memory (the rings are no longer in use)
@@ -376,10 +398,10 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     const int group_rows = a.RG * a.block_r, row0 = me->group * group_rows;
     const int nrows = min(group_rows, a.rows - row0);
     constexpr int cap = 8 * NT;
-    float* part = a.S > 1 ? a.partials + ((size_t)me->group * a.S + me->split) * cap * group_rows : nullptr;
+    float* part = a.S > 1 ? reinterpret_cast<float*>(smem + L.qsums) : nullptr;    // [batch column][row of the group], this CTA's range only
     {
         // four outputs per thread at a time; the warps of a block-row are added in warp order
-        const int total = nrows * a.nb;
+        const int total = dead ? 0 : nrows * a.nb;
         for (int i0 = threadIdx.x; i0 < total; i0 += 4 * blockDim.x) {
             int bb[4], rl[4], w0[4], w1[4], rin[4];
             float sum[4];
@@ -410,39 +432,39 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
         }
     }
     if (part) {
-        // the last CTA of the row group to arrive adds the ranges' partial sums in range order
-        __shared__ uint32_t s_last;
-        __threadfence();
+        // The S CTAs of a row group form a thread-block cluster.  Once all of them have their sums in
+        // shared memory, every CTA adds up the S ranges, in range order, for its share of the group's
+        // rows, reading the other CTAs' sums through distributed shared memory; nobody leaves before
+        // everybody has read.  (The CTA barriers in front keep each warp together for the aligned cluster barrier.)
         __syncthreads();
-        if (threadIdx.x == 0) s_last = atomicAdd(a.arrivals + me->group, 1u) == (uint32_t)a.S - 1u;
-        __syncthreads();
-        if (s_last) {
-            __threadfence();
-            const float* base = a.partials + (size_t)me->group * a.S * cap * group_rows;
-            // four outputs per thread at a time, so that the loads of all ranges' partial sums are in flight together
-            const int total = nrows * a.nb;
-            for (int i0 = threadIdx.x; i0 < total; i0 += 4 * blockDim.x) {
-                int bb[4], rl[4];
-                float sum[4];
+        cluster_barrier();
+        const uint32_t rank = cluster_rank();
+        const int share = (nrows + a.S - 1) / a.S, r_lo = min(nrows, (int)rank * share), r_n = min(nrows, r_lo + share) - r_lo;
+        const uint32_t q_local = smem_u32(part);
+        const int total = dead ? 0 : r_n * a.nb;
+        for (int i0 = threadIdx.x; i0 < total; i0 += 4 * blockDim.x) {
+            int bb[4], rl[4];
+            float sum[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int idx = min(i0 + j * (int)blockDim.x, total - 1);
-                    bb[j] = idx / nrows; rl[j] = idx - bb[j] * nrows;
-                    sum[j] = 0.f;
-                }
-                for (int s2 = 0; s2 < a.S; ++s2) {
-                    float v[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) v[j] = __ldcg(base + ((size_t)s2 * cap + bb[j]) * group_rows + rl[j]);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) sum[j] += v[j];
-                }
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if (i0 + j * (int)blockDim.x < total) a.Y[(long long)bb[j] * a.ldy + row0 + rl[j]] = sum[j];
+            for (int j = 0; j < 4; ++j) {
+                const int idx = min(i0 + j * (int)blockDim.x, total - 1);
+                bb[j] = idx / r_n; rl[j] = r_lo + idx - bb[j] * r_n;
+                sum[j] = 0.f;
             }
-            if (threadIdx.x == 0) a.arrivals[me->group] = 0u;
+            for (int s2 = 0; s2 < a.S; ++s2) {
+                const uint32_t q_remote = map_to_cluster_cta(q_local, (uint32_t)s2);
+                float v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[j] = ld_cluster_f32(q_remote + (uint32_t)(bb[j] * group_rows + rl[j]) * 4u);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) sum[j] += v[j];
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j * (int)blockDim.x < total) a.Y[(long long)bb[j] * a.ldy + row0 + rl[j]] = sum[j];
         }
+        __syncthreads();
+        cluster_barrier();
     }
     SPMM_LAP(7);                                   // sums of the warps, partial sums of the ranges, store
 #ifdef CSB_SPMM_CLOCKS
@@ -480,6 +502,10 @@ static cudaError_t set_smem_attr(size_t bytes) {
     return cudaFuncSetAttribute(csb_spmm_tile_kernel<MT, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
 }
 template <int MT, int NT>
+static cudaError_t max_clusters(int* n, const cudaLaunchConfig_t* cfg) {
+    return cudaOccupancyMaxActiveClusters(n, csb_spmm_tile_kernel<MT, NT>, cfg);
+}
+template <int MT, int NT>
 static cudaError_t launch_tile_kernel(const cudaLaunchConfig_t* cfg, const SpmmArgs& a) {
     return cudaLaunchKernelEx(cfg, csb_spmm_tile_kernel<MT, NT>, a);
 }
@@ -502,7 +528,7 @@ static int build_spmm_plan(const csb_matrix* A, int ci, MmaPlan::PerClass* P) {
     size_t smem = 0;
     for (int ws = 3; ws >= 2 && !x_depth; --ws)
         for (int xd = std::min(8, std::max(2, H.max_tiles)); xd >= 2; --xd) {
-            const SpmmSmem L(spmm_warps(NT), ws, xd, tile_bytes, pitch, MT, NT);
+            const SpmmSmem L(spmm_warps(NT), ws, xd, tile_bytes, pitch, MT, NT, H.S > 1 ? (size_t)8 * NT * H.RG * A->block_r * 4 : 0);
             if (L.total <= A->smem_optin) { w_stages = ws; x_depth = xd; smem = L.total; break; }
         }
     if (!x_depth) { P->unusable = true; return CSB_OK; }
@@ -515,12 +541,19 @@ static int build_spmm_plan(const csb_matrix* A, int ci, MmaPlan::PerClass* P) {
     const size_t xp_bytes = (size_t)A->nbc * A->block_c * pitch;          // whole tiles, so that a tile copy never runs past the end
     CSB_CUDA(cudaMalloc(&P->d_xp, xp_bytes));
     CSB_CUDA(cudaMemset(P->d_xp, 0, xp_bytes));
-    if (H.S > 1) {
-        CSB_CUDA(cudaMalloc((void**)&P->d_partials, (size_t)H.n_groups * H.S * 8 * NT * H.RG * A->block_r * 4));
-        CSB_CUDA(cudaMalloc((void**)&P->d_arrivals, (size_t)H.n_groups * 4));
-        CSB_CUDA(cudaMemset(P->d_arrivals, 0, (size_t)H.n_groups * 4));
-    }
     CSB_CUDA(CSB_SPMM_DISPATCH(set_smem_attr, MT, NT, smem));
+    if (H.S > 1) {
+        // the S CTAs of a row group are launched as one cluster: make sure such a cluster can be resident
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)H.S; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)H.ctas.size()); cfg.blockDim = dim3((unsigned)spmm_warps(NT) * 32u); cfg.dynamicSmemBytes = smem;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        int clusters = 0;
+        CSB_CUDA(CSB_SPMM_DISPATCH(max_clusters, MT, NT, &clusters, &cfg));
+        if (clusters < 1) { P->unusable = true; return CSB_OK; }
+    }
     CSB_CUDA(cudaDeviceSynchronize());
     P->built = true;
     return CSB_OK;
@@ -533,7 +566,7 @@ void free_mma(csb_matrix* A) {
     cudaSetDevice(A->device);
     for (auto& c : A->mma->cls) {
         cudaFree(c.d_stream); cudaFree(c.d_warp_desc); cudaFree(c.d_ctas);
-        cudaFree(c.d_partials); cudaFree(c.d_arrivals); cudaFree(c.d_xp);
+        cudaFree(c.d_xp);
     }
     cudaSetDevice(prev);
     delete A->mma;
@@ -578,7 +611,7 @@ int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch,
     cudaStream_t st = (cudaStream_t)stream;
     SpmmArgs a{};
     a.stream = P.d_stream; a.warp_desc = (const uint4*)P.d_warp_desc; a.ctas = P.d_ctas;
-    a.xp = (const uint8_t*)P.d_xp; a.ldy = ldy; a.partials = P.d_partials; a.arrivals = P.d_arrivals; a.status = PP.d_status;
+    a.xp = (const uint8_t*)P.d_xp; a.ldy = ldy; a.status = PP.d_status;
     a.rows = (int)A->rows; a.cols = (int)A->cols; a.block_r = A->block_r; a.block_c = A->block_c;
     a.RG = P.RG; a.S = P.S; a.x_depth = P.x_depth; a.w_stages = P.w_stages;
     a.tile_cols = spmm_tile_blocks(A->block_c) * A->block_c;
@@ -593,15 +626,18 @@ int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch,
         a.Y = Y + (int64_t)b0 * ldy;
         // both kernels order themselves behind the work in front (pdl_wait), so they may be launched
         // with programmatic stream serialization: their scheduling overlaps its tail
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;             // the CTAs that share a row group
+        attr[1].val.clusterDim.x = (unsigned)P.S; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
         cudaLaunchConfig_t cfg{};
         cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 1;
         cfg.gridDim = dim3((unsigned)((A->cols + 31) / 32)); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0;
         CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_pack_x_kernel, X + (int64_t)b0 * ldx, (long long)ldx, a.nb, (int)A->cols, (uint8_t*)P.d_xp,
                                     a.pitch, NT));
         cfg.gridDim = dim3((unsigned)P.n_ctas); cfg.blockDim = dim3((unsigned)spmm_warps(NT) * 32u); cfg.dynamicSmemBytes = P.smem_bytes;
+        cfg.numAttrs = P.S > 1 ? 2 : 1;
         CSB_CUDA(CSB_SPMM_DISPATCH(launch_tile_kernel, MT, NT, &cfg, a));
         CSB_CUDA(cudaGetLastError());
     }

@@ -10,10 +10,11 @@
 // warps of a row have done about the same amount of work, so they move through the shared ring of
 // input tiles together.  The choice of RG and of the number S of column ranges per row group trades
 // three kinds of traffic per CTA against each other: the weights (once in all), the packed inputs
-// (once per row group, divided by S) and the partial sums that S > 1 CTAs of a row group leave for
-// the last of them to add (in the fixed order of the ranges).
+// (once per row group, divided by S) and the sums that the S > 1 CTAs of a row group, one thread-block
+// cluster, add up through distributed shared memory (in the fixed order of the ranges).
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <numeric>
 
 #include "csb_internal.hpp"
@@ -70,10 +71,12 @@ int plan_spmm_host(const csb_matrix* A, int NT, int sm_count, SpmmHostPlan* out)
     for (int RG = 4; RG >= 1; RG /= 2) {
         const int64_t groups = (nbr + RG - 1) / RG;
         int64_t S = std::max<int64_t>(1, sm_count / groups);
-        S = std::min<int64_t>(S, nbc);
+        S = std::min<int64_t>(std::min<int64_t>(S, nbc), 8);      // the CTAs of a row group form one cluster: at most 8
         const double ctas = (double)(groups * S);
         const double waves = std::ceil(ctas / sm_count);
-        const double per_cta = w_bytes / ctas + x_bytes / (double)S + (S > 1 ? 2.0 * RG * A->block_r * nb_max * 4.0 : 0.0);
+        // (a cluster costs two cluster-wide barriers and the wait for its slowest CTA: as much time as about 120 KB of traffic per CTA (measured: a small GRU layer runs faster without, the 8192 x 8192 sweep with))
+        static const double cluster_cost = getenv("CSB_SPMM_CLUSTER_COST") ? atof(getenv("CSB_SPMM_CLUSTER_COST")) : 120e3;
+        const double per_cta = w_bytes / ctas + x_bytes / (double)S + (S > 1 ? 2.0 * RG * A->block_r * nb_max * 4.0 + cluster_cost : 0.0);
         // short ranges leave a warp only a few items to even its load out with
         const double cost = per_cta * waves * (1.0 + 6.0 * (double)S / (double)nbc);
         if (cost < best) { best = cost; best_RG = RG; best_S = (int)S; }
