@@ -266,6 +266,43 @@ int csb_gru_forward(int n_layers, const csb_matrix_t* const* W, const float* con
                     unsigned flags, void* stream);
 
 /*
+ * Cell variants of the paper's benchmark models (Table 1) and of the GRU reference of Section 2.1.
+ * They run one timestep at a time: per layer and step the CSB products go through the kernels of
+ * csb_spmv / csb_spmm (whichever serves the batch size) and small kernels do the element-wise
+ * part.  Arguments, flags (CSB_FLAG_ASYNC, CSB_FLAG_HOST_IO), caching of per-(matrices, B) device
+ * state on the first call and the no-overlap rule are those of csb_lstm_forward; T = 0 or B = 0
+ * is a no-op; errors are INVALID_ARG, SHAPE, UNSUPPORTED, ALLOC, CUDA, TIMEOUT as there.
+ *
+ * csb_lstmp_forward -- LSTM with a recurrent projection (LSTMP, Table 1: the SR1 layers, whose sizes
+ * fit a projection to 512 units and no peephole weights).
+ *   W[l]   CSB matrix [4*H, I_l + P], rows i, f, g, o; the last P columns multiply the projected state;
+ *          I_l = P above the first layer.   Wp[l]  CSB matrix [P, H], the projection (no bias).
+ *   bias[l] device float32 [4*H] or NULL;  x [T, B, I];  h0 [L, B, P], c0 [L, B, H] or NULL (zeros);
+ *   y [T, B, P] (top layer's projected state) or NULL;  hT [L, B, P], cT [L, B, H] or NULL.
+ *   z = W.[u_t ; r_{t-1}] + b;  c_t = s(z_f) c_{t-1} + s(z_i) tanh(z_g);  m_t = s(z_o) tanh(c_t);  r_t = Wp.m_t.
+ *
+ * csb_ligru_forward -- light GRU (Li-GRU, Table 1: model SR3): no reset gate, rectified candidate.  The
+ * batch normalisation of the cell's feed-forward products is, at inference, a per-unit scale (folded
+ * into the weight rows by the caller) and shift (the bias here).
+ *   W[l]   CSB matrix [2*H, I_l + H], rows z (update gate), c (candidate);  bias[l] [2*H] or NULL.
+ *   a = W.[u_t ; h_{t-1}] + b;  z = s(a_z);  h_t = z h_{t-1} + (1 - z) max(a_c, 0).
+ *
+ * csb_gru_reset_before_forward -- GRU whose reset gate acts BEFORE the candidate's recurrent product
+ * (two dependent products per step, where csb_gru_forward needs one).
+ *   W[l]   CSB matrix [3*H, I_l + H], rows r, z, n;  bias[l] [3*H] = b_r, b_z, b_n or NULL.
+ *   [a_r ; a_z] = W[0:2H].[u_t ; h_{t-1}];  r = s(a_r + b_r);  z = s(a_z + b_z);
+ *   n = tanh(W[2H:3H].[u_t ; r * h_{t-1}] + b_n);  h_t = (1 - z) n + z h_{t-1}.
+ *   The two row ranges run as products of their own, so 2*H must be a multiple of block_r (else UNSUPPORTED).
+ */
+int csb_lstmp_forward(int n_layers, const csb_matrix_t* const* W, const csb_matrix_t* const* Wp, const float* const* bias,
+                      const float* x, int64_t T, int B, const float* h0, const float* c0, float* y, float* hT, float* cT,
+                      unsigned flags, void* stream);
+int csb_ligru_forward(int n_layers, const csb_matrix_t* const* W, const float* const* bias, const float* x, int64_t T, int B,
+                      const float* h0, float* y, float* hT, unsigned flags, void* stream);
+int csb_gru_reset_before_forward(int n_layers, const csb_matrix_t* const* W, const float* const* bias, const float* x, int64_t T,
+                                 int B, const float* h0, float* y, float* hT, unsigned flags, void* stream);
+
+/*
  * csb_test_barrier_hook -- testing aid for the give-up path of the time loop's waits on other
  * CTAs (the paper has no counterpart).  Makes every later recurrent call expect `extra_arrivals`
  * arrivals at its grid barrier that never come (at batch 1, where CTAs exchange h as flagged

@@ -272,5 +272,30 @@ def csb_gru_forward(W: Sequence[CsbMatrix], bias, x, h0, y, hT, flags: int = 0, 
                                _stream(stream)))
 
 
+def csb_lstmp_forward(W: Sequence[CsbMatrix], Wp: Sequence[CsbMatrix], bias, x, h0, c0, y, hT, cT, flags: int = 0, stream=None) -> None:
+    L = len(W)
+    lib.csb_lstmp_forward.argtypes = [C.c_int, C.POINTER(_P), C.POINTER(_P), C.POINTER(_P), _P, C.c_int64, C.c_int, _P, _P, _P, _P, _P, C.c_uint, _P]
+    lib.csb_lstmp_forward.restype = C.c_int
+    b = _ptr_array(bias, L) if bias is not None else None
+    _check(lib.csb_lstmp_forward(L, _ptr_array(W, L), _ptr_array(Wp, L), b, _ptr(x), x.shape[0], x.shape[1], _ptr(h0), _ptr(c0), _ptr(y),
+                                 _ptr(hT), _ptr(cT), flags, _stream(stream)))
+
+
+def _gru_like(fn, W, bias, x, h0, y, hT, flags, stream):
+    L = len(W)
+    fn.argtypes = [C.c_int, C.POINTER(_P), C.POINTER(_P), _P, C.c_int64, C.c_int, _P, _P, _P, C.c_uint, _P]
+    fn.restype = C.c_int
+    b = _ptr_array(bias, L) if bias is not None else None
+    _check(fn(L, _ptr_array(W, L), b, _ptr(x), x.shape[0], x.shape[1], _ptr(h0), _ptr(y), _ptr(hT), flags, _stream(stream)))
+
+
+def csb_ligru_forward(W: Sequence[CsbMatrix], bias, x, h0, y, hT, flags: int = 0, stream=None) -> None:
+    _gru_like(lib.csb_ligru_forward, W, bias, x, h0, y, hT, flags, stream)
+
+
+def csb_gru_reset_before_forward(W: Sequence[CsbMatrix], bias, x, h0, y, hT, flags: int = 0, stream=None) -> None:
+    _gru_like(lib.csb_gru_reset_before_forward, W, bias, x, h0, y, hT, flags, stream)
+
+
 # shorter aliases
 spmv, spmm, lstm_forward, gru_forward = csb_spmv, csb_spmm, csb_lstm_forward, csb_gru_forward

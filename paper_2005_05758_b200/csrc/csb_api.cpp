@@ -20,6 +20,47 @@ void clear_error() { g_err[0] = 0; }
 
 static std::atomic<uint64_t> g_uid{1};
 
+int product_any(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream) {
+    if (spmm_mma_applicable(A, batch)) {
+        const int rc = launch_spmm_mma(A, X, ldx, batch, Y, ldy, stream);
+        if (rc != 1) return rc;                       // 1: the tensor-core plan does not fit this matrix
+    }
+    if (batch == 1 && A->panel && A->panel->built) return launch_panels(A, X, Y, stream);
+    return launch_product(A, X, ldx, batch, Y, ldy, stream);
+}
+
+int slice_block_rows(const csb_matrix* A, int64_t bi0, int64_t bi1, csb_matrix** out) {
+    *out = nullptr;
+    if (bi0 < 0 || bi1 > A->nbr || bi0 >= bi1) { set_error("block-row range [%lld, %lld) of %lld", (long long)bi0, (long long)bi1, (long long)A->nbr); return CSB_ERR_INVALID_ARG; }
+    csb_matrix* S = new (std::nothrow) csb_matrix();
+    if (!S) { set_error("out of host memory"); return CSB_ERR_ALLOC; }
+    int rc = CSB_OK;
+    try {
+        S->rows = std::min<int64_t>(A->rows, bi1 * A->block_r) - bi0 * A->block_r; S->cols = A->cols;
+        S->block_r = A->block_r; S->block_c = A->block_c; S->nbr = bi1 - bi0; S->nbc = A->nbc; S->nblk = S->nbr * S->nbc;
+        S->val_dtype = A->val_dtype; S->device = A->device; S->opts = A->opts; S->uid = g_uid.fetch_add(1);
+        const int64_t b0 = bi0 * A->nbc, b1 = bi1 * A->nbc;
+        const int vs = val_size(A->val_dtype);
+        S->m.assign(A->m.begin() + b0, A->m.begin() + b1);
+        S->n.assign(A->n.begin() + b0, A->n.begin() + b1);
+        S->row_idx.assign(A->row_idx.begin() + A->ridx_off[b0], A->row_idx.begin() + A->ridx_off[b1]);
+        S->col_idx.assign(A->col_idx.begin() + A->cidx_off[b0], A->col_idx.begin() + A->cidx_off[b1]);
+        S->val.assign(A->val.begin() + A->val_off[b0] * vs, A->val.begin() + A->val_off[b1] * vs);
+        S->val_off.resize(S->nblk + 1); S->ridx_off.resize(S->nblk + 1); S->cidx_off.resize(S->nblk + 1);
+        for (int64_t b = 0; b <= S->nblk; ++b) {
+            S->val_off[b] = A->val_off[b0 + b] - A->val_off[b0];
+            S->ridx_off[b] = A->ridx_off[b0 + b] - A->ridx_off[b0];
+            S->cidx_off[b] = A->cidx_off[b0 + b] - A->cidx_off[b0];
+        }
+        S->nnz = (int64_t)S->val_off[S->nblk];
+        rc = validate_host(S);
+        if (rc == CSB_OK && S->device >= 0) { rc = plan_product(S); if (rc == CSB_OK) rc = plan_panels(S); }
+    } catch (const std::bad_alloc&) { set_error("out of host memory while slicing"); rc = CSB_ERR_ALLOC; }
+    if (rc != CSB_OK) { csb_free(S); return rc; }
+    *out = S;
+    return CSB_OK;
+}
+
 }  // namespace csb
 
 using namespace csb;
@@ -169,6 +210,7 @@ int csb_panel_dump(const csb_matrix_t* A, int ctas, int warps_per_cta, int stage
 
 void csb_free(csb_matrix_t* A) {
     if (!A) return;
+    drop_cell_plans(A);
     drop_rnn_plans(A);
     free_mma(A);
     free_panels(A);
@@ -184,12 +226,7 @@ int csb_spmm(const csb_matrix_t* A, const float* X, int64_t ldx, int batch, floa
     if (!X || !Y) { set_error("X or Y is NULL"); return CSB_ERR_INVALID_ARG; }
     if (ldx < A->cols || ldy < A->rows) { set_error("ldx=%lld < cols or ldy=%lld < rows", (long long)ldx, (long long)ldy); return CSB_ERR_SHAPE; }
     if (A->device < 0) { set_error("matrix was encoded host-only (device = -1)"); return CSB_ERR_UNSUPPORTED; }
-    if (spmm_mma_applicable(A, batch)) {
-        const int rc = launch_spmm_mma(A, X, ldx, batch, Y, ldy, stream);
-        if (rc != 1) return rc;                       // 1: the tensor-core plan does not fit this matrix
-    }
-    if (batch == 1 && A->panel && A->panel->built) return launch_panels(A, X, Y, stream);
-    return launch_product(A, X, ldx, batch, Y, ldy, stream);
+    return product_any(A, X, ldx, batch, Y, ldy, stream);
 }
 
 int csb_spmv(const csb_matrix_t* A, const float* x, float* y, void* stream) {

@@ -318,6 +318,15 @@ void free_product(csb_matrix* A);
 int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy,
                    void* stream);
 
+// csb_api.cpp
+// Y[b, :] = A . X[b, :] through whichever kernel serves the batch size (what csb_spmm does after its argument checks).
+int product_any(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream);
+// A new handle (same device, planned) holding block-rows [bi0, bi1) of A; the caller frees it with csb_free.
+int slice_block_rows(const csb_matrix* A, int64_t bi0, int64_t bi1, csb_matrix** out);
+
+// csb_cells.cu
+void drop_cell_plans(const csb_matrix* A); // forget cached plans of the cell variants that use A
+
 // csb_rnn.cu
 void drop_rnn_plans(const csb_matrix* A);  // forget cached time-loop plans that use A
 

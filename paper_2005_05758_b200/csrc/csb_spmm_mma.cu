@@ -39,6 +39,7 @@ namespace csb {
 
 constexpr uint32_t kOffMaskM = 0x3fffffffu;
 constexpr uint32_t kNoRow = 0xffffffffu;
+constexpr size_t kSpmmStaticSmem = 256;       // the kernel's statically allocated shared memory (CTA descriptor, row table), rounded up
 
 struct SpmmArgs {
     const uint8_t* stream;
@@ -529,7 +530,7 @@ static int build_spmm_plan(const csb_matrix* A, int ci, MmaPlan::PerClass* P) {
     for (int ws = 3; ws >= 2 && !x_depth; --ws)
         for (int xd = std::min(8, std::max(2, H.max_tiles)); xd >= 2; --xd) {
             const SpmmSmem L(spmm_warps(NT), ws, xd, tile_bytes, pitch, MT, NT, H.S > 1 ? (size_t)8 * NT * H.RG * A->block_r * 4 : 0);
-            if (L.total <= A->smem_optin) { w_stages = ws; x_depth = xd; smem = L.total; break; }
+            if (L.total + kSpmmStaticSmem <= A->smem_optin) { w_stages = ws; x_depth = xd; smem = L.total; break; }
         }
     if (!x_depth) { P->unusable = true; return CSB_OK; }
     P->RG = H.RG; P->S = H.S; P->n_ctas = (int)H.ctas.size(); P->n_groups = H.n_groups;
@@ -541,7 +542,8 @@ static int build_spmm_plan(const csb_matrix* A, int ci, MmaPlan::PerClass* P) {
     const size_t xp_bytes = (size_t)A->nbc * A->block_c * pitch;          // whole tiles, so that a tile copy never runs past the end
     CSB_CUDA(cudaMalloc(&P->d_xp, xp_bytes));
     CSB_CUDA(cudaMemset(P->d_xp, 0, xp_bytes));
-    CSB_CUDA(CSB_SPMM_DISPATCH(set_smem_attr, MT, NT, smem));
+    // (the limit belongs to the kernel, not to this plan: other matrices launch the same instantiation with other sizes)
+    CSB_CUDA(CSB_SPMM_DISPATCH(set_smem_attr, MT, NT, A->smem_optin - kSpmmStaticSmem));
     if (H.S > 1) {
         // the S CTAs of a row group are launched as one cluster: make sure such a cluster can be resident
         cudaLaunchAttribute attr[1];
