@@ -46,7 +46,8 @@ typedef enum csb_status {
     CSB_ERR_UNSUPPORTED = -8   /* valid request this build does not implement      */
 } csb_status;
 
-enum { CSB_F32 = 0, CSB_F16 = 1 };          /* storage type of the packed values */
+enum { CSB_F32 = 0, CSB_F16 = 1,            /* storage type of the packed values */
+       CSB_Q16 = 2 };                       /* 16-bit fixed point; handles made by csb_encode_q16 only */
 enum { CSB_FLAG_ASYNC = 1u,                 /* recurrent calls: do not wait for the status word */
        CSB_FLAG_HOST_IO = 2u };             /* recurrent calls: sequence and state pointers are host memory */
 
@@ -71,7 +72,7 @@ typedef struct csb_view {
     int64_t rows, cols;
     int32_t block_r, block_c;
     int64_t nbr, nbc, nblk, nnz;
-    int32_t val_dtype;           /* CSB_F32 | CSB_F16                                  */
+    int32_t val_dtype;           /* CSB_F32 | CSB_F16 | CSB_Q16 (int16 values)         */
     const uint16_t* m;           /* [nblk] kept rows per block                         */
     const uint16_t* n;           /* [nblk] kept columns per block                      */
     const uint8_t* row_idx;      /* in-block indices, 0-based, ascending, concatenated */
@@ -264,6 +265,30 @@ int csb_lstm_forward(int n_layers, const csb_matrix_t* const* W, const float* co
 int csb_gru_forward(int n_layers, const csb_matrix_t* const* W, const float* const* bias,
                     const float* x, int64_t T, int B, const float* h0, float* y, float* hT,
                     unsigned flags, void* stream);
+
+/*
+ * 16-bit fixed-point CSB product: the arithmetic of the paper's own processing elements (weights
+ * quantised to 16-bit fixed point, Section 6.2.2; 16-bit fixed-point multipliers, Section 6.3.1).
+ * The paper fixes neither the place of the binary point, the rounding nor the accumulator width;
+ * here a value v with f fraction bits is the integer clamp(rint(v * 2^f), -32768, 32767) (halves
+ * to even, NaN -> 0), f is the caller's choice per matrix and per input, and the product returns
+ * the exact integer accumulators (64 bits, cannot overflow), so the real result is
+ * acc * 2^-(f_w + f_x) and does not depend on the order of summation.
+ *
+ * csb_encode_q16 -- as csb_encode, the values stored as int16 with `frac_bits` fraction bits
+ * (0..30; csb_view then gives val_dtype = CSB_Q16 and int16 values).  block_r and block_c at
+ * most 128.  Such a handle serves csb_spmm_q16 only: the floating-point products and the
+ * recurrent calls refuse it with CSB_ERR_UNSUPPORTED.
+ *
+ * csb_spmm_q16 -- acc[b, :] = A_q . x_q[b, :] in integers.
+ *   Xq   device, int16, batch rows of `cols` fixed-point inputs, row stride ldx >= cols;
+ *   acc  device, int64, batch rows of `rows` accumulators, row stride ldy >= rows, overwritten
+ *        (rows kept in no block become 0).  batch = 0 is a no-op; asynchronous on `stream`.
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED (handle is not CSB_Q16, host-only handle), CUDA.
+ */
+int csb_encode_q16(const float* dense, int64_t rows, int64_t cols, int64_t ld, int block_r, int block_c,
+                   const uint8_t* row_keep, const uint8_t* col_keep, int frac_bits, int device, csb_matrix_t** out);
+int csb_spmm_q16(const csb_matrix_t* A, const int16_t* Xq, int64_t ldx, int batch, int64_t* acc, int64_t ldy, void* stream);
 
 /*
  * Cell variants of the paper's benchmark models (Table 1) and of the GRU reference of Section 2.1.

@@ -21,6 +21,7 @@ lib = C.CDLL(_LIB_PATH)
 
 CSB_F32, CSB_F16 = 0, 1
 CSB_FLAG_ASYNC, CSB_FLAG_HOST_IO = 1, 2
+CSB_Q16 = 2
 _DT = {"f32": CSB_F32, "f16": CSB_F16}
 
 
@@ -116,9 +117,9 @@ class CsbMatrix:
 
         ro = arr(v.ridx_off, nblk + 1, np.uint32)
         co = arr(v.cidx_off, nblk + 1, np.uint32)
-        vdt = np.float16 if v.val_dtype == CSB_F16 else np.float32
+        vdt = {CSB_F16: np.float16, CSB_F32: np.float32, CSB_Q16: np.int16}[v.val_dtype]
         return {"rows": v.rows, "cols": v.cols, "block_r": v.block_r, "block_c": v.block_c, "nbr": v.nbr,
-                "nbc": v.nbc, "nnz": nnz, "val_dtype": "f16" if v.val_dtype == CSB_F16 else "f32",
+                "nbc": v.nbc, "nnz": nnz, "val_dtype": {CSB_F16: "f16", CSB_F32: "f32", CSB_Q16: "q16"}[v.val_dtype],
                 "m": arr(v.m, nblk, np.uint16), "n": arr(v.n, nblk, np.uint16),
                 "row_idx": arr(v.row_idx, int(ro[-1]), np.uint8), "col_idx": arr(v.col_idx, int(co[-1]), np.uint8),
                 "val_off": arr(v.val_off, nblk + 1, np.uint64), "ridx_off": ro, "cidx_off": co,
@@ -173,6 +174,29 @@ def csb_plan_dump(A: CsbMatrix, ctas: int, warps_per_cta: int, stage_bytes: int)
     out = {k: int(v) for k, v in zip(keys, info)}
     out.update(stream=stream[: out["stream_bytes"]], chunk_table=chunks[: out["chunks"]], warp_begin=wbeg)
     return out
+
+
+def csb_encode_q16(dense: np.ndarray, block_r: int, block_c: int, row_keep: np.ndarray, col_keep: np.ndarray, frac_bits: int,
+                   device: int = 0) -> CsbMatrix:
+    """CSB handle with 16-bit fixed-point values (see csb.h); serves csb_spmm_q16 only."""
+    lib.csb_encode_q16.argtypes = [_P, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, _P, _P, C.c_int, C.c_int, C.POINTER(_P)]
+    lib.csb_encode_q16.restype = C.c_int
+    dense = np.ascontiguousarray(dense, dtype=np.float32)
+    rk = np.ascontiguousarray(row_keep, dtype=np.uint8)
+    ck = np.ascontiguousarray(col_keep, dtype=np.uint8)
+    rows, cols = dense.shape
+    out = _P()
+    _check(lib.csb_encode_q16(dense.ctypes.data, rows, cols, cols, block_r, block_c, rk.ctypes.data, ck.ctypes.data, frac_bits, device,
+                              C.byref(out)))
+    return CsbMatrix(out.value)
+
+
+def csb_spmm_q16(A: CsbMatrix, Xq, acc, stream=None) -> None:
+    """acc[b, :] = A_q . Xq[b, :] in integers: Xq torch int16 [batch, cols], acc torch int64 [batch, rows]."""
+    lib.csb_spmm_q16.argtypes = [_P, _P, C.c_int64, C.c_int, _P, C.c_int64, _P]
+    lib.csb_spmm_q16.restype = C.c_int
+    batch = Xq.shape[0]
+    _check(lib.csb_spmm_q16(A.handle, _ptr(Xq), Xq.stride(0) if batch else 0, batch, _ptr(acc), acc.stride(0) if batch else 0, _stream(stream)))
 
 
 def csb_spmm_plan_dump(A: CsbMatrix, batch: int, sm_count: int) -> dict:

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcsb.so")
-SOURCES = ["csb_api.cpp", "csb_encode.cpp", "csb_plan.cpp", "csb_schedule.cpp", "csb_spmm_plan.cpp", "csb_panel_plan.cpp", "csb_product.cu", "csb_panel.cu", "csb_spmm_mma.cu", "csb_rnn.cu", "csb_rnn_step.cu", "csb_cells.cu", "csb_project.cu"]
+SOURCES = ["csb_api.cpp", "csb_encode.cpp", "csb_plan.cpp", "csb_schedule.cpp", "csb_spmm_plan.cpp", "csb_panel_plan.cpp", "csb_product.cu", "csb_panel.cu", "csb_spmm_mma.cu", "csb_rnn.cu", "csb_rnn_step.cu", "csb_cells.cu", "csb_fixed.cu", "csb_project.cu"]
 HEADERS = ["csb_internal.hpp", "csb_device.cuh", os.path.join("..", "..", "include", "csb.h")]
 
 

@@ -84,9 +84,9 @@ const char* csb_strerror(int status) {
 
 const char* csb_last_error(void) { return g_err; }
 
-int csb_encode(const float* dense, int64_t rows, int64_t cols, int64_t ld, int block_r, int block_c,
-               const uint8_t* row_keep, const uint8_t* col_keep, int val_dtype, int device,
-               const csb_plan_opts* opts, csb_matrix_t** out) {
+static int encode_common(const float* dense, int64_t rows, int64_t cols, int64_t ld, int block_r, int block_c,
+                         const uint8_t* row_keep, const uint8_t* col_keep, int val_dtype, int frac_bits, int device,
+                         const csb_plan_opts* opts, csb_matrix_t** out) {
     clear_error();
     if (!out) { set_error("out is NULL"); return CSB_ERR_INVALID_ARG; }
     *out = nullptr;
@@ -94,7 +94,11 @@ int csb_encode(const float* dense, int64_t rows, int64_t cols, int64_t ld, int b
     if (rows <= 0 || cols <= 0 || ld < cols) { set_error("rows=%lld cols=%lld ld=%lld", (long long)rows, (long long)cols, (long long)ld); return CSB_ERR_INVALID_ARG; }
     if (rows > 0x7fffffff || cols > 0x7fffffff) { set_error("dimensions above 2^31-1 are not supported"); return CSB_ERR_UNSUPPORTED; }
     if (block_r < 1 || block_r > 256 || block_c < 1 || block_c > 256) { set_error("block sizes must be 1..256, got %dx%d", block_r, block_c); return CSB_ERR_INVALID_ARG; }
-    if (val_dtype != CSB_F32 && val_dtype != CSB_F16) { set_error("val_dtype %d", val_dtype); return CSB_ERR_DTYPE; }
+    if (val_dtype != CSB_F32 && val_dtype != CSB_F16 && val_dtype != CSB_Q16) { set_error("val_dtype %d", val_dtype); return CSB_ERR_DTYPE; }
+    if (val_dtype == CSB_Q16 && (block_r > 128 || block_c > 128 || frac_bits < 0 || frac_bits > 30)) {
+        set_error("fixed point: blocks up to 128x128 and 0..30 fraction bits, got %dx%d and %d", block_r, block_c, frac_bits);
+        return CSB_ERR_INVALID_ARG;
+    }
     if (device < -1) { set_error("device %d", device); return CSB_ERR_INVALID_ARG; }
     if (opts && (opts->ctas < 0 || opts->warps_per_cta < 0 || opts->warps_per_cta > 16 || opts->stages < 0 || opts->stages > 8 ||
                  (opts->stage_bytes != 0 && (opts->stage_bytes < 1024 || opts->stage_bytes > 16384)))) {
@@ -106,16 +110,44 @@ int csb_encode(const float* dense, int64_t rows, int64_t cols, int64_t ld, int b
     if (!A) { set_error("out of host memory"); return CSB_ERR_ALLOC; }
     A->device = device;
     A->uid = g_uid.fetch_add(1);
+    A->q_frac_bits = frac_bits;
     if (opts) A->opts = *opts;
     int rc = encode_host(dense, rows, cols, ld, block_r, block_c, row_keep, col_keep, val_dtype, A);
     if (rc == CSB_OK) rc = validate_host(A);
     if (rc == CSB_OK && device >= 0) {
-        try { rc = plan_product(A); if (rc == CSB_OK) rc = plan_panels(A); }
+        try {
+            if (val_dtype == CSB_Q16) rc = plan_fixed(A);
+            else { rc = plan_product(A); if (rc == CSB_OK) rc = plan_panels(A); }
+        }
         catch (const std::bad_alloc&) { set_error("out of host memory while planning"); rc = CSB_ERR_ALLOC; }
     }
     if (rc != CSB_OK) { csb_free(A); return rc; }
     *out = A;
     return CSB_OK;
+}
+
+int csb_encode(const float* dense, int64_t rows, int64_t cols, int64_t ld, int block_r, int block_c,
+               const uint8_t* row_keep, const uint8_t* col_keep, int val_dtype, int device,
+               const csb_plan_opts* opts, csb_matrix_t** out) {
+    if (val_dtype == CSB_Q16) { clear_error(); set_error("fixed-point handles are made by csb_encode_q16 (it takes the fraction bits)"); return CSB_ERR_DTYPE; }
+    return encode_common(dense, rows, cols, ld, block_r, block_c, row_keep, col_keep, val_dtype, 0, device, opts, out);
+}
+
+int csb_encode_q16(const float* dense, int64_t rows, int64_t cols, int64_t ld, int block_r, int block_c,
+                   const uint8_t* row_keep, const uint8_t* col_keep, int frac_bits, int device, csb_matrix_t** out) {
+    return encode_common(dense, rows, cols, ld, block_r, block_c, row_keep, col_keep, CSB_Q16, frac_bits, device, nullptr, out);
+}
+
+int csb_spmm_q16(const csb_matrix_t* A, const int16_t* Xq, int64_t ldx, int batch, int64_t* acc, int64_t ldy, void* stream) {
+    clear_error();
+    if (!A) { set_error("A is NULL"); return CSB_ERR_INVALID_ARG; }
+    if (A->val_dtype != CSB_Q16) { set_error("the handle does not hold fixed-point values (make it with csb_encode_q16)"); return CSB_ERR_UNSUPPORTED; }
+    if (batch < 0) { set_error("batch %d", batch); return CSB_ERR_INVALID_ARG; }
+    if (batch == 0) return CSB_OK;
+    if (!Xq || !acc) { set_error("Xq or acc is NULL"); return CSB_ERR_INVALID_ARG; }
+    if (ldx < A->cols || ldy < A->rows) { set_error("ldx=%lld < cols or ldy=%lld < rows", (long long)ldx, (long long)ldy); return CSB_ERR_SHAPE; }
+    if (A->device < 0 || !A->fixed) { set_error("matrix was encoded host-only (device = -1)"); return CSB_ERR_UNSUPPORTED; }
+    return launch_fixed(A, Xq, ldx, batch, acc, ldy, stream);
 }
 
 int csb_view(const csb_matrix_t* A, csb_view_t* v) {
@@ -212,6 +244,7 @@ void csb_free(csb_matrix_t* A) {
     if (!A) return;
     drop_cell_plans(A);
     drop_rnn_plans(A);
+    free_fixed(A);
     free_mma(A);
     free_panels(A);
     free_product(A);
@@ -226,6 +259,7 @@ int csb_spmm(const csb_matrix_t* A, const float* X, int64_t ldx, int batch, floa
     if (!X || !Y) { set_error("X or Y is NULL"); return CSB_ERR_INVALID_ARG; }
     if (ldx < A->cols || ldy < A->rows) { set_error("ldx=%lld < cols or ldy=%lld < rows", (long long)ldx, (long long)ldy); return CSB_ERR_SHAPE; }
     if (A->device < 0) { set_error("matrix was encoded host-only (device = -1)"); return CSB_ERR_UNSUPPORTED; }
+    if (A->val_dtype == CSB_Q16) { set_error("fixed-point handles serve csb_spmm_q16 only"); return CSB_ERR_UNSUPPORTED; }
     return product_any(A, X, ldx, batch, Y, ldy, stream);
 }
 

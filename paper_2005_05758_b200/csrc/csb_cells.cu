@@ -189,6 +189,10 @@ static int cell_forward(int kind, int L, const csb_matrix_t* const* W, const csb
                       l, (long long)W[l]->rows, (long long)W[l]->cols, W[l]->device, G * H, S, S);
             return CSB_ERR_SHAPE;
         }
+        if (W[l]->val_dtype == CSB_Q16 || (kind == kCellLstmp && Wp[l]->val_dtype == CSB_Q16)) {
+            set_error("layer %d holds fixed-point values: those serve csb_spmm_q16 only", l);
+            return CSB_ERR_UNSUPPORTED;
+        }
         if (kind == kCellLstmp && (Wp[l]->rows != S || Wp[l]->cols != H || Wp[l]->device != W[0]->device)) {
             set_error("layer %d: projection is %lld x %lld; expected %d x %d on the same device", l, (long long)Wp[l]->rows, (long long)Wp[l]->cols, S, H);
             return CSB_ERR_SHAPE;

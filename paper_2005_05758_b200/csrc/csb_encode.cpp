@@ -41,6 +41,15 @@ static uint16_t f32_to_f16_rne(float f) {
     return (uint16_t)(sign | q);
 }
 
+// binary32 -> 16-bit fixed point with `frac_bits` fraction bits: the nearest integer to w * 2^frac_bits,
+// halves to the even one, saturated to the int16 range; NaN becomes 0.  (The scaling by a power of
+// two is exact in double precision, nearbyint rounds to nearest-even in the default rounding mode.)
+static int16_t f32_to_q16(float w, int frac_bits) {
+    if (w != w) return 0;
+    const double q = std::nearbyint(std::ldexp((double)w, frac_bits));
+    return (int16_t)(q < -32768.0 ? -32768.0 : q > 32767.0 ? 32767.0 : q);
+}
+
 int encode_host(const float* dense, int64_t rows, int64_t cols, int64_t ld, int br, int bc,
                 const uint8_t* row_keep, const uint8_t* col_keep, int val_dtype, csb_matrix* A) {
     A->rows = rows; A->cols = cols; A->block_r = br; A->block_c = bc; A->val_dtype = val_dtype;
@@ -90,6 +99,7 @@ int encode_host(const float* dense, int64_t rows, int64_t cols, int64_t ld, int 
                     for (int k = 0; k < n; ++k) {
                         const float w = src[ci[k]];
                         if (vs == 4) std::memcpy(v, &w, 4);
+                        else if (val_dtype == CSB_Q16) { const int16_t q = f32_to_q16(w, A->q_frac_bits); std::memcpy(v, &q, 2); }
                         else { const uint16_t h = f32_to_f16_rne(w); std::memcpy(v, &h, 2); }
                         v += vs;
                     }

@@ -108,6 +108,7 @@ struct Planner;                            // csb_plan.cpp
 struct RnnPlan;                            // csb_rnn.cu
 struct MmaPlan;                            // tensor-core SpMM plan (below)
 struct PanelPlan;                          // panel layout of the batch-1 product (below)
+struct FixedPlan;                          // fixed-point product (csb_fixed.cu)
 
 }  // namespace csb
 
@@ -117,6 +118,7 @@ struct csb_matrix {
     int block_r = 0, block_c = 0;
     int64_t nbr = 0, nbc = 0, nblk = 0, nnz = 0;
     int val_dtype = CSB_F16;
+    int q_frac_bits = 0;                   // CSB_Q16: fraction bits of the stored values
     int device = -1;
     csb_plan_opts opts{};
     // canonical arrays (Section 3.1.1 + offsets)
@@ -130,6 +132,7 @@ struct csb_matrix {
     mutable csb::MmaPlan* mma = nullptr;   // tensor-core SpMM plan, built lazily
     mutable std::mutex mma_mu;
     csb::PanelPlan* panel = nullptr;       // panel layout for batch 1 (fp16 values), or NULL
+    csb::FixedPlan* fixed = nullptr;       // device copy of the canonical arrays (CSB_Q16 handles)
     int sm_count = 0;
     size_t smem_optin = 0;
     uint64_t uid = 0;                      // identity for the recurrent-plan cache
@@ -137,7 +140,7 @@ struct csb_matrix {
 
 namespace csb {
 
-inline int val_size(int dt) { return dt == CSB_F16 ? 2 : 4; }
+inline int val_size(int dt) { return dt == CSB_F32 ? 4 : 2; }
 inline int rows_per_word(int dt) { return dt == CSB_F16 ? 2 : 1; }
 inline int max_item_rows(int dt) { return dt == CSB_F16 ? 64 : 32; }
 
@@ -323,6 +326,11 @@ int launch_product(const csb_matrix* A, const float* X, int64_t ldx, int batch, 
 int product_any(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream);
 // A new handle (same device, planned) holding block-rows [bi0, bi1) of A; the caller frees it with csb_free.
 int slice_block_rows(const csb_matrix* A, int64_t bi0, int64_t bi1, csb_matrix** out);
+
+// csb_fixed.cu -- 16-bit fixed-point product straight from the canonical arrays
+int plan_fixed(csb_matrix* A);
+void free_fixed(csb_matrix* A);
+int launch_fixed(const csb_matrix* A, const int16_t* Xq, int64_t ldx, int batch, int64_t* acc, int64_t ldy, void* stream);
 
 // csb_cells.cu
 void drop_cell_plans(const csb_matrix* A); // forget cached plans of the cell variants that use A

@@ -550,5 +550,6 @@ extern "C" int csb_spmv_static_scratch(const csb_matrix_t* A, const float* x, fl
     csb::clear_error();
     if (!A || !x || !y) { csb::set_error("A, x or y is NULL"); return CSB_ERR_INVALID_ARG; }
     if (A->device < 0) { csb::set_error("matrix was encoded host-only (device = -1)"); return CSB_ERR_UNSUPPORTED; }
+    if (A->val_dtype == CSB_Q16) { csb::set_error("fixed-point handles serve csb_spmm_q16 only"); return CSB_ERR_UNSUPPORTED; }
     return csb::launch_spmv_static_scratch(A, x, y, stream);
 }

@@ -805,6 +805,7 @@ static int rnn_forward(int gates, int L, const csb_matrix_t* const* W, const flo
             return CSB_ERR_SHAPE;
         }
         if (W[l]->device < 0) { set_error("layer %d was encoded host-only", l); return CSB_ERR_UNSUPPORTED; }
+        if (W[l]->val_dtype == CSB_Q16) { set_error("layer %d holds fixed-point values: those serve csb_spmm_q16 only", l); return CSB_ERR_UNSUPPORTED; }
         if (W[l]->device != W[0]->device || W[l]->val_dtype != W[0]->val_dtype) {
             set_error("layers must share device and value type");
             return CSB_ERR_UNSUPPORTED;
