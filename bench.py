@@ -517,14 +517,104 @@ def config_entry(binding, torch, dev, flush, w, steps, hbm, l2, sm_mhz, with_cpu
     return e, launches
 
 
+def cells_bench(binding, torch, dev, flush, hbm, l2, sm_mhz, with_cpu):
+    """The cell variants on the layer sizes of the paper's Table 1 (synthetic masks and weights; the
+    paper's own latencies for these models, on its FPGA, are quoted as context): microseconds per
+    timestep at batch 1, the float64 oracle beside them."""
+    from oracle import rnn_oracle as R
+    cases = [("lstmp_SR1", "lstmp", dict(I=153, H=1024, L=2, proj_size=512, lo=0.2, hi=0.35), "6.58 us per frame (Table 3, SR1, ZCU102 FPGA, int16)"),
+             ("ligru_SR3", "ligru", dict(I=39, H=512, L=2, lo=0.3, hi=0.45), None),
+             ("gru_reset_before_SR2", "gru_rb", dict(I=39, H=1024, L=2, lo=0.15, hi=0.3), "5.18 us per frame (Table 3, SR2, GRU, ZCU102 FPGA, int16)")]
+    out, launches = {}, 0
+    for name, cell, kw, ctx in cases:
+        extra = dict(proj_size=kw["proj_size"]) if cell == "lstmp" else {}
+        w = workloads.make_rnn_workload(0, cell, kw["I"], kw["H"], kw["L"], 32, 32, "uniform", lo=kw["lo"], hi=kw["hi"], T=100, B=1, w_std=0.05, **extra)
+        mats = encode_layers(binding, w, dev)
+        proj = [binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, dev) for m in w.proj] if cell == "lstmp" else []
+        S = w.proj_size if cell == "lstmp" else w.hidden_size
+        x = torch.from_numpy(w.x).cuda()
+        y = torch.empty((w.T, 1, S), device="cuda")
+        hT = torch.empty((kw["L"], 1, S), device="cuda")
+        cT = torch.empty((kw["L"], 1, w.hidden_size), device="cuda")
+
+        def fn(flags=binding.CSB_FLAG_ASYNC):
+            if cell == "lstmp":
+                binding.csb_lstmp_forward(mats, proj, None, x, None, None, y, hT, cT, flags)
+            elif cell == "ligru":
+                binding.csb_ligru_forward(mats, None, x, None, y, hT, flags)
+            else:
+                binding.csb_gru_reset_before_forward(mats, None, x, None, y, hT, flags)
+        fn(0)                                              # synchronous: raises if a device-side wait gave up
+        torch.cuda.synchronize()
+        y0 = y.cpu().numpy()
+        ms = time_calls(torch, fn, 10, 3, flush)
+        us = float(np.median(ms)) * 1e3 / w.T
+        infos = [m.info() for m in mats + proj]
+        alg = sum(i["algorithmic_bytes"] for i in infos) + sum((m.cols + m.rows) * 4 for m in w.layers + (w.proj or []))
+        per_step_launches = {"lstmp": 4, "ligru": 2, "gru_rb": 4}[cell] * kw["L"]
+        launches += 14 * w.T * per_step_launches
+        e = {"us_per_timestep": round(us, 3), "T": w.T, "B": 1, "layers": kw["L"], "nnz": sum(i["nnz"] for i in infos),
+             "algorithmic_bytes_per_step": alg, "launches_per_step": per_step_launches, "bound": "latency of %d dependent launches per step" % per_step_launches,
+             "roofline": three_rooflines(alg, us, hbm, l2, sm_mhz), "paper_context": ctx}
+        if with_cpu:
+            lay = layer_tuples(w)
+            prj = [(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype) for m in (w.proj or [])]
+            run = {"lstmp": lambda n: R.lstmp_forward(lay, prj, w.bias, w.x[:n]), "ligru": lambda n: R.ligru_forward(lay, w.bias, w.x[:n]),
+                   "gru_rb": lambda n: R.gru_reset_before_forward(lay, w.bias, w.x[:n])}[cell]
+            t0 = time.perf_counter(); run(2); t1 = time.perf_counter(); want = np.asarray(run(42)[0]); t2 = time.perf_counter()
+            floor = 1e-2 * float(np.sqrt(np.mean(want ** 2)))
+            big = np.abs(want) > floor
+            e["cpu_baseline"] = {"value": round(max((t2 - t1) - (t1 - t0), 1e-9) / 40 * 1e6, 1), "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                 "sample": "slope of the float64 oracle recurrence between 2 and 42 timesteps"}
+            e["max_rel_err"] = float(np.max(np.abs(y0[:42] - want)[big] / np.abs(want)[big]))
+        out[name] = e
+        for m in mats + proj:
+            m.free()
+    return out, launches
+
+
+def fixed_bench(binding, torch, dev, hbm, with_cpu, reps=10):
+    """The 16-bit fixed-point product on the sweep's matrices, cold (rotating copies > L2 in one CUDA
+    graph); integer work, so the check against the oracle is equality."""
+    from oracle import fixed_oracle as F
+    out, launches = [], 0
+    for rate, batch in ((4.0, 1), (4.0, 4), (25.0, 1)):
+        w = workloads.CONFIGS["cfg4"](rate=rate, B=batch)
+        m = w.matrix
+        ncopy = max(2, int(160e6 // (2 * int((m.dense != 0).sum()) // int(rate))) + 1) if False else (6 if rate < 10 else 30)
+        As = [binding.csb_encode_q16(m.dense, 64, 64, m.row_keep, m.col_keep, 16, dev) for _ in range(ncopy)]
+        Xq = torch.from_numpy(F.quantize(w.X, 12).astype(np.int16)).cuda()
+        acc = torch.zeros((batch, m.rows), dtype=torch.int64, device="cuda")
+
+        def run(n):
+            for i in range(n):
+                binding.csb_spmm_q16(As[i % ncopy], Xq, acc)
+        run(ncopy)
+        torch.cuda.synchronize()
+        exact = None
+        if with_cpu:
+            exact = bool(np.array_equal(acc.cpu().numpy(), F.spmm_q16(m.dense, 64, 64, m.row_keep, m.col_keep, 16, Xq.cpu().numpy())))
+        n = ncopy * -(-200 // ncopy)
+        us = graph_us(torch, run, n, reps)
+        launches += n * (reps + 1)
+        v = As[0].view()
+        alg = v["nnz"] * 2 + len(v["row_idx"]) + len(v["col_idx"]) + 6 * len(v["m"]) + m.cols * 2 * batch + m.rows * 8 * batch
+        out.append({"rate": rate, "batch": batch, "nnz": int(v["nnz"]), "us": round(us, 3), "algorithmic_bytes": int(alg), "GBps": round(alg / us / 1e3, 1),
+                    "frac_hbm_measured": round(alg / us / 1e3 / hbm, 4), "GMACs": round(v["nnz"] * batch / us / 1e3, 1), "equals_oracle": exact,
+                    "kernel": "csb_q16_kernel", "copies": ncopy})
+        for a in As:
+            a.free()
+    return out, launches
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="rnn,e2e,spmv,spmm,project,configs,cpu",
-                    help="comma list of: rnn (always), e2e, spmv, spmm, project, configs, cpu")
+    ap.add_argument("--sections", default="rnn,e2e,spmv,spmm,project,configs,cells,fixed,cpu",
+                    help="comma list of: rnn (always), e2e, spmv, spmm, project, configs, cells, fixed, cpu")
     ap.add_argument("--seq-len", type=int, default=512)
     ap.add_argument("--spmv-rates", default="4,8,16,25", help="pruning rates of the bare SpMV sweep")
     ap.add_argument("--spmv-reps", type=int, default=10)
@@ -666,6 +756,12 @@ def main():
             e, n_l = config_entry(binding, torch, local, flush, wc, 10, hbm, l2, sm_mhz, with_cpu, tsamp)
             line["configs"]["%s_B%d" % (name, wc.B)] = e
             launches += n_l
+    if rank == 0 and "cells" in sections:
+        line["cells"], n_l = cells_bench(binding, torch, local, flush, hbm, l2, sm_mhz, with_cpu)
+        launches += n_l
+    if rank == 0 and "fixed" in sections:
+        line["fixed_point"], n_l = fixed_bench(binding, torch, local, hbm, with_cpu)
+        launches += n_l
     line["gpu_launches"] = launches
     if rank == 0:
         print(json.dumps(line))

@@ -7,8 +7,10 @@
 // add through atomics in shared memory without giving up bit-reproducibility.
 //
 // The kernel reads the canonical arrays of Section 3.1.1 as they are (m{}, n{}, RowIdx{}, ColIdx{},
-// Val{} and the offsets), uploaded once.  A CTA owns one block-row; its warps take the blocks of the
-// block-row in turn.  For a block, every lane first fetches the inputs of "its" kept columns
+// Val{} and the offsets), uploaded once.  A CTA works for one block-row and a range of its
+// block-columns (enough ranges to fill the GPU several times over: what a warp does per block is a
+// chain of dependent loads); its warps take the blocks of the range in turn, and the CTAs of a
+// block-row add their sums into the output with 64-bit integer atomics.  For a block, every lane first fetches the inputs of "its" kept columns
 // through ColIdx (lane g of a half-warp takes columns g, g + 16, ...), then the two half-warps
 // walk the kept rows two at a time: a row's values are read with consecutive lanes on consecutive
 // columns, multiplied, summed up inside the half-warp by shuffles, and the total is added into the
@@ -43,7 +45,7 @@ struct FixedArgs {
     const int16_t* val;
     const int16_t* Xq; long long ldx;
     long long* acc; long long ldy;
-    int rows, cols, block_r, block_c, nbc, nb;
+    int rows, cols, block_r, block_c, nbc, nb, cols_per_cta;   // cols_per_cta: block-columns per CTA
 };
 
 constexpr int kFixedWarps = 8, kFixedMaxBlock = 128;
@@ -55,7 +57,8 @@ __global__ void __launch_bounds__(kFixedWarps * 32) csb_q16_kernel(const FixedAr
     const int bi = blockIdx.x;
     for (int i = threadIdx.x; i < a.block_r * BT; i += blockDim.x) s_acc[i] = 0ull;
     __syncthreads();
-    for (int bj = warp; bj < a.nbc; bj += kFixedWarps) {
+    const int bj_end = min(a.nbc, (int)(blockIdx.y + 1) * a.cols_per_cta);
+    for (int bj = blockIdx.y * a.cols_per_cta + warp; bj < bj_end; bj += kFixedWarps) {
         const long long b = (long long)bi * a.nbc + bj;
         const int m = a.m[b], n = a.n[b];
         if (!m || !n) continue;
@@ -103,7 +106,9 @@ __global__ void __launch_bounds__(kFixedWarps * 32) csb_q16_kernel(const FixedAr
     const int nrows = min(a.block_r, a.rows - bi * a.block_r);
     for (int i = threadIdx.x; i < nrows * a.nb; i += blockDim.x) {
         const int bt = i / nrows, r = i - bt * nrows;
-        a.acc[(long long)bt * a.ldy + (long long)bi * a.block_r + r] = (long long)s_acc[r * BT + bt];
+        const unsigned long long v = s_acc[r * BT + bt];
+        if (gridDim.y == 1) a.acc[(long long)bt * a.ldy + (long long)bi * a.block_r + r] = (long long)v;
+        else if (v) atomicAdd(reinterpret_cast<unsigned long long*>(a.acc + (long long)bt * a.ldy + (long long)bi * a.block_r + r), v);
     }
 }
 
@@ -164,11 +169,18 @@ int launch_fixed(const csb_matrix* A, const int16_t* Xq, int64_t ldx, int batch,
     a.cidx_off = P.d_cidx_off; a.val = P.d_val; a.ldx = ldx; a.ldy = ldy;
     a.rows = (int)A->rows; a.cols = (int)A->cols; a.block_r = A->block_r; a.block_c = A->block_c; a.nbc = (int)A->nbc;
     cudaStream_t st = (cudaStream_t)stream;
+    // ranges of block-columns per block-row: about eight CTAs per SM in all, at least one block per warp
+    const int64_t want = std::max<int64_t>(1, (int64_t)8 * A->sm_count / std::max<int64_t>(A->nbr, 1));
+    const int splits = (int)std::max<int64_t>(1, std::min<int64_t>(want, (A->nbc + kFixedWarps - 1) / kFixedWarps));
+    a.cols_per_cta = (int)((A->nbc + splits - 1) / splits);
+    const dim3 grid((unsigned)A->nbr, (unsigned)((A->nbc + a.cols_per_cta - 1) / a.cols_per_cta));
+    if (grid.y > 1)                                       // the CTAs of a block-row add into the output: it starts from zero
+        CSB_CUDA(cudaMemset2DAsync(acc, (size_t)ldy * 8, 0, (size_t)A->rows * 8, (size_t)batch, st));
     for (int b0 = 0; b0 < batch;) {
         const int left = batch - b0;
         a.Xq = Xq + (int64_t)b0 * ldx; a.acc = (long long*)acc + (int64_t)b0 * ldy;
-        if (left >= 2) { a.nb = std::min(4, left); csb_q16_kernel<4><<<(unsigned)A->nbr, kFixedWarps * 32, 0, st>>>(a); }
-        else { a.nb = 1; csb_q16_kernel<1><<<(unsigned)A->nbr, kFixedWarps * 32, 0, st>>>(a); }
+        if (left >= 2) { a.nb = std::min(4, left); csb_q16_kernel<4><<<grid, kFixedWarps * 32, 0, st>>>(a); }
+        else { a.nb = 1; csb_q16_kernel<1><<<grid, kFixedWarps * 32, 0, st>>>(a); }
         CSB_CUDA(cudaGetLastError());
         b0 += a.nb;
     }
