@@ -51,7 +51,7 @@ struct SpmmArgs {
     uint32_t* status;
     int nb, rows, cols, block_r, block_c, tile_cols, RG, S, x_depth, w_stages, pitch, tile_bytes;   // tile_cols: matrix columns per input tile
 #ifdef CSB_SPMM_CLOCKS
-    long long* clocks;         // instrumented build only: [CTA][warp][8] cycles per phase
+    long long* clocks;         // instrumented build only: [CTA][warp][12] cycles per phase
 #endif
 };
 
@@ -63,9 +63,14 @@ struct SpmmArgs {
 
 // Shared-memory carve-up, identical on host and device.  The small fixed part comes first; the two
 // rings follow and are reused for the warps' partial sums once the main loop is over.
+// Floats per row of a warp's sums in shared memory: the fragments go in with 8-byte stores and a row
+// comes out with 16-byte loads, both without bank conflicts at this pitch.
+__host__ __device__ constexpr int spmm_sum_pitch(int NT) { return NT == 1 ? 8 : 8 * NT + 8; }
+__host__ __device__ constexpr size_t spmm_q_bytes(int NT, int group_rows) { return (size_t)8 * NT * (group_rows + 1) * 4; }
+
 struct SpmmSmem {
     size_t wfull, xfull, wcnt, xcnt, dead, zero, rings, wring, xring, qsums, total;
-    // q_bytes: room for the CTA's own sums of its row group when a cluster shares the group (else 0)
+    // q_bytes: room for the CTA's own sums of its row group
     __host__ __device__ SpmmSmem(int n_warps, int w_stages, int x_depth, int tile_bytes, int pitch, int MT, int NT, size_t q_bytes) {
         const int n_streams = n_warps;
         wfull = 0;
@@ -78,7 +83,7 @@ struct SpmmSmem {
         wring = rings;
         xring = wring + (size_t)n_streams * w_stages * kSpmmStageBytes;
         const size_t ring_end = xring + (size_t)x_depth * tile_bytes;
-        qsums = (rings + (size_t)n_warps * MT * 16 * (NT * 8 + 1) * 4 + 127) & ~(size_t)127;
+        qsums = (rings + (size_t)n_warps * MT * 16 * spmm_sum_pitch(NT) * 4 + 127) & ~(size_t)127;
         const size_t sums_end = qsums + q_bytes;
         total = ring_end > sums_end ? ring_end : sums_end;
     }
@@ -141,6 +146,14 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
     asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
     return v;
 }
+// n / d for 0 <= n < 2^23 through the reciprocal inv = 1 / d (a handful of instructions where the
+// integer division is a few dozen; the epilogue divides several times per output)
+__device__ __forceinline__ int div_small(int n, int d, float inv) {
+    int q = __float2int_rz(__int2float_rn(n) * inv);
+    if (q * d > n) --q;
+    else if ((q + 1) * d <= n) ++q;
+    return q;
+}
 __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
@@ -153,7 +166,7 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     pdl_launch_dependents();
     extern __shared__ __align__(128) uint8_t smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const SpmmSmem L(kSpmmWarps, a.w_stages, a.x_depth, a.tile_bytes, a.pitch, MT, NT, a.S > 1 ? (size_t)8 * NT * a.RG * a.block_r * 4 : 0);
+    const SpmmSmem L(kSpmmWarps, a.w_stages, a.x_depth, a.tile_bytes, a.pitch, MT, NT, spmm_q_bytes(NT, a.RG * a.block_r));
     uint64_t* wfull = reinterpret_cast<uint64_t*>(smem + L.wfull) + warp * a.w_stages;
     uint64_t* xfull = reinterpret_cast<uint64_t*>(smem + L.xfull);
     uint32_t* xcnt = reinterpret_cast<uint32_t*>(smem + L.xcnt);
@@ -163,7 +176,7 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     const uint32_t zero_addr = smem_u32(smem + L.zero);
 
 #ifdef CSB_SPMM_CLOCKS
-    long long sprof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    long long sprof[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     long long st_ = clock64();
 #endif
     // the CTA's descriptor goes to shared memory, one word per thread
@@ -382,8 +395,8 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     }
 
     // ---- the warps' sums meet in shared memory (the rings are no longer in use)
-    constexpr int kP = NT * 8 + 1;                         // floats per row: odd, so that a column read is conflict-free
-    float* P = reinterpret_cast<float*>(smem + L.rings);
+    constexpr int kP = spmm_sum_pitch(NT);
+    float* P = reinterpret_cast<float*>(smem + L.rings);           // [warp][row of the block][kP]
     {
         float* Pw = P + (size_t)warp * MT * 16 * kP;
 #pragma unroll
@@ -391,85 +404,78 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 float* q = Pw + (16 * mt + g) * kP + 8 * nt + 2 * t;
-                q[0] = acc[mt][nt][0]; q[1] = acc[mt][nt][1];
-                q[8 * kP] = acc[mt][nt][2]; q[8 * kP + 1] = acc[mt][nt][3];
+                *reinterpret_cast<float2*>(q) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+                *reinterpret_cast<float2*>(q + 8 * kP) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
             }
     }
     __syncthreads();
+    SPMM_LAP(7);                                   // accumulators to shared memory
     const int group_rows = a.RG * a.block_r, row0 = me->group * group_rows;
     const int nrows = min(group_rows, a.rows - row0);
-    constexpr int cap = 8 * NT;
-    float* part = a.S > 1 ? reinterpret_cast<float*>(smem + L.qsums) : nullptr;    // [batch column][row of the group], this CTA's range only
+    // this CTA's sums over its range: [batch column][row of the group], one float of padding per column
+    // (written four columns at a time without bank conflicts, read by the cluster in runs of consecutive rows)
+    float* part = reinterpret_cast<float*>(smem + L.qsums);
+    const int kQ = group_rows + 1;
     {
-        // four outputs per thread at a time; the warps of a block-row are added in warp order
-        const int total = dead ? 0 : nrows * a.nb;
-        for (int i0 = threadIdx.x; i0 < total; i0 += 4 * blockDim.x) {
-            int bb[4], rl[4], w0[4], w1[4], rin[4];
-            float sum[4];
-            int wmax = 0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int idx = min(i0 + j * (int)blockDim.x, total - 1);
-                bb[j] = idx / nrows; rl[j] = idx - bb[j] * nrows;
-                const int rr = rl[j] / a.block_r;
-                rin[j] = rl[j] - rr * a.block_r;
-                w0[j] = s_first[rr]; w1[j] = s_first[rr + 1];
-                wmax = max(wmax, w1[j] - w0[j]);
-                sum[j] = 0.f;
+        // one thread per row and four batch columns; the warps of a block-row are added in warp order
+        constexpr int kQuads = 2 * NT;
+        const int total = dead ? 0 : nrows * kQuads;
+        const float inv_br = 1.f / (float)a.block_r;
+        for (int i = threadIdx.x; i < total; i += blockDim.x) {
+            const int rl = i / kQuads, q4 = i % kQuads;
+            const int rr = div_small(rl, a.block_r, inv_br), rin = rl - rr * a.block_r;
+            const int w0 = s_first[rr], w1 = s_first[rr + 1];
+            const float* src = P + ((size_t)w0 * MT * 16 + rin) * kP + 4 * q4;
+            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int k = w0; k < w1; ++k, src += MT * 16 * kP) {
+                const float4 v = *reinterpret_cast<const float4*>(src);
+                sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
             }
-            for (int k = 0; k < wmax; ++k) {
-                float v[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) v[j] = w0[j] + k < w1[j] ? P[((size_t)(w0[j] + k) * MT * 16 + rin[j]) * kP + bb[j]] : 0.f;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) sum[j] += v[j];
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (i0 + j * (int)blockDim.x < total) {
-                    if (part) part[(size_t)bb[j] * group_rows + rl[j]] = sum[j];
-                    else a.Y[(long long)bb[j] * a.ldy + row0 + rl[j]] = sum[j];
-                }
+            float* dst = part + 4 * q4 * kQ + rl;
+            dst[0] = sum.x; dst[kQ] = sum.y; dst[2 * kQ] = sum.z; dst[3 * kQ] = sum.w;
         }
     }
-    if (part) {
-        // The S CTAs of a row group form a thread-block cluster.  Once all of them have their sums in
-        // shared memory, every CTA adds up the S ranges, in range order, for its share of the group's
-        // rows, reading the other CTAs' sums through distributed shared memory; nobody leaves before
-        // everybody has read.  (The CTA barriers in front keep each warp together for the aligned cluster barrier.)
-        __syncthreads();
-        cluster_barrier();
-        const uint32_t rank = cluster_rank();
+    __syncthreads();
+    SPMM_LAP(8);                                   // sums over the warps of a block-row
+    // The S CTAs of a row group form a thread-block cluster.  Once all of them have their sums in shared
+    // memory, every CTA adds up the S ranges, in range order, for its share of the group's rows, reading
+    // the other CTAs' sums through distributed shared memory; nobody leaves before everybody has read.
+    // (The CTA barriers in front keep each warp together for the aligned cluster barrier.)
+    if (a.S > 1) cluster_barrier();
+    SPMM_LAP(9);                                   // waiting for the cluster's other CTAs
+    {
+        const uint32_t rank = a.S > 1 ? cluster_rank() : 0u;
         const int share = (nrows + a.S - 1) / a.S, r_lo = min(nrows, (int)rank * share), r_n = min(nrows, r_lo + share) - r_lo;
         const uint32_t q_local = smem_u32(part);
-        const int total = dead ? 0 : r_n * a.nb;
-        for (int i0 = threadIdx.x; i0 < total; i0 += 4 * blockDim.x) {
-            int bb[4], rl[4];
-            float sum[4];
+        uint32_t q_of[8];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int idx = min(i0 + j * (int)blockDim.x, total - 1);
-                bb[j] = idx / r_n; rl[j] = r_lo + idx - bb[j] * r_n;
-                sum[j] = 0.f;
+        for (int s2 = 0; s2 < 8; ++s2) q_of[s2] = a.S > 1 && s2 < a.S ? map_to_cluster_cta(q_local, (uint32_t)s2) : q_local;
+        // a warp takes batch columns, its lanes consecutive rows: stores of 128 contiguous bytes
+        for (int b = warp; b < (dead ? 0 : a.nb); b += kSpmmWarps)
+            for (int r = lane; r < r_n; r += 32) {
+                const uint32_t off = (uint32_t)(b * kQ + r_lo + r) * 4u;
+                float sum;
+                if (a.S > 1) {
+                    float v[8];
+#pragma unroll
+                    for (int s2 = 0; s2 < 8; ++s2) v[s2] = s2 < a.S ? ld_cluster_f32(q_of[s2] + off) : 0.f;
+                    sum = v[0];
+#pragma unroll
+                    for (int s2 = 1; s2 < 8; ++s2) sum += v[s2];
+                } else {
+                    sum = part[b * kQ + r_lo + r];
+                }
+                a.Y[(long long)b * a.ldy + row0 + r_lo + r] = sum;
             }
-            for (int s2 = 0; s2 < a.S; ++s2) {
-                const uint32_t q_remote = map_to_cluster_cta(q_local, (uint32_t)s2);
-                float v[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) v[j] = ld_cluster_f32(q_remote + (uint32_t)(bb[j] * group_rows + rl[j]) * 4u);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) sum[j] += v[j];
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (i0 + j * (int)blockDim.x < total) a.Y[(long long)bb[j] * a.ldy + row0 + rl[j]] = sum[j];
-        }
+    }
+    SPMM_LAP(10);                                  // sums over the ranges, store
+    if (a.S > 1) {
         __syncthreads();
         cluster_barrier();
     }
-    SPMM_LAP(7);                                   // sums of the warps, partial sums of the ranges, store
+    SPMM_LAP(11);                                  // until every CTA of the cluster has read
 #ifdef CSB_SPMM_CLOCKS
-    if (lane == 0) for (int i = 0; i < 8; ++i) a.clocks[((size_t)blockIdx.x * kSpmmWarps + warp) * 8 + i] = sprof[i];
+    if (lane == 0) for (int i = 0; i < 12; ++i) a.clocks[((size_t)blockIdx.x * kSpmmWarps + warp) * 12 + i] = sprof[i];
 #endif
 }
 
@@ -529,7 +535,7 @@ static int build_spmm_plan(const csb_matrix* A, int ci, MmaPlan::PerClass* P) {
     size_t smem = 0;
     for (int ws = 3; ws >= 2 && !x_depth; --ws)
         for (int xd = std::min(8, std::max(2, H.max_tiles)); xd >= 2; --xd) {
-            const SpmmSmem L(spmm_warps(NT), ws, xd, tile_bytes, pitch, MT, NT, H.S > 1 ? (size_t)8 * NT * H.RG * A->block_r * 4 : 0);
+            const SpmmSmem L(spmm_warps(NT), ws, xd, tile_bytes, pitch, MT, NT, spmm_q_bytes(NT, H.RG * A->block_r));
             if (L.total + kSpmmStaticSmem <= A->smem_optin) { w_stages = ws; x_depth = xd; smem = L.total; break; }
         }
     if (!x_depth) { P->unusable = true; return CSB_OK; }
@@ -579,7 +585,7 @@ void free_mma(csb_matrix* A) {
 static long long* g_spmm_clocks = nullptr;
 static int g_spmm_clock_warps = 0;
 extern "C" int csb_debug_spmm_clocks(long long* host_out, int max_warps) {
-    cudaMemcpy(host_out, g_spmm_clocks, (size_t)std::min(max_warps, g_spmm_clock_warps) * 8 * 8, cudaMemcpyDeviceToHost);
+    cudaMemcpy(host_out, g_spmm_clocks, (size_t)std::min(max_warps, g_spmm_clock_warps) * 12 * 8, cudaMemcpyDeviceToHost);
     return g_spmm_clock_warps;
 }
 #endif

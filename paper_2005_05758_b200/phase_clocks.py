@@ -10,7 +10,7 @@ build.py), loads it instead of libcsb.so and prints
          (mean / min / max over the CTAs);
   panel: wall-clock stamps of csb_panel_kernel per CTA, in microseconds from the earliest CTA start;
   spmm:  cycles per phase of csb_spmm_tile_kernel, summed per warp (mean / max over the warps, and the
-         same for the slowest CTA).
+         same for the slowest CTA, and the warp that finishes its items last).
 The instrumented kernels are slower than the product ones (thread 0 reads the clock between phases),
 so these figures say where the time goes, never how long a call takes.
 """
@@ -98,7 +98,8 @@ def panel(rates):
 
 SPMM_PHASES = ["set-up, first copies, wait for the work in front", "waiting for weights", "passing tiles, waiting for the item's tile",
                "row map, operand loads, tensor instructions", "ring bookkeeping, item headers", "tiles behind the last item",
-               "waiting for the CTA's other warps", "warp sums, range sums, store"]
+               "waiting for the CTA's other warps", "accumulators to shared memory", "sums over the warps of a block-row",
+               "waiting for the cluster's other CTAs", "sums over the ranges, store", "until the cluster's CTAs have read"]
 
 
 def spmm(cases):
@@ -114,15 +115,17 @@ def spmm(cases):
         for i in range(6):
             binding.csb_spmm(As[i % 3], X, Y)
             torch.cuda.synchronize()
-        ck = np.zeros((1 << 16, 8), np.int64)
+        ck = np.zeros((1 << 16, 12), np.int64)
         n = binding.lib.csb_debug_spmm_clocks(C.c_void_p(ck.ctypes.data), 1 << 16)
         ck = ck[:n].astype(np.float64)
         wpc = 32 if int(B) <= 8 else 16
-        per_cta = ck.reshape(-1, wpc, 8)
+        per_cta = ck.reshape(-1, wpc, 12)
         slow = per_cta[np.argmax(per_cta.sum(axis=2).max(axis=1))]
+        last = ck[np.argmax(ck[:, :6].sum(axis=1))]      # the warp that reaches the end of its items last
         print("cfg4 rate %sx batch %s: %d warps (%d per CTA); cycles per phase, last pass of 32 batch columns" % (rate, B, n, wpc))
         for i, nm in enumerate(SPMM_PHASES):
-            print("   %-52s mean %8.0f  max %8.0f   slowest CTA: mean %8.0f  max %8.0f" % (nm, ck[:, i].mean(), ck[:, i].max(), slow[:, i].mean(), slow[:, i].max()))
+            print("   %-52s mean %8.0f  min %8.0f  max %8.0f   slowest CTA: mean %8.0f  max %8.0f   last warp %8.0f"
+                  % (nm, ck[:, i].mean(), ck[:, i].min(), ck[:, i].max(), slow[:, i].mean(), slow[:, i].max(), last[i]))
         print("   %-52s mean %8.0f  max %8.0f" % ("all phases", ck.sum(axis=1).mean(), ck.sum(axis=1).max()))
         for a in As:
             a.free()
