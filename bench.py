@@ -581,8 +581,9 @@ def fixed_bench(binding, torch, dev, hbm, with_cpu, reps=10):
     for rate, batch in ((4.0, 1), (4.0, 4), (25.0, 1)):
         w = workloads.CONFIGS["cfg4"](rate=rate, B=batch)
         m = w.matrix
-        ncopy = max(2, int(160e6 // (2 * int((m.dense != 0).sum()) // int(rate))) + 1) if False else (6 if rate < 10 else 30)
-        As = [binding.csb_encode_q16(m.dense, 64, 64, m.row_keep, m.col_keep, 16, dev) for _ in range(ncopy)]
+        A0 = binding.csb_encode_q16(m.dense, 64, 64, m.row_keep, m.col_keep, 16, dev)
+        ncopy = max(2, int(160e6 // max(A0.info()["algorithmic_bytes"], 1)) + 1)      # rotating copies larger than L2
+        As = [A0] + [binding.csb_encode_q16(m.dense, 64, 64, m.row_keep, m.col_keep, 16, dev) for _ in range(ncopy - 1)]
         Xq = torch.from_numpy(F.quantize(w.X, 12).astype(np.int16)).cuda()
         acc = torch.zeros((batch, m.rows), dtype=torch.int64, device="cuda")
 
@@ -618,7 +619,7 @@ def main():
     ap.add_argument("--seq-len", type=int, default=512)
     ap.add_argument("--spmv-rates", default="4,8,16,25", help="pruning rates of the bare SpMV sweep")
     ap.add_argument("--spmv-reps", type=int, default=10)
-    ap.add_argument("--spmm-batches", default="8,64", help="batch sizes of the SpMM sweep (section spmm)")
+    ap.add_argument("--spmm-batches", default="8,32,64", help="batch sizes of the SpMM sweep (section spmm)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -738,11 +739,12 @@ def main():
         for bsz in [int(b) for b in args.spmm_batches.split(",")]:
             res, n_l = spmv_sweep(binding, torch, local, rates, bsz, l2, reps=args.spmv_reps, with_cpu=with_cpu)
             line["spmm"] += res
-            launches += 2 * n_l
+            launches += 2 * -(-bsz // 32) * n_l          # per pass of 32 batch columns: the pack kernel and the product kernel
         best = max(line["spmm"], key=lambda r: r["frac_hbm_measured"])
         line["roofline_spmm"] = {"kernel": "csb_spmm_tile_kernel", "bound": "hbm", "achieved": best["GBps"], "peak": hbm, "peak_kind": peak_kind,
                                  "unit": "GB/s", "frac": best["frac_hbm_measured"],
                                  "traffic": counters.get("csb_spmm_tile_kernel cfg4 4x B=64") if (best["rate"] == 4.0 and best["batch"] == 64) else None,
+                                 "traffic_per_pass_4x_batch64": counters.get("csb_spmm_tile_kernel cfg4 4x B=64"),
                                  "workload": "cfg4 8192x8192, 64x64 blocks, rate %gx, batch %d, cold" % (best["rate"], best["batch"])}
     if rank == 0 and "project" in sections:
         line["project"] = project_bench(binding, torch)

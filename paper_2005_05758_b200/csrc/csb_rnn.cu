@@ -139,8 +139,14 @@ __device__ __forceinline__ unsigned int ld_relaxed_u32(const unsigned int* p) {
 //      step (batch 1 only).  With lag 2 the layer below produced u_{t+1} a full tick ago, so that
 //      needs nothing from the barrier it has just arrived at.
 // h of step s of a layer lives in slot s & 3 of a four-slot ring in global memory.
+// Most warps a CTA of the time loop may have; the register budget of the kernel follows from it.
+#ifndef CSB_RNN_MAX_WARPS
+#define CSB_RNN_MAX_WARPS 16
+#endif
+constexpr int kRnnMaxWarps = CSB_RNN_MAX_WARPS;
+
 template <typename T, int BT, int GW, bool RES>
-__global__ void __launch_bounds__(512, 1) csb_rnn_kernel(const RnnArgs a) {
+__global__ void __launch_bounds__(kRnnMaxWarps * 32, 1) csb_rnn_kernel(const RnnArgs a) {
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int G = 32 / GW;
     const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -687,7 +693,7 @@ static int build_rnn_plan(int gates, int L, const csb_matrix* const* W, int B, i
     P->gates = gates; P->L = L; P->B = B; P->H = H; P->device = A0->device; P->val_dtype = A0->val_dtype;
     for (int l = 0; l < L; ++l) { P->uids.push_back(W[l]->uid); P->in_size[l] = in_size[l]; P->max_C = std::max(P->max_C, in_size[l] + H); }
     P->BT = B == 1 ? 1 : (B <= 4 ? 4 : 8);
-    P->warps = std::min(16, std::max(1, env_int("CSB_RNN_WARPS", 16)));
+    P->warps = std::min(kRnnMaxWarps, std::max(1, env_int("CSB_RNN_WARPS", 16)));
     P->stage_bytes = 3072; P->stages = 3;
     int64_t approx = 0;
     for (int l = 0; l < L; ++l) approx += W[l]->nnz * val_size(W[l]->val_dtype) + 32 * W[l]->nblk;

@@ -80,11 +80,17 @@ def panel(rates):
         m = w.matrix
         A = binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, 0)
         n = A.info()["panel_ctas"]
+        # cold the way a stream of different products is cold: rotate through encoded copies whose
+        # total exceeds L2 (a flush by writing would leave HBM busy with write-backs), the stamped
+        # launch last and alone
+        ncopy = max(2, int(200e6 // max(A.info()["algorithmic_bytes"], 1)) + 1)
+        others = [binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, 0) for _ in range(ncopy - 1)]
         x = torch.from_numpy(w.X).cuda()
         y = torch.empty(m.rows, device="cuda")
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
         for _ in range(3):
-            flush.zero_()
+            for o in others:
+                binding.csb_spmv(o, x[0], y)
+            torch.cuda.synchronize()
             binding.csb_spmv(A, x[0], y)
             torch.cuda.synchronize()
         ck = np.zeros((n, 8), np.uint64)
@@ -93,7 +99,8 @@ def panel(rates):
         print("cfg4 rate %sx: %d CTAs, stamps in us from the earliest CTA start (cold L2)" % (rate, n))
         for i, nm in enumerate(PANEL_STAMPS[:6]):
             print("   %-34s mean %6.2f  min %6.2f  max %6.2f" % (nm, t[:, i].mean(), t[:, i].min(), t[:, i].max()))
-        A.free()
+        for o in others + [A]:
+            o.free()
 
 
 SPMM_PHASES = ["set-up, first copies, wait for the work in front", "waiting for weights", "passing tiles, waiting for the item's tile",
