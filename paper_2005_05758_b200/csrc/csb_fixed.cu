@@ -10,10 +10,11 @@
 // Val{} and the offsets), uploaded once.  A CTA works for one block-row and a range of its
 // block-columns (enough ranges to fill the GPU several times over: what a warp does per block is a
 // chain of dependent loads); its warps take the blocks of the range in turn, and the CTAs of a
-// block-row add their sums into the output with 64-bit integer atomics.  For a block, every lane first fetches the inputs of "its" kept columns
-// through ColIdx (lane g of a half-warp takes columns g, g + 16, ...), then the two half-warps
-// walk the kept rows two at a time: a row's values are read with consecutive lanes on consecutive
-// columns, multiplied, summed up inside the half-warp by shuffles, and the total is added into the
+// block-row add their sums into the output with 64-bit integer atomics.  For a block, the lanes first
+// fetch the inputs behind the kept columns through ColIdx (lane g holds columns g, g + 32, ...); then
+// every lane owns one kept row of the kernel matrix (32 rows at a time) and walks it column by column:
+// its own weight times the column's input, handed round by a shuffle, into a 64-bit sum (one
+// multiply-add with a wide result per weight, no reduction across lanes); the sum is added into the
 // block-row's accumulators through RowIdx.
 #include <algorithm>
 
@@ -53,7 +54,7 @@ constexpr int kFixedWarps = 8, kFixedMaxBlock = 128;
 template <int BT>
 __global__ void __launch_bounds__(kFixedWarps * 32) csb_q16_kernel(const FixedArgs a) {
     __shared__ unsigned long long s_acc[kFixedMaxBlock * BT];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, g = lane & 15;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bi = blockIdx.x;
     for (int i = threadIdx.x; i < a.block_r * BT; i += blockDim.x) s_acc[i] = 0ull;
     __syncthreads();
@@ -65,40 +66,38 @@ __global__ void __launch_bounds__(kFixedWarps * 32) csb_q16_kernel(const FixedAr
         const uint8_t* ci = a.cidx + a.cidx_off[b];
         const uint8_t* ri = a.ridx + a.ridx_off[b];
         const int16_t* v = a.val + a.val_off[b];
-        // the inputs behind this lane's kept columns g, g + 16, ... (up to 8 of them: blocks are at most 128 wide)
-        int xk[8][BT];
+        // the inputs behind kept columns lane, lane + 32, ... (up to 4 of them: blocks are at most 128 wide)
+        int xk[4][BT];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int k = g + 16 * j;
+        for (int j = 0; j < 4; ++j) {
+            const int k = lane + 32 * j;
+            const long long col = (long long)bj * a.block_c + (k < n ? (int)ci[k] : 0);
 #pragma unroll
-            for (int bt = 0; bt < BT; ++bt)
-                xk[j][bt] = (k < n && bt < a.nb) ? (int)a.Xq[(long long)bt * a.ldx + (long long)bj * a.block_c + ci[k]] : 0;
+            for (int bt = 0; bt < BT; ++bt) xk[j][bt] = (k < n && bt < a.nb) ? (int)a.Xq[(long long)bt * a.ldx + col] : 0;
         }
-        for (int r0 = 0; r0 < m; r0 += 2) {
-            const int r = r0 + half;
+        for (int r0 = 0; r0 < m; r0 += 32) {
+            const int r = r0 + lane;
+            const bool live = r < m;
+            const int16_t* row = v + (long long)(live ? r : 0) * n;
             long long sum[BT];
 #pragma unroll
             for (int bt = 0; bt < BT; ++bt) sum[bt] = 0;
-            if (r < m) {
-                const int16_t* row = v + (long long)r * n;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int k = g + 16 * j;
-                    if (k < n) {
-                        const int w = (int)row[k];
+            for (int j = 0; j < 4; ++j) {
+                const int kn = min(32, n - 32 * j);                 // warp-uniform
+#pragma unroll 4
+                for (int kk = 0; kk < kn; ++kk) {
+                    const long long w = (long long)row[32 * j + kk];
 #pragma unroll
-                        for (int bt = 0; bt < BT; ++bt) sum[bt] += (long long)(w * xk[j][bt]);     // |w * x| < 2^31: exact in 32 bits
-                    }
+                    for (int bt = 0; bt < BT; ++bt)
+                        sum[bt] += w * (long long)__shfl_sync(0xffffffffu, xk[j][bt], kk);   // 16 x 16 bits: exact
                 }
             }
+            if (live) {
+                const int out = (int)ri[r] * BT;
 #pragma unroll
-            for (int bt = 0; bt < BT; ++bt) {
-#pragma unroll
-                for (int o = 8; o > 0; o >>= 1) sum[bt] += __shfl_xor_sync(0xffffffffu, sum[bt], o, 16);
-            }
-            if (r < m && g == 0) {
-#pragma unroll
-                for (int bt = 0; bt < BT; ++bt) atomicAdd(&s_acc[(int)ri[r] * BT + bt], (unsigned long long)sum[bt]);
+                for (int bt = 0; bt < BT; ++bt)
+                    if (sum[bt]) atomicAdd(&s_acc[out + bt], (unsigned long long)sum[bt]);
             }
         }
     }

@@ -261,7 +261,8 @@ struct MmaPlan {                           // device side, one per batch class, 
         double balance = 1.0, warp_balance = 1.0;
     } cls[3];
 };
-int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream);
+int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream,
+                    const uint8_t* packed = nullptr);
 bool spmm_mma_applicable(const csb_matrix* A, int batch);
 void free_mma(csb_matrix* A);
 

@@ -10,6 +10,11 @@
 // writes h_t into the right part of V_l (for step t + 1) and into the left part of V_{l+1} (the
 // layer above, same step) or into y, and the gate kernel of layer 0 also moves x_{t+1} in.
 //
+// Up to 32 product rows (LSTM: batch <= 32, GRU: batch <= 16) the fp32 buffers V_l do not exist at all:
+// the gate kernels write h_t, and the one of layer 0 also x_{t+1}, straight into the packed binary16
+// (hi, lo) input rows that the product kernel reads, transposed through shared memory so that the
+// stores of a row are contiguous; a step is then two launches per layer (product, gates).
+//
 // GRU (reset gate applied after the recurrent product) needs the input part and the recurrent part
 // of the candidate's pre-activation apart.  One product still does: V_l has 2B rows, row b holds
 // [u_t ; 0] and row B + b holds [0 ; h_{t-1}], so row b of the product is W_x u and row B + b is W_h h.
@@ -41,9 +46,15 @@ struct StepPlan {
     float* d_c = nullptr;              // [L, B, H] cell state
     float* d_stage = nullptr;          // host-I/O staging of x and y
     size_t stage_cap = 0;
+    // packed path (at most 32 product rows): per layer the packed inputs of its product, one row of
+    // `pitch` bytes per column of W_l, and the fp32 h of every layer
+    uint8_t* d_xp[kMaxLayers] = {};
+    float* d_h = nullptr;              // [L, B, H]
+    int pitch = 0, cap = 0;
     ~StepPlan() {
         for (float* p : d_v) cudaFree(p);
-        cudaFree(d_z); cudaFree(d_c); cudaFree(d_stage);
+        for (uint8_t* p : d_xp) cudaFree(p);
+        cudaFree(d_z); cudaFree(d_c); cudaFree(d_stage); cudaFree(d_h);
     }
 };
 static std::mutex g_step_mu;
@@ -131,6 +142,117 @@ __global__ void csb_gru_gates_kernel(const float* __restrict__ Z, const float* _
     }
 }
 
+// ---- the packed path -------------------------------------------------------------------------------------
+// A tile of 32 columns x nb batch values, tile[b][c], goes into slots slot0 .. slot0 + nb - 1 of the
+// packed rows of those columns: x = hi + lo, hi at [slot], lo at [cap + slot] (binary16 each).
+// Consecutive threads take consecutive batch values of a column, so a row's stores are contiguous.
+__device__ __forceinline__ void pack_tile(const float (*tile)[33], int ncols, int nb, uint8_t* rows, int pitch, int cap, int slot0,
+                                          uint8_t* rows2, int slot2) {
+    for (int idx = threadIdx.x; idx < 32 * nb; idx += blockDim.x) {
+        const int c = idx / nb, b = idx - c * nb;
+        if (c >= ncols) break;
+        const float x = tile[b][c];
+        const __half hi = __float2half_rn(x);
+        const __half lo = __float2half_rn(x - __half2float(hi));
+        __half* r = reinterpret_cast<__half*>(rows + (size_t)c * pitch);
+        r[slot0 + b] = hi;
+        r[cap + slot0 + b] = lo;
+        if (rows2) {
+            __half* r2 = reinterpret_cast<__half*>(rows2 + (size_t)c * pitch);
+            r2[slot2 + b] = hi;
+            r2[cap + slot2 + b] = lo;
+        }
+    }
+}
+
+// src [nb, ncols] (row stride ld) -> slots slot0 .. of the packed rows 0 .. ncols - 1 of xp; 256 threads, 32 columns per block.
+__global__ void csb_pack_rows_kernel(const float* __restrict__ src, long long ld, int nb, int ncols, uint8_t* __restrict__ xp, int pitch,
+                                     int cap, int slot0) {
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5, c0 = blockIdx.x * 32;
+    for (int b = ty; b < nb; b += 8) tile[b][tx] = c0 + tx < ncols ? src[(long long)b * ld + c0 + tx] : 0.f;
+    __syncthreads();
+    pack_tile(tile, min(32, ncols - c0), nb, xp + (size_t)c0 * pitch, pitch, cap, slot0, nullptr, 0);
+}
+
+// The LSTM gate arithmetic as in csb_lstm_gates_kernel for 32 hidden units x the batch per block
+// (blocks 0 .. h_blocks - 1); h_t goes, packed, to rows j of xp_self (this layer's recurrent columns)
+// and of xp_next (the input columns of the layer above), as fp32 to hs[b, j] and y_t[b, j].  Blocks from
+// h_blocks on pack x_next [B, I] (the next step's input of layer 0) into rows of xp0.  256 threads.
+__global__ void csb_lstm_gates_pack_kernel(const float* __restrict__ Z, const float* __restrict__ bias, float* __restrict__ c,
+                                           float* __restrict__ hs, uint8_t* __restrict__ xp_self, uint8_t* __restrict__ xp_next,
+                                           float* __restrict__ y_t, const float* __restrict__ x_next, int I, uint8_t* __restrict__ xp0,
+                                           int pitch, int cap, int B, int H, int h_blocks) {
+    pdl_launch_dependents();
+    pdl_wait();                                    // Z comes from the product in front, which also still reads xp0
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    if ((int)blockIdx.x < h_blocks) {
+        const int j0 = blockIdx.x * 32, j = j0 + tx;
+        for (int b = ty; b < B; b += 8) {
+            float h = 0.f;
+            if (j < H) {
+                const float* z = Z + (size_t)b * 4 * H;
+                float zi = z[j], zf = z[H + j], zg = z[2 * H + j], zo = z[3 * H + j];
+                if (bias) { zi += bias[j]; zf += bias[H + j]; zg += bias[2 * H + j]; zo += bias[3 * H + j]; }
+                const size_t e = (size_t)b * H + j;
+                const float cn = logistic(zf) * c[e] + logistic(zi) * tanhf(zg);
+                h = logistic(zo) * tanhf(cn);
+                c[e] = cn;
+                hs[e] = h;
+                if (y_t) y_t[e] = h;
+            }
+            tile[b][tx] = h;
+        }
+        __syncthreads();
+        pack_tile(tile, min(32, H - j0), B, xp_self + (size_t)j0 * pitch, pitch, cap, 0, xp_next ? xp_next + (size_t)j0 * pitch : nullptr, 0);
+    } else {
+        const int c0 = ((int)blockIdx.x - h_blocks) * 32;
+        for (int b = ty; b < B; b += 8) tile[b][tx] = c0 + tx < I ? x_next[(size_t)b * I + c0 + tx] : 0.f;
+        __syncthreads();
+        pack_tile(tile, min(32, I - c0), B, xp0 + (size_t)c0 * pitch, pitch, cap, 0, nullptr, 0);
+    }
+}
+
+// The GRU gate arithmetic as in csb_gru_gates_kernel, same tiling.  The product has 2B rows: slots
+// 0 .. B - 1 of a packed row carry the input part (zero in the recurrent columns), slots B .. 2B - 1
+// the recurrent part (zero in the input columns); the zeros are written once, before the first step.
+__global__ void csb_gru_gates_pack_kernel(const float* __restrict__ Z, const float* __restrict__ bias, float* __restrict__ hs,
+                                          uint8_t* __restrict__ xp_self, uint8_t* __restrict__ xp_next, float* __restrict__ y_t,
+                                          const float* __restrict__ x_next, int I, uint8_t* __restrict__ xp0, int pitch, int cap, int B,
+                                          int H, int h_blocks) {
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    if ((int)blockIdx.x < h_blocks) {
+        const int j0 = blockIdx.x * 32, j = j0 + tx;
+        for (int b = ty; b < B; b += 8) {
+            float h = 0.f;
+            if (j < H) {
+                const float* zx = Z + (size_t)b * 3 * H;
+                const float* zh = Z + (size_t)(B + b) * 3 * H;
+                float ar = zx[j] + zh[j], au = zx[H + j] + zh[H + j], nx = zx[2 * H + j], nh = zh[2 * H + j];
+                if (bias) { ar += bias[j]; au += bias[H + j]; nx += bias[2 * H + j]; nh += bias[3 * H + j]; }
+                const float r = logistic(ar), u = logistic(au);
+                const float cand = tanhf(nx + r * nh);
+                const size_t e = (size_t)b * H + j;
+                h = (1.f - u) * cand + u * hs[e];
+                hs[e] = h;
+                if (y_t) y_t[e] = h;
+            }
+            tile[b][tx] = h;
+        }
+        __syncthreads();
+        pack_tile(tile, min(32, H - j0), B, xp_self + (size_t)j0 * pitch, pitch, cap, B, xp_next ? xp_next + (size_t)j0 * pitch : nullptr, 0);
+    } else {
+        const int c0 = ((int)blockIdx.x - h_blocks) * 32;
+        for (int b = ty; b < B; b += 8) tile[b][tx] = c0 + tx < I ? x_next[(size_t)b * I + c0 + tx] : 0.f;
+        __syncthreads();
+        pack_tile(tile, min(32, I - c0), B, xp0 + (size_t)c0 * pitch, pitch, cap, 0, nullptr, 0);
+    }
+}
+
 static int env_flag(const char* name) {
     const char* v = getenv(name);
     return v && *v ? atoi(v) : 0;
@@ -165,11 +287,16 @@ int rnn_forward_stepwise(int gates, int L, const csb_matrix* const* W, const flo
         if (!P) {
             std::unique_ptr<StepPlan> np(new StepPlan());
             np->L = L; np->B = B; np->H = H; np->gates = gates; np->device = W[0]->device;
+            const int rows_v = (gates == 3 ? 2 : 1) * B;
+            const bool packed_path = rows_v <= 32 && !env_flag("CSB_RNN_STEP_UNPACKED");
+            if (packed_path) { np->pitch = spmm_pitch(spmm_nt(rows_v)); np->cap = 8 * spmm_nt(rows_v); }
             for (int l = 0; l < L; ++l) {
                 np->uids.push_back(W[l]->uid);
                 np->in_size[l] = in_size[l];
-                CSB_CUDA(cudaMalloc((void**)&np->d_v[l], (size_t)(gates == 3 ? 2 : 1) * B * (in_size[l] + H) * 4));
+                if (packed_path) CSB_CUDA(cudaMalloc((void**)&np->d_xp[l], (size_t)(in_size[l] + H) * np->pitch));
+                else CSB_CUDA(cudaMalloc((void**)&np->d_v[l], (size_t)rows_v * (in_size[l] + H) * 4));
             }
+            if (packed_path) CSB_CUDA(cudaMalloc((void**)&np->d_h, (size_t)L * B * H * 4));
             CSB_CUDA(cudaMalloc((void**)&np->d_z, (size_t)(gates == 3 ? 2 : 1) * B * gates * H * 4));
             if (gates == 4) CSB_CUDA(cudaMalloc((void**)&np->d_c, (size_t)L * B * H * 4));
             P = np.get();
@@ -199,6 +326,66 @@ int rnn_forward_stepwise(int gates, int L, const csb_matrix* const* W, const flo
     const size_t hrow = (size_t)H * 4;
     const bool gru = gates == 3;
     const int vrows = gru ? 2 * B : B;                  // rows of V_l and of the product
+    if (P->pitch) {
+        // ---- packed path: the gate kernels feed the products' packed inputs directly
+        const int pitch = P->pitch, cap = P->cap;
+        if (h0) CSB_CUDA(cudaMemcpyAsync(P->d_h, h0, ns * 4, in_kind, st));
+        else CSB_CUDA(cudaMemsetAsync(P->d_h, 0, ns * 4, st));
+        for (int l = 0; l < L; ++l) {
+            CSB_CUDA(cudaMemsetAsync(P->d_xp[l], 0, (size_t)(in_size[l] + H) * pitch, st));
+            if (h0)
+                csb_pack_rows_kernel<<<(H + 31) / 32, 256, 0, st>>>(P->d_h + (size_t)l * B * H, (long long)H, B, H,
+                                                                   P->d_xp[l] + (size_t)in_size[l] * pitch, pitch, cap, gru ? B : 0);
+        }
+        csb_pack_rows_kernel<<<(I0 + 31) / 32, 256, 0, st>>>(dx, (long long)I0, B, I0, P->d_xp[0], pitch, cap, 0);
+        CSB_CUDA(cudaGetLastError());
+        if (!gru) {
+            if (c0) CSB_CUDA(cudaMemcpyAsync(P->d_c, c0, ns * 4, in_kind, st));
+            else CSB_CUDA(cudaMemsetAsync(P->d_c, 0, ns * 4, st));
+        }
+        const int h_blocks = (H + 31) / 32, x_blocks = (I0 + 31) / 32;
+        for (int64_t t = 0; t < T; ++t) {
+            for (int l = 0; l < L; ++l) {
+                const int rc = launch_spmm_mma(W[l], nullptr, 0, vrows, P->d_z, (int64_t)gates * H, stream, P->d_xp[l]);
+                if (rc != CSB_OK) {
+                    if (rc == 1 && t > 0) { set_error("the tensor-core plan of layer %d became unusable in mid-sequence", l); return CSB_ERR_CUDA; }
+                    return rc;
+                }
+                const bool top = l == L - 1;
+                const float* x_next = (l == 0 && t + 1 < T) ? dx + (size_t)(t + 1) * B * I0 : nullptr;
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+                attr[0].val.programmaticStreamSerializationAllowed = 1;
+                cudaLaunchConfig_t cfg{};
+                cfg.gridDim = dim3((unsigned)(h_blocks + (x_next ? x_blocks : 0))); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0;
+                cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 1;
+                const float* bl = bias ? bias[l] : nullptr;
+                float* hs = P->d_h + (size_t)l * B * H;
+                uint8_t* xp_self = P->d_xp[l] + (size_t)in_size[l] * pitch;
+                uint8_t* xp_next = top ? nullptr : P->d_xp[l + 1];
+                float* yt = (top && dy) ? dy + (size_t)t * B * H : nullptr;
+                if (gru)
+                    CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_gru_gates_pack_kernel, (const float*)P->d_z, bl, hs, xp_self, xp_next, yt, x_next, I0,
+                                                P->d_xp[0], pitch, cap, B, H, h_blocks));
+                else
+                    CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_lstm_gates_pack_kernel, (const float*)P->d_z, bl, P->d_c + (size_t)l * B * H, hs, xp_self,
+                                                xp_next, yt, x_next, I0, P->d_xp[0], pitch, cap, B, H, h_blocks));
+                CSB_CUDA(cudaGetLastError());
+            }
+        }
+        if (hT) CSB_CUDA(cudaMemcpyAsync(hT, P->d_h, ns * 4, out_kind, st));
+        if (cT && !gru) CSB_CUDA(cudaMemcpyAsync(cT, P->d_c, ns * 4, out_kind, st));
+        if (host_io && y) CSB_CUDA(cudaMemcpyAsync(y, dy, ny * 4, cudaMemcpyDeviceToHost, st));
+        if (host_io || !(flags & CSB_FLAG_ASYNC)) {
+            CSB_CUDA(cudaStreamSynchronize(st));
+            for (int l = 0; l < L; ++l)
+                if (W[l]->product.h_status && *W[l]->product.h_status != 0) {
+                    set_error("a product kernel of layer %d gave up a bounded wait (code %u)", l, *W[l]->product.h_status);
+                    return CSB_ERR_TIMEOUT;
+                }
+        }
+        return CSB_OK;
+    }
     // V_l = [u_0 ; h_{-1}]: h0 (or zeros) on the right, x_0 on the left of layer 0.  GRU: the
     // recurrent rows (B ..) carry h and zeros on the left, the input rows zeros on the right.
     for (int l = 0; l < L; ++l) {

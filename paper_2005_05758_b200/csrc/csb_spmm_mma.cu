@@ -421,18 +421,35 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
         constexpr int kQuads = 2 * NT;
         const int total = dead ? 0 : nrows * kQuads;
         const float inv_br = 1.f / (float)a.block_r;
-        for (int i = threadIdx.x; i < total; i += blockDim.x) {
-            const int rl = i / kQuads, q4 = i % kQuads;
-            const int rr = div_small(rl, a.block_r, inv_br), rin = rl - rr * a.block_r;
-            const int w0 = s_first[rr], w1 = s_first[rr + 1];
-            const float* src = P + ((size_t)w0 * MT * 16 + rin) * kP + 4 * q4;
-            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int k = w0; k < w1; ++k, src += MT * 16 * kP) {
-                const float4 v = *reinterpret_cast<const float4*>(src);
-                sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+        // (four of a thread's outputs at a time, so that their loads are in flight together)
+        for (int i0 = threadIdx.x; i0 < total; i0 += 4 * blockDim.x) {
+            const float* src[4];
+            int cnt[4], rl[4], q4[4], cmax = 0;
+            float4 sum[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int i = min(i0 + j * (int)blockDim.x, total - 1);
+                rl[j] = i / kQuads; q4[j] = i % kQuads;
+                const int rr = div_small(rl[j], a.block_r, inv_br), rin = rl[j] - rr * a.block_r;
+                const int w0 = s_first[rr];
+                cnt[j] = s_first[rr + 1] - w0;
+                cmax = max(cmax, cnt[j]);
+                src[j] = P + ((size_t)w0 * MT * 16 + rin) * kP + 4 * q4[j];
+                sum[j] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            float* dst = part + 4 * q4 * kQ + rl;
-            dst[0] = sum.x; dst[kQ] = sum.y; dst[2 * kQ] = sum.z; dst[3 * kQ] = sum.w;
+            for (int k = 0; k < cmax; ++k) {
+                float4 v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[j] = k < cnt[j] ? *reinterpret_cast<const float4*>(src[j] + (size_t)k * MT * 16 * kP) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { sum[j].x += v[j].x; sum[j].y += v[j].y; sum[j].z += v[j].z; sum[j].w += v[j].w; }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j * (int)blockDim.x < total) {
+                    float* dst = part + 4 * q4[j] * kQ + rl[j];
+                    dst[0] = sum[j].x; dst[kQ] = sum[j].y; dst[2 * kQ] = sum[j].z; dst[3 * kQ] = sum[j].w;
+                }
         }
     }
     __syncthreads();
@@ -451,21 +468,29 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
 #pragma unroll
         for (int s2 = 0; s2 < 8; ++s2) q_of[s2] = a.S > 1 && s2 < a.S ? map_to_cluster_cta(q_local, (uint32_t)s2) : q_local;
         // a warp takes batch columns, its lanes consecutive rows: stores of 128 contiguous bytes
-        for (int b = warp; b < (dead ? 0 : a.nb); b += kSpmmWarps)
-            for (int r = lane; r < r_n; r += 32) {
-                const uint32_t off = (uint32_t)(b * kQ + r_lo + r) * 4u;
-                float sum;
-                if (a.S > 1) {
-                    float v[8];
+        // (two batch columns x two runs of rows per lane at a time: up to 32 remote loads in flight)
+        for (int b0 = warp; b0 < (dead ? 0 : a.nb); b0 += 2 * kSpmmWarps)
+            for (int r0 = lane; r0 < r_n; r0 += 64) {
+                float v[4][8];
 #pragma unroll
-                    for (int s2 = 0; s2 < 8; ++s2) v[s2] = s2 < a.S ? ld_cluster_f32(q_of[s2] + off) : 0.f;
-                    sum = v[0];
+                for (int j = 0; j < 4; ++j) {
+                    const int b = b0 + (j >> 1) * kSpmmWarps, r = r0 + (j & 1) * 32;
+                    const bool live = b < a.nb && r < r_n;
+                    const uint32_t off = (uint32_t)(b * kQ + r_lo + r) * 4u;
 #pragma unroll
-                    for (int s2 = 1; s2 < 8; ++s2) sum += v[s2];
-                } else {
-                    sum = part[b * kQ + r_lo + r];
+                    for (int s2 = 0; s2 < 8; ++s2) {
+                        if (a.S > 1) v[j][s2] = live && s2 < a.S ? ld_cluster_f32(q_of[s2] + off) : 0.f;
+                        else v[j][s2] = live && s2 == 0 ? part[b * kQ + r_lo + r] : 0.f;
+                    }
                 }
-                a.Y[(long long)b * a.ldy + row0 + r_lo + r] = sum;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int b = b0 + (j >> 1) * kSpmmWarps, r = r0 + (j & 1) * 32;
+                    float sum = v[j][0];
+#pragma unroll
+                    for (int s2 = 1; s2 < 8; ++s2) sum += v[j][s2];
+                    if (b < a.nb && r < r_n) a.Y[(long long)b * a.ldy + row0 + r_lo + r] = sum;
+                }
             }
     }
     SPMM_LAP(10);                                  // sums over the ranges, store
@@ -591,7 +616,11 @@ extern "C" int csb_debug_spmm_clocks(long long* host_out, int max_warps) {
 #endif
 
 // Returns CSB_OK after launching, or 1 when the caller should use the CUDA-core path.
-int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream) {
+// With `packed` (and X == nullptr) the inputs are taken from a buffer the caller has filled in the
+// packed layout of the batch's class (one row of spmm_pitch(NT) bytes per matrix column: the hi parts of
+// 8 * NT batch slots, then the lo parts); a single pass, so at most 32 batch columns.
+int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream, const uint8_t* packed) {
+    if (packed && batch > 32) { set_error("pre-packed inputs serve at most 32 batch columns"); return CSB_ERR_INVALID_ARG; }
     const ProductPlan& PP = A->product;
     if (PP.h_status && *PP.h_status != 0) { set_error("an earlier product on this handle gave up waiting on the device (code %u)", *PP.h_status); return CSB_ERR_TIMEOUT; }
     int prev = 0;
@@ -619,7 +648,7 @@ int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch,
     cudaStream_t st = (cudaStream_t)stream;
     SpmmArgs a{};
     a.stream = P.d_stream; a.warp_desc = (const uint4*)P.d_warp_desc; a.ctas = P.d_ctas;
-    a.xp = (const uint8_t*)P.d_xp; a.ldy = ldy; a.status = PP.d_status;
+    a.xp = packed ? packed : (const uint8_t*)P.d_xp; a.ldy = ldy; a.status = PP.d_status;
     a.rows = (int)A->rows; a.cols = (int)A->cols; a.block_r = A->block_r; a.block_c = A->block_c;
     a.RG = P.RG; a.S = P.S; a.x_depth = P.x_depth; a.w_stages = P.w_stages;
     a.tile_cols = spmm_tile_blocks(A->block_c) * A->block_c;
@@ -642,8 +671,9 @@ int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch,
         cudaLaunchConfig_t cfg{};
         cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 1;
         cfg.gridDim = dim3((unsigned)((A->cols + 31) / 32)); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0;
-        CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_pack_x_kernel, X + (int64_t)b0 * ldx, (long long)ldx, a.nb, (int)A->cols, (uint8_t*)P.d_xp,
-                                    a.pitch, NT));
+        if (!packed)
+            CSB_CUDA(cudaLaunchKernelEx(&cfg, csb_pack_x_kernel, X + (int64_t)b0 * ldx, (long long)ldx, a.nb, (int)A->cols, (uint8_t*)P.d_xp,
+                                        a.pitch, NT));
         cfg.gridDim = dim3((unsigned)P.n_ctas); cfg.blockDim = dim3((unsigned)spmm_warps(NT) * 32u); cfg.dynamicSmemBytes = P.smem_bytes;
         cfg.numAttrs = P.S > 1 ? 2 : 1;
         CSB_CUDA(CSB_SPMM_DISPATCH(launch_tile_kernel, MT, NT, &cfg, a));

@@ -2,7 +2,7 @@
 
     python -m paper_2005_05758_b200.phase_clocks rnn   [cfg1 cfg2 cfg3 cfg5]
     python -m paper_2005_05758_b200.phase_clocks panel [4 8 16 25]
-    python -m paper_2005_05758_b200.phase_clocks spmm  [rate:batch ...]      (default 4:8 4:32 25:8)
+    python -m paper_2005_05758_b200.phase_clocks spmm  [rate:batch | cfgN:batch ...]   (default 4:8 4:32 25:8; cfgN = first layer of that config)
 
 Builds libcsb_clocks.so beside the normal library with -DCSB_PHASE_CLOCKS -DCSB_PANEL_CLOCKS (see
 build.py), loads it instead of libcsb.so and prints
@@ -114,10 +114,14 @@ def spmm(cases):
     torch, binding = _load()
     for case in cases:
         rate, B = case.split(":")
-        w = workloads.CONFIGS["cfg4"](rate=float(rate), B=int(B))
-        m = w.matrix
+        if rate.startswith("cfg"):                 # first layer of a recurrent config, e.g. cfg5:32
+            m = workloads.CONFIGS[rate](T=1).layers[0]
+            X = np.random.default_rng(1).standard_normal((int(B), m.cols)).astype(np.float32)
+        else:
+            w = workloads.CONFIGS["cfg4"](rate=float(rate), B=int(B))
+            m, X = w.matrix, w.X
         As = [binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, 0) for _ in range(3)]
-        X = torch.from_numpy(w.X).cuda()
+        X = torch.from_numpy(X).cuda()
         Y = torch.empty((int(B), m.rows), device="cuda")
         for i in range(6):
             binding.csb_spmm(As[i % 3], X, Y)
@@ -129,7 +133,8 @@ def spmm(cases):
         per_cta = ck.reshape(-1, wpc, 12)
         slow = per_cta[np.argmax(per_cta.sum(axis=2).max(axis=1))]
         last = ck[np.argmax(ck[:, :6].sum(axis=1))]      # the warp that reaches the end of its items last
-        print("cfg4 rate %sx batch %s: %d warps (%d per CTA); cycles per phase, last pass of 32 batch columns" % (rate, B, n, wpc))
+        print("%s batch %s: %d warps (%d per CTA); cycles per phase, last pass of 32 batch columns"
+              % (rate if rate.startswith("cfg") else "cfg4 rate %sx" % rate, B, n, wpc))
         for i, nm in enumerate(SPMM_PHASES):
             print("   %-52s mean %8.0f  min %8.0f  max %8.0f   slowest CTA: mean %8.0f  max %8.0f   last warp %8.0f"
                   % (nm, ck[:, i].mean(), ck[:, i].min(), ck[:, i].max(), slow[:, i].mean(), slow[:, i].max(), last[i]))

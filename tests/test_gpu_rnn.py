@@ -155,6 +155,20 @@ def test_lstm_large_batch_both_paths_agree(monkeypatch):
     assert np.max(np.abs(ya - yb)) < 1e-4
 
 
+@pytest.mark.parametrize("cell,B,I", [("lstm", 32, 153), ("lstm", 9, 40), ("gru", 16, 70), ("gru", 11, 33)])
+def test_step_by_step_packed_inputs_equal_the_fp32_buffers(monkeypatch, cell, B, I):
+    # up to 32 product rows the gate kernels write h_t and x_{t+1} straight into the products' packed
+    # binary16 (hi, lo) inputs; the same numbers as packing the fp32 buffers in a kernel of its own
+    w = workloads.make_rnn_workload(33, cell, I, 512, 2, 32, 32, "lognormal", rate=4.0, T=5, B=B, w_std=0.15,
+                                    bias_std=0.2, state_std=0.4)
+    ya, ha, ca = check(w)
+    monkeypatch.setenv("CSB_RNN_STEP_UNPACKED", "1")
+    yb, hb, cb = check(w)
+    assert np.array_equal(ya, yb) and np.array_equal(ha, hb)
+    if cell == "lstm":
+        assert np.array_equal(ca, cb)
+
+
 @pytest.mark.parametrize("B,I,H,L,br,bc", [(16, 40, 48, 2, 16, 16), (20, 39, 100, 1, 32, 32), (33, 70, 192, 2, 64, 32), (8, 300, 512, 1, 32, 32)])
 def test_gru_batch_runs_step_by_step_on_tensor_cores(B, I, H, L, br, bc):
     # GRU from batch 16 (from batch 8 for layers of 100 k weights and more): one product over 2B rows ([u ; 0] and [0 ; h]) keeps the candidate's two parts apart
