@@ -264,6 +264,17 @@ struct MmaPlan {                           // device side, one per batch class, 
 int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch, float* Y, int64_t ldy, void* stream,
                     const uint8_t* packed = nullptr);
 bool spmm_mma_applicable(const csb_matrix* A, int batch);
+// The time loop of a recurrent stack inside the batched product kernel (csb_spmm_mma.cu): everything on the device.
+struct RnnTileLoop {
+    int L, B, H, gates; int64_t T;
+    const csb_matrix* const* W; const float* const* bias; const int* in_size;
+    const float* x; float* y;              // [T, B, I0]; [T, B, H] or null
+    uint8_t* const* xp;                    // per layer: packed inputs of its product, initialised for step 0
+    float* z; float* c; float* hs;         // pre-activations [rows of the product, gates * H]; c [L, B, H] (LSTM); h [L, B, H]
+    unsigned int* gbar;                    // one word for the grid barrier
+    int pitch, cap;
+};
+int launch_rnn_tile_loop(const RnnTileLoop& R, void* stream);
 void free_mma(csb_matrix* A);
 
 // ---- panel layout of the batch-1 product (csb_panel_plan.cpp, csb_panel.cu) ----

@@ -11,9 +11,12 @@
 // layer above, same step) or into y, and the gate kernel of layer 0 also moves x_{t+1} in.
 //
 // Up to 32 product rows (LSTM: batch <= 32, GRU: batch <= 16) the fp32 buffers V_l do not exist at all:
-// the gate kernels write h_t, and the one of layer 0 also x_{t+1}, straight into the packed binary16
+// the gate arithmetic writes h_t, and that of layer 0 also x_{t+1}, straight into the packed binary16
 // (hi, lo) input rows that the product kernel reads, transposed through shared memory so that the
-// stores of a row are contiguous; a step is then two launches per layer (product, gates).
+// stores of a row are contiguous; a step is then two launches per layer (product, gates).  With
+// CSB_RNN_STEP_LOOP=1, and where the layers' plans allow it, the whole sequence is instead ONE
+// cooperative launch of the product kernel's time loop (product pass, grid barrier, gates, grid barrier
+// per layer and step: csb_spmm_mma.cu).
 //
 // GRU (reset gate applied after the recurrent product) needs the input part and the recurrent part
 // of the candidate's pre-activation apart.  One product still does: V_l has 2B rows, row b holds
@@ -25,6 +28,7 @@
 
 #include "csb_internal.hpp"
 #include "csb_device.cuh"
+#include "csb_gates.cuh"
 
 namespace csb {
 
@@ -50,11 +54,12 @@ struct StepPlan {
     // `pitch` bytes per column of W_l, and the fp32 h of every layer
     uint8_t* d_xp[kMaxLayers] = {};
     float* d_h = nullptr;              // [L, B, H]
+    unsigned int* d_gbar = nullptr;    // grid-barrier word of the one-launch time loop
     int pitch = 0, cap = 0;
     ~StepPlan() {
         for (float* p : d_v) cudaFree(p);
         for (uint8_t* p : d_xp) cudaFree(p);
-        cudaFree(d_z); cudaFree(d_c); cudaFree(d_stage); cudaFree(d_h);
+        cudaFree(d_z); cudaFree(d_c); cudaFree(d_stage); cudaFree(d_h); cudaFree(d_gbar);
     }
 };
 static std::mutex g_step_mu;
@@ -142,43 +147,16 @@ __global__ void csb_gru_gates_kernel(const float* __restrict__ Z, const float* _
     }
 }
 
-// ---- the packed path -------------------------------------------------------------------------------------
-// A tile of 32 columns x nb batch values, tile[b][c], goes into slots slot0 .. slot0 + nb - 1 of the
-// packed rows of those columns: x = hi + lo, hi at [slot], lo at [cap + slot] (binary16 each).
-// Consecutive threads take consecutive batch values of a column, so a row's stores are contiguous.
-__device__ __forceinline__ void pack_tile(const float (*tile)[33], int ncols, int nb, uint8_t* rows, int pitch, int cap, int slot0,
-                                          uint8_t* rows2, int slot2) {
-    for (int idx = threadIdx.x; idx < 32 * nb; idx += blockDim.x) {
-        const int c = idx / nb, b = idx - c * nb;
-        if (c >= ncols) break;
-        const float x = tile[b][c];
-        const __half hi = __float2half_rn(x);
-        const __half lo = __float2half_rn(x - __half2float(hi));
-        __half* r = reinterpret_cast<__half*>(rows + (size_t)c * pitch);
-        r[slot0 + b] = hi;
-        r[cap + slot0 + b] = lo;
-        if (rows2) {
-            __half* r2 = reinterpret_cast<__half*>(rows2 + (size_t)c * pitch);
-            r2[slot2 + b] = hi;
-            r2[cap + slot2 + b] = lo;
-        }
-    }
-}
-
-// src [nb, ncols] (row stride ld) -> slots slot0 .. of the packed rows 0 .. ncols - 1 of xp; 256 threads, 32 columns per block.
+// ---- the packed path (device functions in csb_gates.cuh) ----------------------------------------------
+// src [nb, ncols] (row stride ld) -> slots slot0 .. of the packed rows 0 .. ncols - 1 of xp; 32 columns per block.
 __global__ void csb_pack_rows_kernel(const float* __restrict__ src, long long ld, int nb, int ncols, uint8_t* __restrict__ xp, int pitch,
                                      int cap, int slot0) {
     __shared__ float tile[32][33];
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5, c0 = blockIdx.x * 32;
-    for (int b = ty; b < nb; b += 8) tile[b][tx] = c0 + tx < ncols ? src[(long long)b * ld + c0 + tx] : 0.f;
-    __syncthreads();
-    pack_tile(tile, min(32, ncols - c0), nb, xp + (size_t)c0 * pitch, pitch, cap, slot0, nullptr, 0);
+    pack_columns(tile, src, ld, nb, ncols, (int)blockIdx.x * 32, xp, pitch, cap, slot0);
 }
 
-// The LSTM gate arithmetic as in csb_lstm_gates_kernel for 32 hidden units x the batch per block
-// (blocks 0 .. h_blocks - 1); h_t goes, packed, to rows j of xp_self (this layer's recurrent columns)
-// and of xp_next (the input columns of the layer above), as fp32 to hs[b, j] and y_t[b, j].  Blocks from
-// h_blocks on pack x_next [B, I] (the next step's input of layer 0) into rows of xp0.  256 threads.
+// Blocks 0 .. h_blocks - 1: the LSTM gates of 32 hidden units x the batch each; blocks from h_blocks on
+// pack x_next [B, I] (the next step's input of layer 0) into rows of xp0.
 __global__ void csb_lstm_gates_pack_kernel(const float* __restrict__ Z, const float* __restrict__ bias, float* __restrict__ c,
                                            float* __restrict__ hs, uint8_t* __restrict__ xp_self, uint8_t* __restrict__ xp_next,
                                            float* __restrict__ y_t, const float* __restrict__ x_next, int I, uint8_t* __restrict__ xp0,
@@ -186,37 +164,11 @@ __global__ void csb_lstm_gates_pack_kernel(const float* __restrict__ Z, const fl
     pdl_launch_dependents();
     pdl_wait();                                    // Z comes from the product in front, which also still reads xp0
     __shared__ float tile[32][33];
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    if ((int)blockIdx.x < h_blocks) {
-        const int j0 = blockIdx.x * 32, j = j0 + tx;
-        for (int b = ty; b < B; b += 8) {
-            float h = 0.f;
-            if (j < H) {
-                const float* z = Z + (size_t)b * 4 * H;
-                float zi = z[j], zf = z[H + j], zg = z[2 * H + j], zo = z[3 * H + j];
-                if (bias) { zi += bias[j]; zf += bias[H + j]; zg += bias[2 * H + j]; zo += bias[3 * H + j]; }
-                const size_t e = (size_t)b * H + j;
-                const float cn = logistic(zf) * c[e] + logistic(zi) * tanhf(zg);
-                h = logistic(zo) * tanhf(cn);
-                c[e] = cn;
-                hs[e] = h;
-                if (y_t) y_t[e] = h;
-            }
-            tile[b][tx] = h;
-        }
-        __syncthreads();
-        pack_tile(tile, min(32, H - j0), B, xp_self + (size_t)j0 * pitch, pitch, cap, 0, xp_next ? xp_next + (size_t)j0 * pitch : nullptr, 0);
-    } else {
-        const int c0 = ((int)blockIdx.x - h_blocks) * 32;
-        for (int b = ty; b < B; b += 8) tile[b][tx] = c0 + tx < I ? x_next[(size_t)b * I + c0 + tx] : 0.f;
-        __syncthreads();
-        pack_tile(tile, min(32, I - c0), B, xp0 + (size_t)c0 * pitch, pitch, cap, 0, nullptr, 0);
-    }
+    if ((int)blockIdx.x < h_blocks) lstm_gates_tile(tile, Z, bias, c, hs, xp_self, xp_next, y_t, pitch, cap, B, H, (int)blockIdx.x * 32);
+    else pack_columns(tile, x_next, (long long)I, B, I, ((int)blockIdx.x - h_blocks) * 32, xp0, pitch, cap, 0);
 }
 
-// The GRU gate arithmetic as in csb_gru_gates_kernel, same tiling.  The product has 2B rows: slots
-// 0 .. B - 1 of a packed row carry the input part (zero in the recurrent columns), slots B .. 2B - 1
-// the recurrent part (zero in the input columns); the zeros are written once, before the first step.
+// The same for the GRU (its product has 2B rows: the zeros of the unused slots are written once, before the first step).
 __global__ void csb_gru_gates_pack_kernel(const float* __restrict__ Z, const float* __restrict__ bias, float* __restrict__ hs,
                                           uint8_t* __restrict__ xp_self, uint8_t* __restrict__ xp_next, float* __restrict__ y_t,
                                           const float* __restrict__ x_next, int I, uint8_t* __restrict__ xp0, int pitch, int cap, int B,
@@ -224,33 +176,8 @@ __global__ void csb_gru_gates_pack_kernel(const float* __restrict__ Z, const flo
     pdl_launch_dependents();
     pdl_wait();
     __shared__ float tile[32][33];
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    if ((int)blockIdx.x < h_blocks) {
-        const int j0 = blockIdx.x * 32, j = j0 + tx;
-        for (int b = ty; b < B; b += 8) {
-            float h = 0.f;
-            if (j < H) {
-                const float* zx = Z + (size_t)b * 3 * H;
-                const float* zh = Z + (size_t)(B + b) * 3 * H;
-                float ar = zx[j] + zh[j], au = zx[H + j] + zh[H + j], nx = zx[2 * H + j], nh = zh[2 * H + j];
-                if (bias) { ar += bias[j]; au += bias[H + j]; nx += bias[2 * H + j]; nh += bias[3 * H + j]; }
-                const float r = logistic(ar), u = logistic(au);
-                const float cand = tanhf(nx + r * nh);
-                const size_t e = (size_t)b * H + j;
-                h = (1.f - u) * cand + u * hs[e];
-                hs[e] = h;
-                if (y_t) y_t[e] = h;
-            }
-            tile[b][tx] = h;
-        }
-        __syncthreads();
-        pack_tile(tile, min(32, H - j0), B, xp_self + (size_t)j0 * pitch, pitch, cap, B, xp_next ? xp_next + (size_t)j0 * pitch : nullptr, 0);
-    } else {
-        const int c0 = ((int)blockIdx.x - h_blocks) * 32;
-        for (int b = ty; b < B; b += 8) tile[b][tx] = c0 + tx < I ? x_next[(size_t)b * I + c0 + tx] : 0.f;
-        __syncthreads();
-        pack_tile(tile, min(32, I - c0), B, xp0 + (size_t)c0 * pitch, pitch, cap, 0, nullptr, 0);
-    }
+    if ((int)blockIdx.x < h_blocks) gru_gates_tile(tile, Z, bias, hs, xp_self, xp_next, y_t, pitch, cap, B, H, (int)blockIdx.x * 32);
+    else pack_columns(tile, x_next, (long long)I, B, I, ((int)blockIdx.x - h_blocks) * 32, xp0, pitch, cap, 0);
 }
 
 static int env_flag(const char* name) {
@@ -296,7 +223,10 @@ int rnn_forward_stepwise(int gates, int L, const csb_matrix* const* W, const flo
                 if (packed_path) CSB_CUDA(cudaMalloc((void**)&np->d_xp[l], (size_t)(in_size[l] + H) * np->pitch));
                 else CSB_CUDA(cudaMalloc((void**)&np->d_v[l], (size_t)rows_v * (in_size[l] + H) * 4));
             }
-            if (packed_path) CSB_CUDA(cudaMalloc((void**)&np->d_h, (size_t)L * B * H * 4));
+            if (packed_path) {
+                CSB_CUDA(cudaMalloc((void**)&np->d_h, (size_t)L * B * H * 4));
+                CSB_CUDA(cudaMalloc((void**)&np->d_gbar, 4));
+            }
             CSB_CUDA(cudaMalloc((void**)&np->d_z, (size_t)(gates == 3 ? 2 : 1) * B * gates * H * 4));
             if (gates == 4) CSB_CUDA(cudaMalloc((void**)&np->d_c, (size_t)L * B * H * 4));
             P = np.get();
@@ -343,8 +273,22 @@ int rnn_forward_stepwise(int gates, int L, const csb_matrix* const* W, const flo
             if (c0) CSB_CUDA(cudaMemcpyAsync(P->d_c, c0, ns * 4, in_kind, st));
             else CSB_CUDA(cudaMemsetAsync(P->d_c, 0, ns * 4, st));
         }
+        // On request (CSB_RNN_STEP_LOOP=1) the whole sequence in one launch of the product kernel's time loop,
+        // where that serves the stack.  Not the default: measured, two grid barriers per layer and step cost
+        // as much as the two launch hand-overs they replace (47.6 against 48-51 us per step on a two-layer
+        // 2048-unit LSTM at batch 32, 14.0 against 11.4 on a 1024-unit GRU at batch 8).
+        bool looped = false;
+        if (env_flag("CSB_RNN_STEP_LOOP") && T < (1 << 24)) {
+            RnnTileLoop R{};
+            R.L = L; R.B = B; R.H = H; R.gates = gates; R.T = T; R.W = W; R.bias = bias; R.in_size = in_size;
+            R.x = dx; R.y = dy; R.xp = P->d_xp; R.z = P->d_z; R.c = gru ? nullptr : P->d_c; R.hs = P->d_h; R.gbar = P->d_gbar;
+            R.pitch = pitch; R.cap = cap;
+            const int rc = launch_rnn_tile_loop(R, stream);
+            if (rc == CSB_OK) looped = true;
+            else if (rc != 1) return rc;
+        }
         const int h_blocks = (H + 31) / 32, x_blocks = (I0 + 31) / 32;
-        for (int64_t t = 0; t < T; ++t) {
+        for (int64_t t = 0; t < T && !looped; ++t) {
             for (int l = 0; l < L; ++l) {
                 const int rc = launch_spmm_mma(W[l], nullptr, 0, vrows, P->d_z, (int64_t)gates * H, stream, P->d_xp[l]);
                 if (rc != CSB_OK) {

@@ -34,11 +34,13 @@
 
 #include "csb_internal.hpp"
 #include "csb_device.cuh"
+#include "csb_gates.cuh"
 
 namespace csb {
 
 constexpr uint32_t kOffMaskM = 0x3fffffffu;
 constexpr uint32_t kNoRow = 0xffffffffu;
+constexpr size_t kLoopTileBytes = 32 * 33 * 4;  // the time loop's transposition tile of the gate arithmetic
 constexpr size_t kSpmmStaticSmem = 256;       // the kernel's statically allocated shared memory (CTA descriptor, row table), rounded up
 
 struct SpmmArgs {
@@ -50,9 +52,33 @@ struct SpmmArgs {
     long long ldy;
     uint32_t* status;
     int nb, rows, cols, block_r, block_c, tile_cols, RG, S, x_depth, w_stages, pitch, tile_bytes;   // tile_cols: matrix columns per input tile
+    int q_rows;                // rows of the largest row group the shared-memory carve-up must hold (RG * block_r of one product)
 #ifdef CSB_SPMM_CLOCKS
-    long long* clocks;         // instrumented build only: [CTA][warp][12] cycles per phase
+    long long* clocks;         // instrumented build only: [CTA][warp][16] cycles per phase
 #endif
+};
+
+// The recurrent time loop around the product (batches of 8 and more, up to 32 product rows): one
+// cooperative launch runs all steps of all layers.  Per layer and step: the product pass of that
+// layer's matrix over its packed inputs into Z, a grid barrier, the gate arithmetic (tiles of 32 hidden
+// units dealt to the CTAs; h_t goes straight into the packed inputs of the next products), a grid barrier.
+struct SpmmLoopLayer {
+    const uint8_t* stream; const uint4* warp_desc; const SpmmCta* ctas;
+    const uint8_t* xp;         // packed inputs of this layer's product, rows 0 .. in_size + H - 1
+    const float* bias; float* c; float* hs;
+    uint8_t* xp_self;          // = xp + in_size * pitch: where h_t of this layer goes
+    uint8_t* xp_next;          // the input rows of the layer above, or null
+    int rows, cols, n_ctas, RG;
+};
+struct SpmmLoop {
+    SpmmLoopLayer layer[kMaxLayers];
+    float* Z; long long ldz;   // pre-activations of the layer being worked on: [product rows][gates * H]
+    const float* x;            // [T, B, I0]
+    float* y;                  // [T, B, H] or null
+    uint8_t* xp0;              // packed inputs of layer 0 (x_{t+1} is packed into its first I0 rows)
+    unsigned int* gbar;        // grid barrier counter, zero at launch
+    unsigned long long barrier_ns;
+    int T, L, B, H, I0, gates, cap;
 };
 
 #ifdef CSB_SPMM_CLOCKS
@@ -69,9 +95,11 @@ __host__ __device__ constexpr int spmm_sum_pitch(int NT) { return NT == 1 ? 8 : 
 __host__ __device__ constexpr size_t spmm_q_bytes(int NT, int group_rows) { return (size_t)8 * NT * (group_rows + 1) * 4; }
 
 struct SpmmSmem {
-    size_t wfull, xfull, wcnt, xcnt, dead, zero, rings, wring, xring, qsums, total;
-    // q_bytes: room for the CTA's own sums of its row group
-    __host__ __device__ SpmmSmem(int n_warps, int w_stages, int x_depth, int tile_bytes, int pitch, int MT, int NT, size_t q_bytes) {
+    size_t wfull, xfull, wcnt, xcnt, dead, zero, extra, rings, wring, xring, qsums, total;
+    // q_bytes: room for the CTA's own sums of its row group; extra_bytes: a region outside the rings (the time
+    // loop's tile of the gate arithmetic, which runs while the next pass's first weights are on their way)
+    __host__ __device__ SpmmSmem(int n_warps, int w_stages, int x_depth, int tile_bytes, int pitch, int MT, int NT, size_t q_bytes,
+                                 size_t extra_bytes = 0) {
         const int n_streams = n_warps;
         wfull = 0;
         xfull = wfull + (size_t)n_streams * w_stages * 8;
@@ -79,7 +107,8 @@ struct SpmmSmem {
         xcnt = wcnt + (size_t)n_streams * w_stages * 4;
         dead = xcnt + (size_t)x_depth * 4;
         zero = (dead + 4 + 127) & ~(size_t)127;
-        rings = (zero + (size_t)pitch + 127) & ~(size_t)127;
+        extra = (zero + (size_t)pitch + 127) & ~(size_t)127;
+        rings = (extra + extra_bytes + 127) & ~(size_t)127;
         wring = rings;
         xring = wring + (size_t)n_streams * w_stages * kSpmmStageBytes;
         const size_t ring_end = xring + (size_t)x_depth * tile_bytes;
@@ -160,13 +189,20 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
     return v;
 }
 
-template <int MT, int NT>
-__global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_kernel(const SpmmArgs a) {
+__device__ __forceinline__ unsigned int ld_acquire_gpu_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// One product pass (LOOP = false: the whole kernel), or the time loop of a recurrent stack around it.
+template <int MT, int NT, bool LOOP>
+__device__ __forceinline__ void spmm_tile_body(SpmmArgs a, const SpmmLoop* lp) {
     constexpr int kSpmmWarps = NT == 1 ? 32 : 16;
-    pdl_launch_dependents();
+    if (!LOOP) pdl_launch_dependents();
     extern __shared__ __align__(128) uint8_t smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const SpmmSmem L(kSpmmWarps, a.w_stages, a.x_depth, a.tile_bytes, a.pitch, MT, NT, spmm_q_bytes(NT, a.RG * a.block_r));
+    const SpmmSmem L(kSpmmWarps, a.w_stages, a.x_depth, a.tile_bytes, a.pitch, MT, NT, spmm_q_bytes(NT, a.q_rows), LOOP ? kLoopTileBytes : 0);
     uint64_t* wfull = reinterpret_cast<uint64_t*>(smem + L.wfull) + warp * a.w_stages;
     uint64_t* xfull = reinterpret_cast<uint64_t*>(smem + L.xfull);
     uint32_t* xcnt = reinterpret_cast<uint32_t*>(smem + L.xcnt);
@@ -176,15 +212,12 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     const uint32_t zero_addr = smem_u32(smem + L.zero);
 
 #ifdef CSB_SPMM_CLOCKS
-    long long sprof[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    long long sprof[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     long long st_ = clock64();
 #endif
     // the CTA's descriptor goes to shared memory, one word per thread
     __shared__ __align__(16) SpmmCta s_me;
     __shared__ int s_first[5];                     // first warp of every block-row of the group (the warps of a row are neighbours)
-    if (threadIdx.x < sizeof(SpmmCta) / 4) reinterpret_cast<uint32_t*>(&s_me)[threadIdx.x] = reinterpret_cast<const uint32_t*>(a.ctas + blockIdx.x)[threadIdx.x];
-    const uint4 wd = __ldg(a.warp_desc + (size_t)blockIdx.x * kSpmmWarps + warp);
-    const uint32_t n_chunks = wd.y;
     if (threadIdx.x == 0) {
         for (int i = 0; i < kSpmmWarps * a.w_stages; ++i) mbar_init(reinterpret_cast<uint64_t*>(smem + L.wfull) + i, 1);
         for (int i = 0; i < a.x_depth; ++i) { mbar_init(&xfull[i], 1); xcnt[i] = 0u; }
@@ -192,6 +225,49 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
         mbar_fence_init();
     }
     for (int i = threadIdx.x; i < (a.pitch + 16) / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem + L.zero)[i] = 0u;
+    // ring positions: they run on from pass to pass of the time loop (every use of a slot is one phase of its barrier)
+    int xs = 0, s = 0;                             // slot of the input ring the warp is at; stage of its weight ring
+    uint32_t xpar = 0u, parity = 0u;               // and the parities of their current uses
+    unsigned int gbar_round = 0;                   // grid barriers passed (time loop)
+    // time loop: what the next pass starts with is fetched while this one ends
+    bool primed = false;
+    uint4 wd_next = make_uint4(0u, 0u, 0u, 0u);
+    uint32_t me_word_next = 0u, issue_off_next = 0u;
+    // The first chunks of a warp's weight stream go out, into the stages in ring order from where the warp
+    // stands; returns where the next chunk to be fetched starts.  (A warp's chunks lie back to back.)
+    auto first_weights = [&](const uint8_t* stream, const uint4& d) -> uint32_t {
+        const uint32_t first[3] = {d.z & 0xffffu, d.z >> 16, d.w};
+        uint32_t off = d.x;
+        // (time loop: the rings were last touched by ordinary loads and stores, the sums of the pass in front,
+        // which a CTA barrier separates from these copies)
+        int si = s;
+        for (int k = 0; k < a.w_stages && k < (int)d.y; ++k) {
+            if (lane == 0) {
+                mbar_expect_tx(&wfull[si], first[k]);
+                bulk_g2s(wring + (size_t)si * kSpmmStageBytes, stream + (size_t)off * 16, first[k], &wfull[si]);
+            }
+            off += first[k] >> 4;
+            if (++si == a.w_stages) si = 0;
+        }
+        return off;
+    };
+    const int n_pass = LOOP ? lp->T * lp->L : 1;
+    for (int pass = 0; pass < n_pass; ++pass) {
+    const int layer = LOOP ? pass % lp->L : 0, step = LOOP ? pass / lp->L : 0;
+    bool pass_dead = false;
+    if (LOOP) {
+        const SpmmLoopLayer& ly = lp->layer[layer];
+        a.stream = ly.stream; a.warp_desc = ly.warp_desc; a.ctas = ly.ctas; a.xp = ly.xp;
+        a.rows = ly.rows; a.cols = ly.cols; a.RG = ly.RG; a.Y = lp->Z; a.ldy = lp->ldz;
+    }
+    if (!LOOP || (int)blockIdx.x < lp->layer[layer].n_ctas) {
+    // (time loop: descriptors and first weights of this pass were fetched during the pass in front, where there was one)
+    const bool was_primed = LOOP && primed;
+    primed = false;
+    if (threadIdx.x < sizeof(SpmmCta) / 4)
+        reinterpret_cast<uint32_t*>(&s_me)[threadIdx.x] = was_primed ? me_word_next : reinterpret_cast<const uint32_t*>(a.ctas + blockIdx.x)[threadIdx.x];
+    const uint4 wd = was_primed ? wd_next : __ldg(a.warp_desc + (size_t)blockIdx.x * kSpmmWarps + warp);
+    const uint32_t n_chunks = wd.y;
     __syncthreads();
     const SpmmCta* me = &s_me;
     const int ntiles = me->ntiles, tile0 = me->tile0;
@@ -199,17 +275,7 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     auto tile_src = [&](int tl) { return a.xp + (size_t)(tile0 * a.block_c + tl * a.tile_cols) * a.pitch; };
     // the weights were written at plan time: their first copies go out before the work in front is waited for
     // (a warp's chunks lie back to back; issue_off is where the next one to be fetched starts)
-    uint32_t issue_off = wd.x;
-    {
-        const uint32_t first[3] = {wd.z & 0xffffu, wd.z >> 16, wd.w};
-        for (int s = 0; s < a.w_stages && s < (int)n_chunks; ++s) {
-            if (lane == 0) {
-                mbar_expect_tx(&wfull[s], first[s]);
-                bulk_g2s(wring + (size_t)s * kSpmmStageBytes, a.stream + (size_t)issue_off * 16, first[s], &wfull[s]);
-            }
-            issue_off += first[s] >> 4;
-        }
-    }
+    uint32_t issue_off = was_primed ? issue_off_next : first_weights(a.stream, wd);
     if (threadIdx.x == 0) {
         int rr = 0;
         s_first[0] = 0;
@@ -217,7 +283,10 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
             while (rr < (int)me->warp_row[w]) s_first[++rr] = w;
         while (rr < 4) s_first[++rr] = kSpmmWarps;
     }
-    pdl_wait();                                    // the packed inputs and Y belong to the work in front on the stream
+    if (!LOOP) pdl_wait();                         // the packed inputs and Y belong to the work in front on the stream
+    // (time loop: the packed inputs were written with ordinary stores by other CTAs, before the grid barrier;
+    // every lane that may issue a copy of them orders that behind its view of the barrier, once per pass)
+    if (LOOP && lane == 0) fence_proxy_async_all();
     // One lane fetches a tile with one bulk copy.  (No proxy fence in front of a refill: the slot's
     // readers have their data in registers by the time they release it, and the release orders them
     // before this copy is issued.)
@@ -227,7 +296,7 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
             bulk_g2s(xring + (size_t)slot * a.tile_bytes, tile_src(tl), tile_bytes_of(tl), &xfull[slot]);
         }
     };
-    if (warp < a.x_depth && warp < ntiles) fetch_tile(warp, warp);          // the first tiles, one warp each
+    if (warp < a.x_depth && warp < ntiles) fetch_tile((xs + warp) % a.x_depth, warp);     // the first tiles, one warp each
     SPMM_LAP(0);                                   // set-up, first copies out, the work in front waited for
     // A wait gives up after a second, or as soon as any warp of the CTA has given up.
     auto wait_bar = [&](uint64_t* bar, uint32_t parity) -> bool {
@@ -249,8 +318,7 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     };
     // The tile this warp is at (tcur) sits in slot xs of the input ring, in the use of that slot with
     // parity xpar; both move along with tcur, so nothing is divided.
-    int tcur = 0, xs = 0;
-    uint32_t xpar = 0u;
+    int tcur = 0;
     auto wait_x = [&]() -> bool { return wait_bar(&xfull[xs], xpar); };
     // This warp is done with tile tcur; the last warp of the CTA to say so refills the slot.
     auto release_x = [&]() {
@@ -280,8 +348,6 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
     const uint32_t x_lane_off = (uint32_t)(lane >> 4) * 16u;                 // this lane's 16 bytes inside a tile row
     const int kr_lane = ((lane >> 3) & 1) * 8 + (lane & 7);                  // its k row inside a 16-column slab
     bool alive = true;
-    int s = 0;                                     // stage of this warp's weight ring, and the parity of its current use
-    uint32_t parity = 0u;
     for (uint32_t c = 0; c < n_chunks && alive; ++c) {
         SPMM_LAP(4);
         if (!wait_bar(&wfull[s], parity)) { alive = false; break; }
@@ -383,6 +449,15 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
         release_x();
     }
     SPMM_LAP(5);                                   // the tiles behind this warp's last item
+    if (LOOP && pass + 1 < n_pass) {
+        // descriptors of this CTA in the next pass: asked for now, used once the sums below are done
+        const SpmmLoopLayer& nx = lp->layer[(pass + 1) % lp->L];
+        if ((int)blockIdx.x < nx.n_ctas) {
+            wd_next = __ldg(nx.warp_desc + (size_t)blockIdx.x * kSpmmWarps + warp);
+            if (threadIdx.x < sizeof(SpmmCta) / 4) me_word_next = __ldg(reinterpret_cast<const uint32_t*>(nx.ctas + blockIdx.x) + threadIdx.x);
+            primed = true;
+        }
+    }
     __syncthreads();
     SPMM_LAP(6);                                   // waiting for the other warps of the CTA
     const bool dead = *s_dead != 0u;
@@ -391,7 +466,8 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
         // time to land before the CTA's shared memory goes away, and write nothing
         const unsigned long long t0 = global_ns();
         while (global_ns() - t0 < 200000ull) __nanosleep(1000);
-        if (a.S == 1) return;                      // (a CTA of a cluster still has to keep the cluster's barriers company)
+        if (!LOOP && a.S == 1) return;             // (a CTA of a cluster still has to keep the cluster's barriers company)
+        pass_dead = true;
     }
 
     // ---- the warps' sums meet in shared memory (the rings are no longer in use)
@@ -499,9 +575,77 @@ __global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_ker
         cluster_barrier();
     }
     SPMM_LAP(11);                                  // until every CTA of the cluster has read
+    // (time loop) the rings are free again: the next pass's first weights go out and land while the gates are done
+    if (LOOP) {
+        __syncthreads();                           // every thread is done reading the sums that lie where the rings are
+        if (primed && !pass_dead) issue_off_next = first_weights(lp->layer[(pass + 1) % lp->L].stream, wd_next);
+        else primed = false;
+    }
+    }                                              // (CTAs beyond this layer's plan sit the pass out)
+    if (LOOP) {
+        // ---- every CTA's part of Z is written: gate arithmetic of (layer, step), then on to the next pass.
+        // A CTA that gave up does not come here; the others then run into the bound of the barrier.
+        if (pass_dead) break;
+        auto grid_sync = [&]() -> bool {
+            __syncthreads();
+            ++gbar_round;
+            if (threadIdx.x == 0) {
+                __threadfence();
+                atomicAdd(lp->gbar, 1u);
+                const unsigned int target = gbar_round * gridDim.x;
+                unsigned long long t0 = 0;
+                unsigned int spins = 0;
+                while (ld_acquire_gpu_u32(lp->gbar) < target) {
+                    if ((++spins & 63u) == 0) {
+                        const unsigned long long now = global_ns();
+                        if (t0 == 0) t0 = now;
+                        else if (now - t0 > lp->barrier_ns) { *s_dead = 1u; *(volatile uint32_t*)a.status = (uint32_t)kDevBarrierTimeout; break; }
+                    }
+                }
+            }
+            __syncthreads();
+            return *s_dead == 0u;
+        };
+        SPMM_LAP(15);                              // (time loop) next pass's first weights out
+        if (!grid_sync()) break;
+        SPMM_LAP(12);                              // (time loop) grid barrier behind the product pass
+        {
+            const SpmmLoopLayer& ly = lp->layer[layer];
+            float (*tile)[33] = reinterpret_cast<float (*)[33]>(smem + L.extra);
+            const int B = lp->B, H = lp->H, h_tiles = (H + 31) / 32;
+            const bool pack_x = layer == 0 && step + 1 < lp->T;
+            const int n_tiles = h_tiles + (pack_x ? (lp->I0 + 31) / 32 : 0);
+            float* y_t = (layer == lp->L - 1 && lp->y) ? lp->y + (size_t)step * B * H : nullptr;
+            for (int tl = blockIdx.x; tl < n_tiles; tl += gridDim.x) {
+                if (tl < h_tiles) {
+                    if (lp->gates == 4) lstm_gates_tile(tile, lp->Z, ly.bias, ly.c, ly.hs, ly.xp_self, ly.xp_next, y_t, a.pitch, lp->cap, B, H, tl * 32);
+                    else gru_gates_tile(tile, lp->Z, ly.bias, ly.hs, ly.xp_self, ly.xp_next, y_t, a.pitch, lp->cap, B, H, tl * 32);
+                } else {
+                    pack_columns(tile, lp->x + (size_t)(step + 1) * B * lp->I0, (long long)lp->I0, B, lp->I0, (tl - h_tiles) * 32, lp->xp0,
+                                 a.pitch, lp->cap, 0);
+                }
+                __syncthreads();                   // the tile is free again
+            }
+        }
+        SPMM_LAP(13);                              // (time loop) gate arithmetic
+        if (pass + 1 < n_pass && !grid_sync()) break;
+        SPMM_LAP(14);                              // (time loop) grid barrier behind the gates
+    }
+    }                                              // passes
 #ifdef CSB_SPMM_CLOCKS
-    if (lane == 0) for (int i = 0; i < 12; ++i) a.clocks[((size_t)blockIdx.x * kSpmmWarps + warp) * 12 + i] = sprof[i];
+    if (lane == 0) for (int i = 0; i < 16; ++i) a.clocks[((size_t)blockIdx.x * kSpmmWarps + warp) * 16 + i] = sprof[i];
 #endif
+}
+
+template <int MT, int NT>
+__global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_spmm_tile_kernel(const SpmmArgs a) {
+    spmm_tile_body<MT, NT, false>(a, nullptr);
+}
+
+// The recurrent time loop (see SpmmLoop): launched cooperatively, so that the bounded grid barriers can be passed.
+template <int MT, int NT>
+__global__ void __launch_bounds__((NT == 1 ? 32 : 16) * 32, 1) csb_rnn_tile_kernel(const SpmmArgs a, const __grid_constant__ SpmmLoop lp) {
+    spmm_tile_body<MT, NT, true>(a, &lp);
 }
 
 #define CSB_CUDA(call)                                                                     \
@@ -610,10 +754,28 @@ void free_mma(csb_matrix* A) {
 static long long* g_spmm_clocks = nullptr;
 static int g_spmm_clock_warps = 0;
 extern "C" int csb_debug_spmm_clocks(long long* host_out, int max_warps) {
-    cudaMemcpy(host_out, g_spmm_clocks, (size_t)std::min(max_warps, g_spmm_clock_warps) * 12 * 8, cudaMemcpyDeviceToHost);
+    cudaMemcpy(host_out, g_spmm_clocks, (size_t)std::min(max_warps, g_spmm_clock_warps) * 16 * 8, cudaMemcpyDeviceToHost);
     return g_spmm_clock_warps;
 }
 #endif
+
+// The plan of A for batch class ci, built on first use (the device of A is current).  CSB_OK, an error, or 1 = the
+// tensor-core layout does not serve this matrix.
+static int ensure_spmm_plan(const csb_matrix* A, int ci) {
+    std::lock_guard<std::mutex> lk(A->mma_mu);
+    if (!A->mma) {
+        A->mma = new (std::nothrow) MmaPlan();
+        if (!A->mma) { set_error("out of host memory"); return CSB_ERR_ALLOC; }
+    }
+    MmaPlan::PerClass& C = A->mma->cls[ci];
+    if (!C.built && !C.unusable) {
+        int rc;
+        try { rc = build_spmm_plan(A, ci, &C); }
+        catch (const std::bad_alloc&) { set_error("out of host memory while planning the batched product"); rc = CSB_ERR_ALLOC; }
+        if (rc != CSB_OK) { C.unusable = true; return rc; }
+    }
+    return (C.unusable || !C.built) ? 1 : CSB_OK;
+}
 
 // Returns CSB_OK after launching, or 1 when the caller should use the CUDA-core path.
 // With `packed` (and X == nullptr) the inputs are taken from a buffer the caller has filled in the
@@ -629,28 +791,17 @@ int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch,
     struct Restore { int prev, cur; ~Restore() { if (prev != cur) cudaSetDevice(prev); } } restore{prev, A->device};
     const int ci = spmm_class_index(batch);
     {
-        std::lock_guard<std::mutex> lk(A->mma_mu);
-        if (!A->mma) {
-            A->mma = new (std::nothrow) MmaPlan();
-            if (!A->mma) { set_error("out of host memory"); return CSB_ERR_ALLOC; }
-        }
-        MmaPlan::PerClass& C = A->mma->cls[ci];
-        if (!C.built && !C.unusable) {
-            int rc;
-            try { rc = build_spmm_plan(A, ci, &C); }
-            catch (const std::bad_alloc&) { set_error("out of host memory while planning the batched product"); rc = CSB_ERR_ALLOC; }
-            if (rc != CSB_OK) { C.unusable = true; return rc; }
-        }
+        const int rc = ensure_spmm_plan(A, ci);
+        if (rc != CSB_OK) return rc;
     }
     const MmaPlan::PerClass& P = A->mma->cls[ci];
-    if (P.unusable || !P.built) return 1;
     const int NT = 1 << ci, MT = mt_of(A), cap = 8 * NT;
     cudaStream_t st = (cudaStream_t)stream;
     SpmmArgs a{};
     a.stream = P.d_stream; a.warp_desc = (const uint4*)P.d_warp_desc; a.ctas = P.d_ctas;
     a.xp = packed ? packed : (const uint8_t*)P.d_xp; a.ldy = ldy; a.status = PP.d_status;
     a.rows = (int)A->rows; a.cols = (int)A->cols; a.block_r = A->block_r; a.block_c = A->block_c;
-    a.RG = P.RG; a.S = P.S; a.x_depth = P.x_depth; a.w_stages = P.w_stages;
+    a.RG = P.RG; a.S = P.S; a.x_depth = P.x_depth; a.w_stages = P.w_stages; a.q_rows = P.RG * A->block_r;
     a.tile_cols = spmm_tile_blocks(A->block_c) * A->block_c;
     a.pitch = spmm_pitch(NT); a.tile_bytes = (a.tile_cols * a.pitch + 127) & ~127;
 #ifdef CSB_SPMM_CLOCKS
@@ -679,6 +830,99 @@ int launch_spmm_mma(const csb_matrix* A, const float* X, int64_t ldx, int batch,
         CSB_CUDA(CSB_SPMM_DISPATCH(launch_tile_kernel, MT, NT, &cfg, a));
         CSB_CUDA(cudaGetLastError());
     }
+    return CSB_OK;
+}
+
+template <int MT, int NT>
+static cudaError_t set_loop_smem_attr(size_t bytes) {
+    return cudaFuncSetAttribute(csb_rnn_tile_kernel<MT, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+template <int MT, int NT>
+static cudaError_t max_loop_clusters(int* n, const cudaLaunchConfig_t* cfg) {
+    return cudaOccupancyMaxActiveClusters(n, csb_rnn_tile_kernel<MT, NT>, cfg);
+}
+template <int MT, int NT>
+static cudaError_t launch_loop_kernel(const cudaLaunchConfig_t* cfg, const SpmmArgs& a, const SpmmLoop& lp) {
+    return cudaLaunchKernelEx(cfg, csb_rnn_tile_kernel<MT, NT>, a, lp);
+}
+
+// The whole sequence of a recurrent stack in one cooperative launch of the product kernel's time loop.
+// Returns CSB_OK after launching, an error, or 1 when the loop does not serve this stack (layers whose
+// plans differ in block shape or cluster size, a plan that does not fit, a grid that cannot be
+// co-resident): the caller then issues the steps as separate launches.  The device of W[0] is current.
+int launch_rnn_tile_loop(const RnnTileLoop& R, void* stream) {
+    const csb_matrix* A0 = R.W[0];
+    const int vrows = R.gates == 3 ? 2 * R.B : R.B;
+    if (vrows > 32 || R.L > kMaxLayers) return 1;
+    const int ci = spmm_class_index(vrows), NT = 1 << ci, MT = mt_of(A0);
+    SpmmArgs a{};
+    SpmmLoop lp{};
+    int S = 0, n_ctas = 0, w_stages = 3, x_depth = 8, q_rows = 0;
+    for (int l = 0; l < R.L; ++l) {
+        const csb_matrix* A = R.W[l];
+        if (A->block_r != A0->block_r || A->block_c != A0->block_c || A->device != A0->device) return 1;
+        const int rc = ensure_spmm_plan(A, ci);
+        if (rc != CSB_OK) return rc;
+        if (A->product.h_status && *A->product.h_status != 0) { set_error("an earlier product on a layer's handle gave up waiting on the device"); return CSB_ERR_TIMEOUT; }
+        const MmaPlan::PerClass& P = A->mma->cls[ci];
+        if (l == 0) S = P.S;
+        if (P.S != S) return 1;                              // one cluster shape per launch
+        n_ctas = std::max(n_ctas, P.n_ctas);
+        w_stages = std::min(w_stages, P.w_stages); x_depth = std::min(x_depth, P.x_depth);
+        q_rows = std::max(q_rows, P.RG * A->block_r);
+        SpmmLoopLayer& ly = lp.layer[l];
+        ly.stream = P.d_stream; ly.warp_desc = (const uint4*)P.d_warp_desc; ly.ctas = P.d_ctas; ly.xp = R.xp[l];
+        ly.bias = R.bias ? R.bias[l] : nullptr;
+        ly.c = R.c ? R.c + (size_t)l * R.B * R.H : nullptr;
+        ly.hs = R.hs + (size_t)l * R.B * R.H;
+        ly.xp_self = R.xp[l] + (size_t)R.in_size[l] * R.pitch;
+        ly.xp_next = l + 1 < R.L ? R.xp[l + 1] : nullptr;
+        ly.rows = (int)A->rows; ly.cols = (int)A->cols; ly.n_ctas = P.n_ctas; ly.RG = P.RG;
+    }
+    a.status = A0->product.d_status;
+    a.nb = vrows; a.block_r = A0->block_r; a.block_c = A0->block_c; a.S = S; a.x_depth = x_depth; a.w_stages = w_stages; a.q_rows = q_rows;
+    a.tile_cols = spmm_tile_blocks(A0->block_c) * A0->block_c;
+    a.pitch = spmm_pitch(NT); a.tile_bytes = (a.tile_cols * a.pitch + 127) & ~127;
+    if (a.pitch != R.pitch) { set_error("packed inputs of another batch class"); return CSB_ERR_INVALID_ARG; }
+    // the loop's own tile may cost the input ring a slot
+    while (x_depth > 2 && SpmmSmem(spmm_warps(NT), w_stages, x_depth, a.tile_bytes, a.pitch, MT, NT, spmm_q_bytes(NT, q_rows), kLoopTileBytes).total +
+                                  kSpmmStaticSmem > A0->smem_optin)
+        --x_depth;
+    a.x_depth = x_depth;
+    const SpmmSmem Lay(spmm_warps(NT), w_stages, x_depth, a.tile_bytes, a.pitch, MT, NT, spmm_q_bytes(NT, q_rows), kLoopTileBytes);
+    if (Lay.total + kSpmmStaticSmem > A0->smem_optin) return 1;
+#ifdef CSB_SPMM_CLOCKS
+    if (!g_spmm_clocks) cudaMalloc((void**)&g_spmm_clocks, (size_t)1 << 24);
+    a.clocks = g_spmm_clocks;
+    g_spmm_clock_warps = n_ctas * spmm_warps(NT);
+#endif
+    lp.Z = R.z; lp.ldz = (long long)R.gates * R.H; lp.x = R.x; lp.y = R.y; lp.xp0 = R.xp[0]; lp.gbar = R.gbar;
+    lp.barrier_ns = 2000000000ull;
+    lp.T = (int)R.T; lp.L = R.L; lp.B = R.B; lp.H = R.H; lp.I0 = R.in_size[0]; lp.gates = R.gates; lp.cap = R.cap;
+    cudaStream_t st = (cudaStream_t)stream;
+    CSB_CUDA(CSB_SPMM_DISPATCH(set_loop_smem_attr, MT, NT, A0->smem_optin - kSpmmStaticSmem));
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)S; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = S > 1 ? 2 : 1;
+    cfg.gridDim = dim3((unsigned)n_ctas); cfg.blockDim = dim3((unsigned)spmm_warps(NT) * 32u); cfg.dynamicSmemBytes = Lay.total;
+    // every CTA must be resident at once, or the grid barrier cannot be passed
+    int fit = 0;
+    if (S > 1) {
+        int clusters = 0;
+        if (CSB_SPMM_DISPATCH(max_loop_clusters, MT, NT, &clusters, &cfg) != cudaSuccess) { cudaGetLastError(); return 1; }
+        fit = clusters * S;
+    } else {
+        fit = A0->sm_count;                                  // one CTA of this size per SM
+    }
+    if (n_ctas > fit) return 1;
+    if ((unsigned long long)2 * (unsigned long long)R.T * R.L * n_ctas >= (1ull << 32)) return 1;   // the barrier counts arrivals in 32 bits
+    CSB_CUDA(cudaMemsetAsync(R.gbar, 0, 4, st));
+    // a launch that is refused (a grid that cannot be co-resident after all) is no error: the caller issues the steps
+    if (CSB_SPMM_DISPATCH(launch_loop_kernel, MT, NT, &cfg, a, lp) != cudaSuccess) { cudaGetLastError(); return 1; }
     return CSB_OK;
 }
 

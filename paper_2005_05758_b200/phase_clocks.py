@@ -2,6 +2,7 @@
 
     python -m paper_2005_05758_b200.phase_clocks rnn   [cfg1 cfg2 cfg3 cfg5]
     python -m paper_2005_05758_b200.phase_clocks panel [4 8 16 25]
+    python -m paper_2005_05758_b200.phase_clocks loop  [cfgN:batch ...]      (default cfg5:32 cfg3:8: the one-launch time loop at batch)
     python -m paper_2005_05758_b200.phase_clocks spmm  [rate:batch | cfgN:batch ...]   (default 4:8 4:32 25:8; cfgN = first layer of that config)
 
 Builds libcsb_clocks.so beside the normal library with -DCSB_PHASE_CLOCKS -DCSB_PANEL_CLOCKS (see
@@ -106,7 +107,9 @@ def panel(rates):
 SPMM_PHASES = ["set-up, first copies, wait for the work in front", "waiting for weights", "passing tiles, waiting for the item's tile",
                "row map, operand loads, tensor instructions", "ring bookkeeping, item headers", "tiles behind the last item",
                "waiting for the CTA's other warps", "accumulators to shared memory", "sums over the warps of a block-row",
-               "waiting for the cluster's other CTAs", "sums over the ranges, store", "until the cluster's CTAs have read"]
+               "waiting for the cluster's other CTAs", "sums over the ranges, store", "until the cluster's CTAs have read",
+               "(time loop) grid barrier behind the product pass", "(time loop) gate arithmetic", "(time loop) grid barrier behind the gates",
+               "(time loop) next pass's first weights out"]
 
 
 def spmm(cases):
@@ -126,11 +129,11 @@ def spmm(cases):
         for i in range(6):
             binding.csb_spmm(As[i % 3], X, Y)
             torch.cuda.synchronize()
-        ck = np.zeros((1 << 16, 12), np.int64)
+        ck = np.zeros((1 << 16, 16), np.int64)
         n = binding.lib.csb_debug_spmm_clocks(C.c_void_p(ck.ctypes.data), 1 << 16)
         ck = ck[:n].astype(np.float64)
         wpc = 32 if int(B) <= 8 else 16
-        per_cta = ck.reshape(-1, wpc, 12)
+        per_cta = ck.reshape(-1, wpc, 16)
         slow = per_cta[np.argmax(per_cta.sum(axis=2).max(axis=1))]
         last = ck[np.argmax(ck[:, :6].sum(axis=1))]      # the warp that reaches the end of its items last
         print("%s batch %s: %d warps (%d per CTA); cycles per phase, last pass of 32 batch columns"
@@ -143,6 +146,39 @@ def spmm(cases):
             a.free()
 
 
+def loop(names):
+    """The one-launch time loop of the batched recurrent path: cycles per phase and pass (layer and step)."""
+    import workloads
+    torch, binding = _load()
+    for case in names:
+        name, B = case.split(":")
+        w = workloads.CONFIGS[name](B=int(B), T=32)
+        mats = [binding.csb_encode(m.dense, m.block_r, m.block_c, m.row_keep, m.col_keep, m.val_dtype, 0) for m in w.layers]
+        L, B, H, T = len(w.layers), w.B, w.hidden_size, w.T
+        x = torch.from_numpy(w.x).cuda()
+        y = torch.empty((T, B, H), device="cuda")
+        hT = torch.empty((L, B, H), device="cuda")
+        cT = torch.empty((L, B, H), device="cuda")
+        for _ in range(3):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            if w.cell == "lstm":
+                binding.csb_lstm_forward(mats, None, x, None, None, y, hT, cT, 0)
+            else:
+                binding.csb_gru_forward(mats, None, x, None, y, hT, 0)
+            b.record()
+            torch.cuda.synchronize()
+        ck = np.zeros((1 << 16, 16), np.int64)
+        n = binding.lib.csb_debug_spmm_clocks(C.c_void_p(ck.ctypes.data), 1 << 16)
+        ck = ck[:n].astype(np.float64) / (T * L)
+        print("%s batch %d: T=%d, %d warps, %.2f us per step (instrumented); cycles per phase and pass" % (name, B, T, n, a.elapsed_time(b) * 1e3 / T))
+        for i, nm in enumerate(SPMM_PHASES):
+            print("   %-52s mean %8.0f  min %8.0f  max %8.0f" % (nm, ck[:, i].mean(), ck[:, i].min(), ck[:, i].max()))
+        print("   %-52s mean %8.0f" % ("all phases", ck.sum(axis=1).mean()))
+        for m in mats:
+            m.free()
+
+
 if __name__ == "__main__":
     what = sys.argv[1] if len(sys.argv) > 1 else "rnn"
     rest = sys.argv[2:]
@@ -152,5 +188,7 @@ if __name__ == "__main__":
         panel(rest or ["4", "25"])
     elif what == "spmm":
         spmm(rest or ["4:8", "4:32", "25:8"])
+    elif what == "loop":
+        loop(rest or ["cfg5:32", "cfg3:8"])
     else:
         raise SystemExit(__doc__)

@@ -169,6 +169,23 @@ def test_step_by_step_packed_inputs_equal_the_fp32_buffers(monkeypatch, cell, B,
         assert np.array_equal(ca, cb)
 
 
+@pytest.mark.parametrize("cell,B,I,H,L,br", [("lstm", 32, 153, 512, 2, 32), ("lstm", 16, 40, 48, 2, 16), ("gru", 16, 70, 512, 2, 32),
+                                             ("gru", 8, 300, 512, 1, 32), ("lstm", 24, 64, 256, 3, 64)])
+def test_one_launch_time_loop_equals_the_launches(monkeypatch, cell, B, I, H, L, br):
+    # CSB_RNN_STEP_LOOP=1: all steps of all layers in one cooperative launch of the product kernel
+    # (product pass, grid barrier, gates, grid barrier); the same arithmetic in the same order
+    w = workloads.make_rnn_workload(34, cell, I, H, L, br, br, "lognormal", rate=4.0, T=9, B=B, w_std=0.15,
+                                    bias_std=0.2, state_std=0.4)
+    ya, ha, ca = check(w)
+    monkeypatch.setenv("CSB_RNN_STEP_LOOP", "1")
+    yb, hb, cb = check(w)
+    assert np.array_equal(ya, yb) and np.array_equal(ha, hb)
+    if cell == "lstm":
+        assert np.array_equal(ca, cb)
+    yc, hc, cc = run(w, chunks=[(0, 4), (4, 9)])
+    assert np.array_equal(ya, yc) and np.array_equal(ha, hc)
+
+
 @pytest.mark.parametrize("B,I,H,L,br,bc", [(16, 40, 48, 2, 16, 16), (20, 39, 100, 1, 32, 32), (33, 70, 192, 2, 64, 32), (8, 300, 512, 1, 32, 32)])
 def test_gru_batch_runs_step_by_step_on_tensor_cores(B, I, H, L, br, bc):
     # GRU from batch 16 (from batch 8 for layers of 100 k weights and more): one product over 2B rows ([u ; 0] and [0 ; h]) keeps the candidate's two parts apart
