@@ -164,18 +164,11 @@ __global__ void __launch_bounds__(1024, 1) csb_panel_kernel(const __grid_constan
         if (s < slots) { done[s] = 0u; issued[s] = 0u; }
         if (s == slots) *s_dead = 0u;
         mbar_fence_init();
-        // the bookkeeping first (everything else waits for it), then the values, then x, which
-        // may still be being written by the kernel in front
+        // the bookkeeping first, then x (the gather of the inputs, which everything else waits for, needs
+        // both; x may still be being written by the kernel in front), then the values
         if (s == slots) {
             mbar_expect_tx(metabar, meta_bytes);
             bulk_g2s(smem + L.meta, panel, meta_bytes, metabar);
-        }
-        __syncwarp(slots + 2u >= 32u ? 0xffffffffu : (1u << (slots + 2u)) - 1u);
-        if (s < slots && s < n_stages) {
-            const uint32_t bytes = min(SB, value_bytes - (s << a.log2_stage));
-            issued[s] = 1u;
-            mbar_expect_tx(&full[s], bytes);
-            bulk_g2s(ring + ((size_t)s << a.log2_stage), values + ((size_t)s << a.log2_stage), bytes, &full[s]);
         }
         if (s == slots + 1u && x_bulk) {
             grid_dependency_wait();
@@ -183,6 +176,13 @@ __global__ void __launch_bounds__(1024, 1) csb_panel_kernel(const __grid_constan
             mbar_expect_tx(xbar, xb);
             for (uint32_t off = 0; off < xb; off += 16384u)
                 bulk_g2s(smem + L.xs + off, reinterpret_cast<const uint8_t*>(a.x) + off, min(16384u, xb - off), xbar);
+        }
+        __syncwarp(slots + 2u >= 32u ? 0xffffffffu : (1u << (slots + 2u)) - 1u);
+        if (s < slots && s < n_stages) {
+            const uint32_t bytes = min(SB, value_bytes - (s << a.log2_stage));
+            issued[s] = 1u;
+            mbar_expect_tx(&full[s], bytes);
+            bulk_g2s(ring + ((size_t)s << a.log2_stage), values + ((size_t)s << a.log2_stage), bytes, &full[s]);
         }
     }
     for (int i = threadIdx.x; i < W * a.max_rows; i += blockDim.x) zs_all[i] = 0.f;

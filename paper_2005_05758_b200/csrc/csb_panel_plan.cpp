@@ -41,13 +41,17 @@ static inline int panel_item_steps(int mi, int n) {
     const int gw = 32 >> panel_item_logg(mi), S = gw >> log2_ceil(mi);
     return ((n >> 3) + S - 1) / S;
 }
-// Modelled issue slots, from instruction counts of the kernel on matrices with a fixed number
-// of kept lines per block: a fixed part per bundle, and per member its loop steps, remainder
-// columns and joining shuffles.
-constexpr double kPanelBundleFixed = 110.0;
+// Modelled time of a bundle: a fixed part, and per member its loop steps, remainder columns and
+// joining shuffles.  The shape follows the kernel's instruction counts (110 fixed, 28 per step), but
+// the two weights are fitted to measured times of the 8192 x 8192 sweep: what a CTA's time follows is
+// the number of its bundles far more than their length (with the instruction counts as weights the
+// CTAs of one product finished between 5.1 and 8.2 us after their gather; 4x: 11.2 -> 10.35 us,
+// 8x: 8.3 -> 7.65, 25x: 6.0 -> 5.75 with the fitted ones).  CSB_PANEL_COST_FIXED / _STEP override them.
+static const double kPanelBundleFixed = getenv("CSB_PANEL_COST_FIXED") ? atof(getenv("CSB_PANEL_COST_FIXED")) : 55.0;
+static const double kPanelStep = getenv("CSB_PANEL_COST_STEP") ? atof(getenv("CSB_PANEL_COST_STEP")) : 4.0;
 static double panel_member_cost(int mi, int n) {
     const int gw = 32 >> panel_item_logg(mi), S = gw >> log2_ceil(mi);
-    return 28.0 * panel_item_steps(mi, n) + ((n & 7) ? 34.0 : 0.0) + 8.0 * log2_ceil(S);
+    return kPanelStep * panel_item_steps(mi, n) + ((n & 7) ? 34.0 : 0.0) + 8.0 * log2_ceil(S);
 }
 // Cost of an item as seen by the row cut: its share of a bundle.
 static double panel_item_cost(int mi, int n) {
