@@ -149,6 +149,7 @@ def spmm(cases):
 def loop(names):
     """The one-launch time loop of the batched recurrent path: cycles per phase and pass (layer and step)."""
     import workloads
+    os.environ["CSB_RNN_STEP_LOOP"] = "1"          # the loop is not the default path
     torch, binding = _load()
     for case in names:
         name, B = case.split(":")
